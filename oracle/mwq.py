@@ -1,0 +1,185 @@
+"""Oracle: Matryoshka Weight Quantization (Section 3.3.1).  Test infrastructure only.
+
+Calibration-free form: the paper optimises the zero points and scales against activations X
+(Eq. 3, Eq. 5) and compensates block errors through a Hessian factor (Algorithm 1).  No
+calibration data exists here; with X proportional to the identity the Hessian factor is diagonal
+and the compensation update is zero, so what is left is Eq. 2 followed by the one-bit residual
+steps of Eq. 4, which is what this file writes out.
+
+Readings taken where the paper is silent (each also listed in the design notes):
+* ``round`` in Eq. 2 is round-half-to-even; the base code is clamped to [0, 2^b1 - 1].
+* Zero point is real-valued (Eq. 2 has z in R); it is stored as ``lo = -z*s``, an fp16 value rounded
+  toward -inf from the group minimum, and the scale ``s1`` is the fp16 value rounded toward +inf
+  from (max - lo)/(2^b1 - 1), so the base grid always covers the group.  s1 == 0 becomes 2^-14.
+* Eq. 4 with Q in {+1,-1}: Q = sign of the residual, sign(0) = +1.
+* Residual scales are tied, s_j = s1 * 2^-(j+1) for the j-th extra bit (the expected absolute
+  residual of a uniform residual on a cell of width s_{j-1}*2), which makes the b-bit code the
+  b most significant bits of the top-width code.
+* The reconstruction rule printed below Eq. 5 has a garbled summation index; it is read as
+  W_hat_{b_k} = W_hat_{b_1} + sum_i s_{b_i} Q_{W_{b_i}}.
+* Width lists that skip widths (2,4,8) run every one-bit step internally and expose only the
+  listed widths.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Sequence, Tuple
+
+import numpy as np
+
+F32 = np.float32
+
+
+def fp16_round_down(x: np.ndarray) -> np.ndarray:
+    """Largest fp16-representable value <= x, returned as fp32."""
+    x = np.asarray(x, dtype=F32)
+    h = x.astype(np.float16)
+    too_big = h.astype(F32) > x
+    h = np.where(too_big, np.nextafter(h, np.float16(-np.inf)), h).astype(np.float16)
+    return h.astype(F32)
+
+
+def fp16_round_up(x: np.ndarray) -> np.ndarray:
+    """Smallest fp16-representable value >= x, returned as fp32."""
+    x = np.asarray(x, dtype=F32)
+    h = x.astype(np.float16)
+    too_small = h.astype(F32) < x
+    h = np.where(too_small, np.nextafter(h, np.float16(np.inf)), h).astype(np.float16)
+    return h.astype(F32)
+
+
+@dataclass
+class MWQTensor:
+    """Nested code of one weight matrix.
+
+    code : uint8 [rows, cols], the top-width code (``bits[-1]`` significant bits).
+    s1   : fp32 [rows, cols/g], base scale (an fp16-representable value).
+    lo   : fp32 [rows, cols/g], base offset = -z*s of Eq. 2 (an fp16-representable value).
+    """
+    code: np.ndarray
+    s1: np.ndarray
+    lo: np.ndarray
+    bits: Tuple[int, ...]
+    group_size: int
+
+    @property
+    def top(self) -> int:
+        return self.bits[-1]
+
+    @property
+    def b1(self) -> int:
+        return self.bits[0]
+
+
+def check_bits(bits: Sequence[int]) -> None:
+    assert len(bits) >= 1 and bits[0] >= 1 and bits[-1] <= 8
+    assert all(bits[i] < bits[i + 1] for i in range(len(bits) - 1)), "widths must ascend"
+
+
+def quantize(W: np.ndarray, bits: Sequence[int], group_size: int) -> MWQTensor:
+    """MWQ of W [rows, cols] with groups of ``group_size`` along the input (column) axis.
+
+    Step 1 is the per-group asymmetric b1-bit quantization of Eq. 2; steps 2.. are the binary
+    residual quantization of Eq. 4, one bit per step up to the top width.  All arithmetic is fp32
+    with one rounding per operation (numpy does not contract a*b+c).
+    """
+    check_bits(bits)
+    W = np.ascontiguousarray(W, dtype=F32)
+    rows, cols = W.shape
+    g = group_size
+    assert cols % g == 0
+    b1, top = bits[0], bits[-1]
+    Wg = W.reshape(rows, cols // g, g)
+
+    wmin = Wg.min(axis=2)
+    wmax = Wg.max(axis=2)
+    lo = fp16_round_down(wmin)
+    s1 = fp16_round_up((wmax - lo) / F32(2 ** b1 - 1))
+    s1 = np.where(s1 == 0, F32(2.0 ** -14), s1).astype(F32)
+
+    lo_b = lo[:, :, None]
+    s1_b = s1[:, :, None]
+    # Eq. 2: Q = round(W/s + z) with z = -lo/s, evaluated as round((W - lo)/s)
+    Q = np.clip(np.rint((Wg - lo_b) / s1_b), F32(0), F32(2 ** b1 - 1)).astype(F32)
+    What = (lo_b + Q * s1_b).astype(F32)              # (Q - z) * s
+    R = (Wg - What).astype(F32)
+    code = Q.astype(np.int32)
+    for j in range(1, top - b1 + 1):
+        s_j = (s1_b * F32(2.0 ** -(j + 1))).astype(F32)   # exact: power-of-two multiple
+        bit = R >= 0                                       # Eq. 4, Q in {+1,-1}
+        What = (What + np.where(bit, s_j, -s_j)).astype(F32)
+        R = (Wg - What).astype(F32)
+        code = code * 2 + bit.astype(np.int32)
+    assert code.min() >= 0 and code.max() < (1 << top)
+    return MWQTensor(code.reshape(rows, cols).astype(np.uint8), s1, lo, tuple(bits), g)
+
+
+def slice_code(q: MWQTensor, b: int) -> np.ndarray:
+    """Code at width b: the b most significant bits of the top-width code (matryoshka nesting)."""
+    assert q.b1 <= b <= q.top
+    return (q.code >> (q.top - b)).astype(np.uint8)
+
+
+def dequantize(q: MWQTensor, b: int) -> np.ndarray:
+    """fp64 weights at width b by the paper's additive rule (below Eq. 5):
+    W_hat_b = (Q_b1 - z) * s_b1 + sum over the extra bits j = 1..b-b1 of s_j * (+1 or -1)."""
+    assert q.b1 <= b <= q.top
+    rows, cols = q.code.shape
+    g = q.group_size
+    code = q.code.reshape(rows, cols // g, g).astype(np.int64)
+    s1 = q.s1.astype(np.float64)[:, :, None]
+    lo = q.lo.astype(np.float64)[:, :, None]
+    base = code >> (q.top - q.b1)
+    W = lo + base.astype(np.float64) * s1
+    for j in range(1, b - q.b1 + 1):
+        bit = (code >> (q.top - q.b1 - j)) & 1
+        W = W + np.where(bit == 1, 1.0, -1.0) * (s1 * 2.0 ** -(j + 1))
+    return W.reshape(rows, cols)
+
+
+def dequantize_closed_form(q: MWQTensor, b: int) -> np.ndarray:
+    """Same weights from the sliced integer code alone: with q_b = code >> (top-b) and
+    s_b = s1 / 2^(b-b1), W_hat_b = (lo - s1/2) + s_b * (q_b + 1/2), the midpoint of cell q_b of a
+    uniform grid of 2^b cells.  Used to pin ``dequantize`` (two independent formulas)."""
+    rows, cols = q.code.shape
+    g = q.group_size
+    qb = slice_code(q, b).reshape(rows, cols // g, g).astype(np.float64)
+    s1 = q.s1.astype(np.float64)[:, :, None]
+    lo = q.lo.astype(np.float64)[:, :, None]
+    sb = s1 / 2.0 ** (b - q.b1)
+    return ((lo - s1 / 2) + sb * (qb + 0.5)).reshape(rows, cols)
+
+
+def segments(bits: Sequence[int]) -> List[Tuple[int, int]]:
+    """The nested store as segments: (shift, width) of each segment inside the top-width code.
+    Segment 0 holds the b1 base bits; segment j the bits[j]-bits[j-1] bits added next."""
+    check_bits(bits)
+    top = bits[-1]
+    out, prev = [], 0
+    for b in bits:
+        out.append((top - b, b - prev))
+        prev = b
+    return out
+
+
+def segment_values(q: MWQTensor) -> List[np.ndarray]:
+    return [((q.code >> sh) & ((1 << w) - 1)).astype(np.uint8) for sh, w in segments(q.bits)]
+
+
+def segments_read(width_idx: int) -> List[int]:
+    """Segments an expert call at ``bits[width_idx]`` reads: all up to and including its own."""
+    return list(range(width_idx + 1))
+
+
+def segment_use_counts(width_idx_of_requests: Sequence[int], n_bits: int) -> List[int]:
+    """How many requests on one expert read each segment (Section 3.4's plane-reuse example)."""
+    counts = [0] * n_bits
+    for k in width_idx_of_requests:
+        for j in segments_read(k):
+            counts[j] += 1
+    return counts
+
+
+def nested_store_bits_per_weight(bits: Sequence[int]) -> int:
+    """Bits stored per weight by the nested store: the top width only, whatever the list is."""
+    return sum(w for _, w in segments(bits))
