@@ -1,0 +1,176 @@
+/*
+ * d2moe.h - C ABI of the B200 (sm_100a) dual-routed MoE layer over matryoshka-weight-quantized
+ * (MWQ) experts, after "D2MoE: Dual Routing and Dynamic Scheduling for Efficient On-Device
+ * MoE-based LLM Serving" (Sections 3.2 and 3.3).
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers are host
+ *     memory.  The caller owns every buffer; the library allocates nothing and keeps no state
+ *     between calls (unless an entry point's comment says otherwise).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and the
+ *     call returns without synchronising.
+ *   - The return value reports what the host can see before and at launch: null pointers, bad
+ *     configuration or shapes, short buffers, a failed launch.  Nothing is launched when an
+ *     argument check fails.  Anomalies only the device can see (non-finite router logits, a bounded
+ *     wait that ran out) are OR-ed into the optional `device_status` word, which the caller reads
+ *     after its own synchronisation.  No call aborts, traps or throws.
+ *   - bf16 tensors are passed as `const void*` to 16-bit elements (upper half of an fp32).
+ */
+#ifndef D2MOE_H
+#define D2MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    D2MOE_OK = 0,
+    D2MOE_ERR_NULL = 1,        /* a required pointer is NULL                                  */
+    D2MOE_ERR_CONFIG = 2,      /* d2moe_config is inconsistent                                */
+    D2MOE_ERR_SHAPE = 3,       /* a size does not fit the configuration                       */
+    D2MOE_ERR_UNSUPPORTED = 4, /* valid but not built (e.g. scale_mode 1)                     */
+    D2MOE_ERR_WORKSPACE = 5,   /* workspace or output buffer too small                        */
+    D2MOE_ERR_CUDA = 6,        /* a CUDA runtime call or launch failed                        */
+    D2MOE_ERR_TIMEOUT = 7,     /* device_status bit: a bounded device-side wait ran out       */
+    D2MOE_ERR_NONFINITE = 8    /* device_status bit: a router logit was NaN or infinite       */
+} d2moe_status;
+
+/* bits set in *device_status */
+#define D2MOE_DEV_NONFINITE 0x1
+#define D2MOE_DEV_TIMEOUT   0x2
+#define D2MOE_DEV_BAD_INDEX 0x4  /* a supplied routing index was out of range and was skipped */
+
+/* kernel_path values */
+#define D2MOE_PATH_AUTO      0   /* tensor-core grouped kernels where the shape allows          */
+#define D2MOE_PATH_CUDA_CORE 1   /* plain fp32 CUDA-core kernels (any supported shape)          */
+#define D2MOE_PATH_TENSOR    2   /* tcgen05 grouped kernels; D2MOE_ERR_UNSUPPORTED if not possible */
+
+/*
+ * One MoE layer.  Candidate widths {b_k} of Section 3.3.1 are `bits[0..n_bits-1]`, ascending,
+ * 1 <= bits[0], bits[n_bits-1] <= 8; every expert matrix is stored once at the top width and read
+ * at any listed width (the nested store).  `group_size` is g of Eq. 2 (groups run along the input
+ * dimension of each matrix) and must be a multiple of 32.  Experts are SwiGLU FFNs without bias:
+ * gate and up projections [d_ffn, d_model], down projection [d_model, d_ffn].
+ */
+typedef struct {
+    int32_t d_model, d_ffn, n_experts, top_k, n_shared, group_size;
+    int32_t n_bits, bits[8];
+    int32_t renormalize;   /* 1: weights of the selected experts are divided by their sum       */
+    int32_t scale_mode;    /* 0: tied residual scales s_j = s1 / 2^(j+1).  1 (free per-level
+                              scales of Eq. 5) is not built: D2MOE_ERR_UNSUPPORTED               */
+    int32_t kernel_path;   /* D2MOE_PATH_*                                                      */
+    int32_t reserved[3];   /* must be 0                                                         */
+} d2moe_config;
+
+const char* d2moe_status_string(d2moe_status s);
+
+/* Checks a configuration on the host. */
+d2moe_status d2moe_check_config(const d2moe_config* cfg);
+
+/*
+ * Size in bytes of the packed form of one [rows, cols] matrix (cols % group_size == 0).
+ * total = header + code bytes + metadata bytes; code_bytes and meta_bytes (either may be NULL) give
+ * the split: code_bytes = rows_padded*cols*bits[n_bits-1]/8 when every segment width is 1, 2, 4 or 8
+ * bits (segments of 3 / 5..7 bits are stored in 4 / 8), metadata = one (fp16 scale, fp16 offset)
+ * pair per row and group.  The nested store costs the top width only, whatever n_bits is.
+ */
+d2moe_status d2moe_packed_bytes(const d2moe_config* cfg, int64_t rows, int64_t cols,
+                                size_t* total_bytes, size_t* code_bytes, size_t* meta_bytes);
+
+/*
+ * MWQ quantization and packing of one matrix (Section 3.3.1: Eq. 2 base step at bits[0], then one
+ * binary residual step of Eq. 4 per extra bit up to bits[n_bits-1], tied scales, calibration-free).
+ *   W       device, fp32 [rows, cols] row-major, finite, |W| < 65504
+ *   packed  device, packed_bytes >= d2moe_packed_bytes(); 256-byte aligned; layout is private to
+ *           this library (bit-plane segments tiled for the expert kernels) and versioned by a header.
+ * The b-bit code of a weight is the b most significant bits of its top-width code.
+ */
+d2moe_status d2moe_pack_mwq(const d2moe_config* cfg, const float* W, int64_t rows, int64_t cols,
+                            void* packed, size_t packed_bytes, void* stream);
+
+/*
+ * Test hook: canonical codes of a packed matrix at width `bits` (bits[0] <= bits <= top width, need
+ * not be a listed width): codes[r*cols + c] = top-width code >> (top - bits), one byte per weight.
+ * scale / offset (either may be NULL): device fp32 [rows, cols/group_size], the stored s1 and lo.
+ */
+d2moe_status d2moe_unpack_codes(const d2moe_config* cfg, const void* packed, int64_t rows,
+                                int64_t cols, int bits, uint8_t* codes, float* scale, float* offset,
+                                void* stream);
+
+/* Workspace (device bytes) d2moe_route and d2moe_moe_forward need for up to max_tokens tokens. */
+size_t d2moe_workspace_bytes(const d2moe_config* cfg, int64_t max_tokens);
+
+/*
+ * Dual routing of T tokens (Section 3.2; the models of Section 5.1) and grouping by
+ * (expert, width): the histogram of the grouping is B_{j,k} of Section 3.4.3.
+ * Inputs (device): x bf16 [T, d_model]; exactly one of gate_w (bf16 [E, d_model]) and logits
+ * (fp32 [T, E]); exactly one of bit_w (bf16 [E, n_bits, d_model], one linear bit-width router per
+ * expert) and forced_bit_idx (int8 [T, top_k], a width index per selected expert).
+ * Outputs (device, all required):
+ *   topk_idx  int32 [T, top_k]  selected experts, by descending logit, ties to the lower index
+ *   topk_w    fp32  [T, top_k]  softmax weight of each (renormalised if cfg->renormalize)
+ *   bit_idx   int8  [T, top_k]  width index: argmax of the expert's bit-width router, ties to the
+ *                               lower width
+ *   perm      int32 [T*top_k]   sorted position -> assignment id a = t*top_k + slot; assignments
+ *                               are sorted by (expert, width index), then by a (stable)
+ *   inv_perm  int32 [T*top_k]   assignment id -> sorted position
+ *   group_off int32 [E*n_bits+1] exclusive prefix sum of the (expert, width) histogram
+ * Logits are fp32 sums in a fixed order (32 strided partial sums of fused multiply-adds, then a
+ * butterfly reduction), so the integer outputs are reproducible bit for bit.
+ */
+d2moe_status d2moe_route(const d2moe_config* cfg, int64_t T,
+                         const void* x_bf16, const void* gate_w_bf16, const float* logits,
+                         const void* bit_w_bf16, const int8_t* forced_bit_idx,
+                         int32_t* topk_idx, float* topk_w, int8_t* bit_idx,
+                         int32_t* perm, int32_t* inv_perm, int32_t* group_off,
+                         int32_t* device_status, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+typedef struct {
+    const void* gate_w_bf16;        /* device bf16 [E, d_model] or NULL */
+    const float* logits;            /* device fp32 [T, E] or NULL       */
+    const void* bit_w_bf16;         /* device bf16 [E, n_bits, d_model] or NULL */
+    const int8_t* forced_bit_idx;   /* device int8 [T, top_k] or NULL   */
+} d2moe_route_in;
+
+typedef struct {                    /* outputs of an earlier d2moe_route on the same stream */
+    const int32_t* topk_idx; const float* topk_w; const int8_t* bit_idx;
+    const int32_t* perm; const int32_t* inv_perm; const int32_t* group_off;
+} d2moe_route_out;
+
+/*
+ * The whole layer: y_t = sum over selected experts of w * Expert_{e,b}(x_t), each expert run on its
+ * weights dequantized at the routed width b (Fig. 1; Section 3.3.1 reconstruction rule), plus the
+ * shared experts (always on, top width, weight 1).  Expert_{e,b}(x) = Wd_b (silu(Wg_b x) * (Wu_b x)).
+ *   x_bf16    device bf16 [T, d_model]
+ *   expert_w  HOST array of 3*(n_experts+n_shared) device pointers to packed matrices, order
+ *             [expert][gate, up, down], shared experts last; read during the call only
+ *   in        routing inputs (see d2moe_route); ignored when `pre` is given
+ *   pre       optional: routing already computed by d2moe_route (same T, same stream order)
+ *   y_bf16    device bf16 [T, d_model], overwritten
+ * Arithmetic: weights dequantized to 16-bit floating point in registers, fp32 accumulation, bf16
+ * output (round to nearest even).  T == 0 is a no-op.
+ */
+d2moe_status d2moe_moe_forward(const d2moe_config* cfg, int64_t T, const void* x_bf16,
+                               const void* const* expert_w, const d2moe_route_in* in,
+                               const d2moe_route_out* pre, void* y_bf16, int32_t* device_status,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One layer of the FFN-only stack used by the multi-layer benchmark configuration (not in the
+ * paper): x <- bf16( x + MoE( bf16( x / sqrt(mean(x^2) + eps) ) ) ), unit gain.  x_bf16 is updated
+ * in place; xn_bf16 is a caller-provided bf16 [T, d_model] scratch that receives the normalised
+ * input.  Other arguments as d2moe_moe_forward.
+ */
+d2moe_status d2moe_stack_layer(const d2moe_config* cfg, int64_t T, void* x_bf16, void* xn_bf16,
+                               float eps, const void* const* expert_w, const d2moe_route_in* in,
+                               int32_t* device_status, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D2MOE_H */

@@ -1,0 +1,146 @@
+// Shared declarations of the d2moe library: packed-weight layout, workspace carving, launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/d2moe.h"
+
+#define D2MOE_MAX_SEG 8
+#define D2MOE_TILE_ROWS 64          // rows per packed block
+#define D2MOE_HEADER_BYTES 256
+#define D2MOE_MAGIC 0x4D32444Du     // "MD2M"
+#define D2MOE_LAYOUT_VERSION 1u
+#define D2MOE_MAX_EXPERTS 320       // routed + shared
+
+// ------------------------------------------------------------------------------------------------
+// Packed layout of one [rows, cols] matrix.
+//
+//   blob   = header (256 B) | block(rt = 0, G = 0) | block(0, 1) | ... | block(n_rt-1, n_groups-1)
+//   block  = meta | segment 0 | segment 1 | ...           (64 rows x one group of g input columns)
+//   meta   = 64 x (fp16 s1, fp16 lo), row r at byte 4r
+//   segment j holds, for each of the 64 rows, the g codes of that segment (bits
+//   [shift_j + w_j - 1 : shift_j] of the top-width code) stored sw_j in {1,2,4,8} bits each, i.e.
+//   g*sw_j/8 bytes per row, cut in chunks of cs_j = min(16, g*sw_j/8) bytes; chunk c of row r lies
+//   at byte (c*64 + r)*cs_j of the segment, so 32 consecutive rows read 32 consecutive chunks.
+//   Inside a row's bytes, 32-bit word m holds 32/sw codes: with per = 16/sw, the code of element
+//   k = 2*(m*per + e) + h (h = 0,1) sits at bit 16*h + sw*e.  (One AND with a mask that has the
+//   same field in both 16-bit halves therefore yields the pair (k, k+1) as two 16-bit lanes.)
+//
+// A call at width bits[kk] needs meta and segments 0..kk of a block: one contiguous prefix.
+// ------------------------------------------------------------------------------------------------
+struct PackLayout {
+    int rows, cols, g, n_groups, rows_pad, n_rt;
+    int n_seg, top, b1;
+    int seg_w[D2MOE_MAX_SEG];      // logical width of segment j
+    int seg_sw[D2MOE_MAX_SEG];     // storage width (1, 2, 4, 8)
+    int seg_shift[D2MOE_MAX_SEG];  // position of the segment inside the top-width code
+    int seg_cs[D2MOE_MAX_SEG];     // chunk size in bytes
+    int seg_off[D2MOE_MAX_SEG + 1];// byte offset of segment j inside a block; [n_seg] = block size
+    int block_bytes;
+};
+
+struct PackHeader {
+    uint32_t magic, version;
+    int32_t rows, cols, g, n_bits;
+    int32_t bits[8];
+    uint32_t s1_max_bits;          // bit pattern of the largest fp32 s1 in the matrix
+    uint32_t pad[49];
+};
+static_assert(sizeof(PackHeader) == D2MOE_HEADER_BYTES, "header size");
+
+__host__ __device__ inline int d2moe_storage_width(int w) { return w <= 1 ? 1 : (w <= 2 ? 2 : (w <= 4 ? 4 : 8)); }
+
+__host__ __device__ inline void d2moe_make_layout(PackLayout& L, const int* bits, int n_bits, int g,
+                                                  long long rows, long long cols) {
+    L.rows = (int)rows; L.cols = (int)cols; L.g = g; L.n_groups = (int)(cols / g);
+    L.rows_pad = (int)((rows + D2MOE_TILE_ROWS - 1) / D2MOE_TILE_ROWS * D2MOE_TILE_ROWS);
+    L.n_rt = L.rows_pad / D2MOE_TILE_ROWS;
+    L.n_seg = n_bits; L.top = bits[n_bits - 1]; L.b1 = bits[0];
+    int off = D2MOE_TILE_ROWS * 4, prev = 0;
+    for (int j = 0; j < D2MOE_MAX_SEG; ++j) {
+        if (j < n_bits) {
+            L.seg_w[j] = bits[j] - prev; prev = bits[j];
+            L.seg_sw[j] = d2moe_storage_width(L.seg_w[j]);
+            L.seg_shift[j] = L.top - bits[j];
+            int row_bytes = g * L.seg_sw[j] / 8;
+            L.seg_cs[j] = row_bytes < 16 ? row_bytes : 16;
+            L.seg_off[j] = off;
+            off += D2MOE_TILE_ROWS * row_bytes;
+        } else {
+            L.seg_w[j] = L.seg_sw[j] = L.seg_shift[j] = L.seg_cs[j] = 0; L.seg_off[j] = off;
+        }
+    }
+    L.seg_off[n_bits < D2MOE_MAX_SEG ? n_bits : D2MOE_MAX_SEG] = off;
+    if (n_bits == D2MOE_MAX_SEG) L.seg_off[D2MOE_MAX_SEG] = off;
+    L.block_bytes = off;
+}
+
+// Byte offset (inside a block) of the 32-bit word that holds element k of row r in segment j, and
+// the bit position of the element inside that word.
+__host__ __device__ inline int d2moe_elem_word(const PackLayout& L, int j, int r, int k, int* bitpos) {
+    int sw = L.seg_sw[j], per = 16 / sw;
+    int i = k >> 1, h = k & 1;
+    int m = i / per, e = i - m * per;
+    *bitpos = 16 * h + sw * e;
+    int ob = 4 * m, cs = L.seg_cs[j];
+    int c = ob / cs, within = ob - c * cs;
+    return L.seg_off[j] + (c * D2MOE_TILE_ROWS + r) * cs + within;
+}
+
+__host__ __device__ inline size_t d2moe_block_offset(const PackLayout& L, int rt, int G) {
+    return (size_t)D2MOE_HEADER_BYTES + ((size_t)rt * L.n_groups + G) * (size_t)L.block_bytes;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Problem description handed to the kernels (by value).
+// ------------------------------------------------------------------------------------------------
+struct MoeDims {
+    int T, d, F, E, k, n_shared, g, K;   // K = n_bits
+    int bits[8];
+    int A;        // routed assignments T*k
+    int A_tot;    // A + n_shared*T
+    int renormalize;
+};
+
+struct ExpertPtrs {                       // [expert][gate, up, down]
+    const uint8_t* w[3 * D2MOE_MAX_EXPERTS];
+};
+
+struct RouteBufs {
+    int32_t* topk_idx; float* topk_w; int8_t* bit_idx;
+    int32_t* perm; int32_t* inv_perm; int32_t* group_off;
+};
+
+// Workspace carving (all offsets 256-byte aligned).
+struct Workspace {
+    size_t total;
+    size_t off_logits, off_keys, off_hist;
+    size_t off_topk_idx, off_topk_w, off_bit_idx, off_perm, off_inv_perm, off_group_off;
+    size_t off_h, off_o, off_status;
+};
+
+void d2moe_carve_workspace(const d2moe_config* cfg, long long max_tokens, Workspace* ws);
+
+// kernels_pack.cu
+cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const float* W, uint8_t* packed,
+                        cudaStream_t st);
+cudaError_t launch_unpack(const PackLayout& L, const uint8_t* packed, int bits, uint8_t* codes,
+                          float* scale, float* offset, cudaStream_t st);
+
+// kernels_route.cu
+cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
+                         const float* logits_in, const __nv_bfloat16* bit_w, const int8_t* forced,
+                         const RouteBufs& R, float* logits_ws, int32_t* keys_ws, int32_t* hist_ws,
+                         int32_t* device_status, cudaStream_t st);
+
+// kernels_ffn_cc.cu  (plain CUDA-core path)
+cudaError_t launch_ffn_cuda_core(const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                                 const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R,
+                                 float* hbuf, float* obuf, int32_t* device_status, cudaStream_t st);
+cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* obuf, int n_split,
+                           const __nv_bfloat16* residual, __nv_bfloat16* y, cudaStream_t st);
+cudaError_t launch_rmsnorm(int T, int d, float eps, const __nv_bfloat16* x, __nv_bfloat16* xn, cudaStream_t st);

@@ -1,0 +1,177 @@
+// Plain CUDA-core expert kernels: every (assignment, output row) is one warp's fp32 dot product over
+// weights dequantized on the fly at the assignment's routed width (Section 3.3.1 reconstruction
+// rule, in its closed form W_hat_b = (lo - s1/2) + s_b (q_b + 1/2), s_b = s1 / 2^(b-b1)).
+// Works for every supported shape; it is the path of last resort and the on-device cross-check of
+// the tensor-core kernels.  Also: the weighted combine (with optional residual) and RMSNorm.
+#include "d2moe_common.cuh"
+
+namespace {
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Resolve assignment id a (routed: a < A; shared experts after) into token, expert, width index.
+__device__ __forceinline__ bool resolve_assignment(const MoeDims& D, const RouteBufs& R, int a, int* t,
+                                                   int* e, int* kk, int32_t* device_status) {
+    if (a < D.A) {
+        *t = a / D.k;
+        *e = R.topk_idx[a];
+        *kk = R.bit_idx[a];
+        if (*e < 0 || *e >= D.E || *kk < 0 || *kk >= D.K) {
+            if (device_status) atomicOr(device_status, D2MOE_DEV_BAD_INDEX);
+            return false;
+        }
+    } else {
+        const int s = (a - D.A) / D.T;
+        *t = (a - D.A) - s * D.T;
+        *e = D.E + s;
+        *kk = D.K - 1;
+    }
+    return true;
+}
+
+// Dot product of packed row `row` of one matrix, read at width index kk, with vector v (length
+// L.cols).  All 32 lanes take part; the result is valid in every lane.
+template <typename VT>
+__device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed, int row, int kk,
+                         const VT* __restrict__ v, int lane) {
+    const int rt = row / D2MOE_TILE_ROWS, r = row - rt * D2MOE_TILE_ROWS;
+    const int b = L.seg_shift[kk];                      // top - bits[kk]
+    const int width = L.top - b;
+    const float inv = 1.0f / (float)(1 << (width - L.b1));
+    float acc = 0.0f;
+    for (int G = 0; G < L.n_groups; ++G) {
+        const uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
+        const __half2 m = reinterpret_cast<const __half2*>(blk)[r];
+        const float s1 = __low2float(m), lo = __high2float(m);
+        const float sb = s1 * inv;
+        const float base = lo - 0.5f * s1;
+        const VT* vg = v + (size_t)G * L.g;
+        for (int i = lane; i < L.g / 2; i += 32) {      // pair (2i, 2i+1)
+            unsigned q0 = 0, q1 = 0;
+            for (int j = 0; j <= kk; ++j) {
+                int bitpos;
+                const int wo = d2moe_elem_word(L, j, r, 2 * i, &bitpos);
+                const uint32_t word = *reinterpret_cast<const uint32_t*>(blk + wo);
+                const unsigned mask = (1u << L.seg_w[j]) - 1u;
+                q0 |= ((word >> bitpos) & mask) << L.seg_shift[j];
+                q1 |= ((word >> (bitpos + 16)) & mask) << L.seg_shift[j];
+            }
+            q0 >>= b; q1 >>= b;
+            const float w0 = fmaf(sb, (float)q0 + 0.5f, base);
+            const float w1 = fmaf(sb, (float)q1 + 0.5f, base);
+            acc = fmaf(w0, to_f32(vg[2 * i]), acc);
+            acc = fmaf(w1, to_f32(vg[2 * i + 1]), acc);
+        }
+    }
+    for (int off = 16; off; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    return acc;
+}
+
+// h[a, r] = silu(Wg_{e,b}[r,:] . x_t) * (Wu_{e,b}[r,:] . x_t);  grid (ceil(F/8), A_tot), 8 warps.
+__global__ void __launch_bounds__(256)
+gateup_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, const __nv_bfloat16* __restrict__ x, RouteBufs R,
+                 float* __restrict__ hbuf, int32_t* device_status) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int a = blockIdx.y;
+    if (row >= D.F) return;
+    int t, e, kk;
+    if (!resolve_assignment(D, R, a, &t, &e, &kk, device_status)) {
+        if (lane == 0) hbuf[(size_t)a * D.F + row] = 0.0f;
+        return;
+    }
+    const __nv_bfloat16* xt = x + (size_t)t * D.d;
+    const float g = row_dot(L, P.w[3 * e + 0], row, kk, xt, lane);
+    const float u = row_dot(L, P.w[3 * e + 1], row, kk, xt, lane);
+    if (lane == 0) hbuf[(size_t)a * D.F + row] = g / (1.0f + expf(-g)) * u;
+}
+
+// o[a, r] = Wd_{e,b}[r,:] . h[a,:];  grid (ceil(d/8), A_tot)
+__global__ void __launch_bounds__(256)
+down_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, RouteBufs R, const float* __restrict__ hbuf,
+               float* __restrict__ obuf, int32_t* device_status) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int a = blockIdx.y;
+    if (row >= D.d) return;
+    int t, e, kk;
+    if (!resolve_assignment(D, R, a, &t, &e, &kk, nullptr)) {
+        if (lane == 0) obuf[(size_t)a * D.d + row] = 0.0f;
+        return;
+    }
+    const float o = row_dot(L, P.w[3 * e + 2], row, kk, hbuf + (size_t)a * D.F, lane);
+    if (lane == 0) obuf[(size_t)a * D.d + row] = o;
+}
+
+// y[t, c] = bf16( residual[t, c] + sum_slot w[t,slot] * o[row(t,slot), c] + sum_shared o[...] )
+// where o may come as n_split partial sums (split-K); row_map (optional) maps an assignment id to
+// its row in obuf.
+__global__ void combine_kernel(MoeDims D, RouteBufs R, const float* __restrict__ obuf, int n_split,
+                               size_t split_stride, const int32_t* __restrict__ row_map,
+                               const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ y) {
+    const int t = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= D.d) return;
+    float acc = residual ? __bfloat162float(residual[(size_t)t * D.d + c]) : 0.0f;
+    float sum = 0.0f;
+    for (int s = 0; s < D.k + D.n_shared; ++s) {
+        const int a = s < D.k ? t * D.k + s : D.A + (s - D.k) * D.T + t;
+        const float w = s < D.k ? R.topk_w[a] : 1.0f;
+        const size_t row = row_map ? (size_t)row_map[a] : (size_t)a;
+        float o = 0.0f;
+        for (int sp = 0; sp < n_split; ++sp) o += obuf[sp * split_stride + row * D.d + c];
+        sum = fmaf(w, o, sum);
+    }
+    y[(size_t)t * D.d + c] = __float2bfloat16_rn(acc + sum);
+}
+
+// xn = bf16( x / sqrt(mean(x^2) + eps) ), fp64 inside so the rounding matches a double-precision
+// evaluation; one block per token.
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(int d, double eps, const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xn) {
+    __shared__ double red[8];
+    const int t = blockIdx.x;
+    double ss = 0.0;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const double v = (double)__bfloat162float(x[(size_t)t * d + i]);
+        ss += v * v;
+    }
+    for (int off = 16; off; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    double tot = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+    const double inv = 1.0 / sqrt(tot / (double)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const double v = (double)__bfloat162float(x[(size_t)t * d + i]) * inv;
+        xn[(size_t)t * d + i] = __float2bfloat16_rn((float)v);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_ffn_cuda_core(const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                                 const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R,
+                                 float* hbuf, float* obuf, int32_t* device_status, cudaStream_t st) {
+    if (D.A_tot == 0) return cudaSuccess;
+    dim3 g1((D.F + 7) / 8, D.A_tot);
+    gateup_cc_kernel<<<g1, 256, 0, st>>>(D, Lgu, P, x, R, hbuf, device_status);
+    dim3 g2((D.d + 7) / 8, D.A_tot);
+    down_cc_kernel<<<g2, 256, 0, st>>>(D, Ld, P, R, hbuf, obuf, device_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* obuf, int n_split,
+                           const __nv_bfloat16* residual, __nv_bfloat16* y, cudaStream_t st) {
+    if (D.T == 0) return cudaSuccess;
+    dim3 grid((D.d + 255) / 256, D.T);
+    combine_kernel<<<grid, 256, 0, st>>>(D, R, obuf, n_split, (size_t)D.A_tot * D.d, nullptr, residual, y);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rmsnorm(int T, int d, float eps, const __nv_bfloat16* x, __nv_bfloat16* xn, cudaStream_t st) {
+    if (T == 0) return cudaSuccess;
+    rmsnorm_kernel<<<T, 256, 0, st>>>(d, (double)eps, x, xn);
+    return cudaGetLastError();
+}

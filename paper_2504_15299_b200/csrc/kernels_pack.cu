@@ -1,0 +1,153 @@
+// MWQ quantization + packing (Section 3.3.1, Eq. 2 and Eq. 4) and the unpack test hook.
+#include "d2moe_common.cuh"
+
+namespace {
+
+constexpr int PACK_THREADS = 256;
+
+__global__ void pack_header_kernel(PackHeader* h, PackLayout L, int n_bits,
+                                   int b0, int b1, int b2, int b3, int b4, int b5, int b6, int b7) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        h->magic = D2MOE_MAGIC; h->version = D2MOE_LAYOUT_VERSION;
+        h->rows = L.rows; h->cols = L.cols; h->g = L.g; h->n_bits = n_bits;
+        int b[8] = {b0, b1, b2, b3, b4, b5, b6, b7};
+        for (int i = 0; i < 8; ++i) h->bits[i] = b[i];
+        // s1_max_bits was zeroed by the memset that precedes this kernel
+    }
+}
+
+// One thread block per packed block (64 rows x one group).  Phase A: a warp per row computes the
+// group's (s1, lo) and the top-width code of every element, in exactly the fp32 operation order of
+// the definition (one IEEE rounding per operation, no contraction).  Phase B: the block assembles
+// the segment words and writes them with coalesced stores.
+__global__ void __launch_bounds__(PACK_THREADS)
+pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ packed) {
+    extern __shared__ uint8_t smem[];
+    uint8_t* codes = smem;                                  // [64][g]
+    const int G = blockIdx.x, rt = blockIdx.y;
+    const int g = L.g;
+    uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float levels = (float)((1 << L.b1) - 1);
+    unsigned s1_max_local = 0;
+
+    for (int r = warp; r < D2MOE_TILE_ROWS; r += PACK_THREADS / 32) {
+        const long long row = (long long)rt * D2MOE_TILE_ROWS + r;
+        if (row >= L.rows) {                                // padding rows: zero codes, zero meta
+            for (int k = lane; k < g; k += 32) codes[r * g + k] = 0;
+            if (lane == 0) reinterpret_cast<uint32_t*>(blk)[r] = 0u;
+            continue;
+        }
+        const float* src = W + row * (long long)L.cols + (long long)G * g;
+        float wmin = INFINITY, wmax = -INFINITY;
+        for (int k = lane; k < g; k += 32) { float v = src[k]; wmin = fminf(wmin, v); wmax = fmaxf(wmax, v); }
+        for (int off = 16; off; off >>= 1) {
+            wmin = fminf(wmin, __shfl_xor_sync(0xffffffffu, wmin, off));
+            wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, off));
+        }
+        const __half lo_h = __float2half_rd(wmin);
+        const float lo = __half2float(lo_h);
+        __half s1_h = __float2half_ru(__fdiv_rn(__fsub_rn(wmax, lo), levels));
+        float s1 = __half2float(s1_h);
+        if (s1 == 0.0f) { s1 = 6.103515625e-05f; s1_h = __float2half_rn(s1); }   // 2^-14
+        for (int k = lane; k < g; k += 32) {
+            const float w = src[k];
+            float q = rintf(__fdiv_rn(__fsub_rn(w, lo), s1));
+            q = fminf(fmaxf(q, 0.0f), levels);
+            float what = __fadd_rn(lo, __fmul_rn(q, s1));
+            float res = __fsub_rn(w, what);
+            int code = (int)q;
+            float sj = __fmul_rn(s1, 0.25f);                 // s_1 = s1 * 2^-2
+            for (int j = 1; j <= L.top - L.b1; ++j) {
+                const bool bit = res >= 0.0f;
+                what = __fadd_rn(what, bit ? sj : -sj);
+                res = __fsub_rn(w, what);
+                code = code * 2 + (bit ? 1 : 0);
+                sj = __fmul_rn(sj, 0.5f);
+            }
+            codes[r * g + k] = (uint8_t)code;
+        }
+        if (lane == 0) {
+            __half2 m = __halves2half2(s1_h, lo_h);          // low half = s1, high half = lo
+            reinterpret_cast<__half2*>(blk)[r] = m;
+            s1_max_local = max(s1_max_local, __float_as_uint(s1));
+        }
+    }
+    if (lane == 0 && s1_max_local)
+        atomicMax(&reinterpret_cast<PackHeader*>(packed)->s1_max_bits, s1_max_local);
+    __syncthreads();
+
+    for (int j = 0; j < L.n_seg; ++j) {
+        const int sw = L.seg_sw[j], per = 16 / sw, cs = L.seg_cs[j];
+        const int row_bytes = g * sw / 8;
+        const int n_words = D2MOE_TILE_ROWS * row_bytes / 4;
+        const unsigned mask = (1u << L.seg_w[j]) - 1u;
+        uint32_t* dst = reinterpret_cast<uint32_t*>(blk + L.seg_off[j]);
+        for (int wi = threadIdx.x; wi < n_words; wi += PACK_THREADS) {
+            const int ob = wi * 4;
+            const int c = ob / (D2MOE_TILE_ROWS * cs);
+            const int rem = ob - c * D2MOE_TILE_ROWS * cs;
+            const int r = rem / cs, within = rem - r * cs;
+            const int m = (c * cs + within) >> 2;
+            uint32_t word = 0;
+            for (int e = 0; e < per; ++e)
+                for (int h = 0; h < 2; ++h) {
+                    const int k = 2 * (m * per + e) + h;
+                    const uint32_t v = (codes[r * g + k] >> L.seg_shift[j]) & mask;
+                    word |= v << (16 * h + sw * e);
+                }
+            dst[wi] = word;
+        }
+    }
+}
+
+__global__ void unpack_kernel(PackLayout L, const uint8_t* __restrict__ packed, int bits,
+                              uint8_t* __restrict__ codes, float* __restrict__ scale,
+                              float* __restrict__ offset) {
+    const long long n = (long long)L.rows * L.cols;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int row = (int)(idx / L.cols), col = (int)(idx - (long long)row * L.cols);
+        const int rt = row / D2MOE_TILE_ROWS, r = row - rt * D2MOE_TILE_ROWS;
+        const int G = col / L.g, k = col - G * L.g;
+        const uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
+        unsigned code = 0;
+        for (int j = 0; j < L.n_seg; ++j) {
+            int bitpos;
+            const int wo = d2moe_elem_word(L, j, r, k, &bitpos);
+            const uint32_t word = *reinterpret_cast<const uint32_t*>(blk + wo);
+            code |= ((word >> bitpos) & ((1u << L.seg_w[j]) - 1u)) << L.seg_shift[j];
+        }
+        codes[idx] = (uint8_t)(code >> (L.top - bits));
+        if (k == 0) {
+            const __half2 m = reinterpret_cast<const __half2*>(blk)[r];
+            if (scale) scale[(long long)row * L.n_groups + G] = __low2float(m);
+            if (offset) offset[(long long)row * L.n_groups + G] = __high2float(m);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const float* W, uint8_t* packed,
+                        cudaStream_t st) {
+    cudaError_t err = cudaMemsetAsync(packed, 0, D2MOE_HEADER_BYTES, st);
+    if (err != cudaSuccess) return err;
+    int b[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int i = 0; i < n_bits; ++i) b[i] = bits[i];
+    pack_header_kernel<<<1, 32, 0, st>>>(reinterpret_cast<PackHeader*>(packed), L, n_bits,
+                                         b[0], b[1], b[2], b[3], b[4], b[5], b[6], b[7]);
+    dim3 grid(L.n_groups, L.n_rt);
+    size_t smem = (size_t)D2MOE_TILE_ROWS * L.g;
+    pack_kernel<<<grid, PACK_THREADS, smem, st>>>(L, W, packed);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack(const PackLayout& L, const uint8_t* packed, int bits, uint8_t* codes,
+                          float* scale, float* offset, cudaStream_t st) {
+    long long n = (long long)L.rows * L.cols;
+    int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+    if (blocks < 1) blocks = 1;
+    unpack_kernel<<<blocks, 256, 0, st>>>(L, packed, bits, codes, scale, offset);
+    return cudaGetLastError();
+}

@@ -1,0 +1,197 @@
+// Dual routing (expert gate top-k + per-expert bit-width choice, Section 3.2) and the stable
+// grouping of assignments by (expert, width); its histogram is B_{j,k} of Section 3.4.3.
+#include "d2moe_common.cuh"
+
+namespace {
+
+constexpr int MAX_TOPK = 8;
+constexpr int MAX_E_PER_LANE = 8;        // up to 256 experts
+
+// fp32 dot product in the pinned order: lane l accumulates elements l, l+32, ... with one fused
+// multiply-add each, then a butterfly reduction with offsets 16, 8, 4, 2, 1.
+__device__ __forceinline__ float dot_pinned(const __nv_bfloat16* __restrict__ a,
+                                            const __nv_bfloat16* __restrict__ b, int d, int lane) {
+    float acc = 0.0f;
+    for (int i = lane; i < d; i += 32)
+        acc = fmaf(__bfloat162float(a[i]), __bfloat162float(b[i]), acc);
+    for (int off = 16; off; off >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, off);
+    return acc;
+}
+
+// One warp per token.
+__global__ void __launch_bounds__(128)
+route_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gate_w,
+             const float* __restrict__ logits_in, const __nv_bfloat16* __restrict__ bit_w,
+             const int8_t* __restrict__ forced, RouteBufs R, int32_t* __restrict__ keys,
+             int32_t* __restrict__ device_status) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= D.T) return;
+    const int E = D.E;
+    const __nv_bfloat16* xt = x + (size_t)t * D.d;
+
+    float lg[MAX_E_PER_LANE];
+#pragma unroll
+    for (int m = 0; m < MAX_E_PER_LANE; ++m) lg[m] = -INFINITY;
+    if (logits_in) {
+#pragma unroll
+        for (int m = 0; m < MAX_E_PER_LANE; ++m) {
+            const int e = lane + 32 * m;
+            if (e < E) lg[m] = logits_in[(size_t)t * E + e];
+        }
+    } else {
+        for (int e = 0; e < E; ++e) {
+            const float v = dot_pinned(xt, gate_w + (size_t)e * D.d, D.d, lane);
+#pragma unroll
+            for (int m = 0; m < MAX_E_PER_LANE; ++m)
+                if (m == (e >> 5) && lane == (e & 31)) lg[m] = v;
+        }
+    }
+    bool bad = false;
+#pragma unroll
+    for (int m = 0; m < MAX_E_PER_LANE; ++m)
+        if (lane + 32 * m < E && !isfinite(lg[m])) bad = true;
+    if (__any_sync(0xffffffffu, bad) && lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_NONFINITE);
+
+    // k rounds of arg-max over the remaining logits, ties to the lower index
+    unsigned taken = 0;
+    int sel[MAX_TOPK];
+    float selv[MAX_TOPK];
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s) {
+        sel[s] = 0; selv[s] = 0.0f;
+        if (s < D.k) {
+            float bv = -INFINITY; int bi = 0x7fffffff;
+#pragma unroll
+            for (int m = 0; m < MAX_E_PER_LANE; ++m) {
+                const int e = lane + 32 * m;
+                if (e < E && !((taken >> m) & 1u)) {
+                    if (bi == 0x7fffffff || lg[m] > bv) { bv = lg[m]; bi = e; }
+                }
+            }
+            for (int off = 16; off; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                const bool take = (oi != 0x7fffffff) &&
+                                  (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
+                if (take) { bv = ov; bi = oi; }
+            }
+            sel[s] = bi; selv[s] = bv;
+            if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+        }
+    }
+
+    // softmax over all experts, gathered at the selected ones
+    const float mx = selv[0];
+    float part = 0.0f;
+#pragma unroll
+    for (int m = 0; m < MAX_E_PER_LANE; ++m)
+        if (lane + 32 * m < E) part += expf(lg[m] - mx);
+    for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    float w[MAX_TOPK];
+    float wsum = 0.0f;
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s) {
+        w[s] = 0.0f;
+        if (s < D.k) { w[s] = expf(selv[s] - mx) / part; wsum += w[s]; }
+    }
+
+    // bit-width choice per selected expert
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s) {
+        if (s < D.k) {
+            const int a = t * D.k + s;
+            int kk;
+            if (forced) {
+                kk = forced[a];
+                if (kk < 0 || kk >= D.K) {
+                    if (lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_BAD_INDEX);
+                    kk = kk < 0 ? 0 : D.K - 1;
+                }
+            } else {
+                float best = 0.0f; kk = 0;
+                for (int c = 0; c < D.K; ++c) {
+                    const float u = dot_pinned(xt, bit_w + ((size_t)sel[s] * D.K + c) * D.d, D.d, lane);
+                    if (c == 0 || u > best) { best = u; kk = c; }
+                }
+            }
+            if (lane == 0) {
+                R.topk_idx[a] = sel[s];
+                R.topk_w[a] = D.renormalize ? w[s] / wsum : w[s];
+                R.bit_idx[a] = (int8_t)kk;
+                keys[a] = sel[s] * D.K + kk;
+            }
+        }
+    }
+}
+
+// One warp per key: count the assignments that carry it.
+__global__ void count_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ hist) {
+    const int lane = threadIdx.x & 31;
+    const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (key >= n_keys) return;
+    int cnt = 0;
+    for (int base = 0; base < A; base += 32) {
+        const int a = base + lane;
+        const bool m = a < A && keys[a] == key;
+        cnt += __popc(__ballot_sync(0xffffffffu, m));
+    }
+    if (lane == 0) hist[key] = cnt;
+}
+
+// Exclusive prefix sum of the histogram by one warp.
+__global__ void scan_kernel(int n_keys, const int32_t* __restrict__ hist, int32_t* __restrict__ group_off) {
+    const int lane = threadIdx.x;
+    int carry = 0;
+    for (int base = 0; base < n_keys; base += 32) {
+        const int i = base + lane;
+        const int v = i < n_keys ? hist[i] : 0;
+        int incl = v;
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (i < n_keys) group_off[i] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) group_off[n_keys] = carry;
+}
+
+// One warp per key: write its assignments, in ascending assignment id, from group_off[key] on.
+__global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ keys,
+                               const int32_t* __restrict__ group_off, int32_t* __restrict__ perm,
+                               int32_t* __restrict__ inv_perm) {
+    const int lane = threadIdx.x & 31;
+    const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (key >= n_keys) return;
+    int pos = group_off[key];
+    const int end = group_off[key + 1];
+    if (pos == end) return;
+    for (int base = 0; base < A; base += 32) {
+        const int a = base + lane;
+        const bool m = a < A && keys[a] == key;
+        const unsigned bal = __ballot_sync(0xffffffffu, m);
+        if (m) {
+            const int p = pos + __popc(bal & ((1u << lane) - 1u));
+            perm[p] = a;
+            inv_perm[a] = p;
+        }
+        pos += __popc(bal);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
+                         const float* logits_in, const __nv_bfloat16* bit_w, const int8_t* forced,
+                         const RouteBufs& R, float* /*logits_ws*/, int32_t* keys_ws, int32_t* hist_ws,
+                         int32_t* device_status, cudaStream_t st) {
+    const int warps_per_block = 4;
+    const int n_keys = D.E * D.K;
+    route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+        D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
+    count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);
+    scan_kernel<<<1, 32, 0, st>>>(n_keys, hist_ws, R.group_off);
+    scatter_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+    return cudaGetLastError();
+}

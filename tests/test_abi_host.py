@@ -1,0 +1,112 @@
+"""The C-ABI library: it loads, exports what include/d2moe.h declares, and rejects bad arguments on
+the host before any launch.  No kernel runs here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2504_15299_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "d2moe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(d2moe_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert set(names) == set(binding.EXPORTS)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def good():
+    return binding.Config(256, 512, 4, 2, 64, (2, 4, 8))
+
+
+def test_status_strings(lib):
+    assert binding.status_string(0) == "ok"
+    assert "NULL" in binding.status_string(1)
+    assert binding.status_string(99) == "unknown status"
+
+
+@pytest.mark.parametrize("mutate,code", [
+    (lambda c: setattr(c, "top_k", 5), 2),
+    (lambda c: setattr(c, "top_k", 0), 2),
+    (lambda c: setattr(c, "bits", (4, 2, 8)), 2),
+    (lambda c: setattr(c, "bits", (2, 4, 9)), 2),
+    (lambda c: setattr(c, "bits", (0, 4)), 2),
+    (lambda c: setattr(c, "group_size", 48), 2),
+    (lambda c: setattr(c, "group_size", 128), 0),
+    (lambda c: setattr(c, "d_model", 200), 2),
+    (lambda c: setattr(c, "scale_mode", 1), 4),
+    (lambda c: setattr(c, "renormalize", 2), 2),
+    (lambda c: setattr(c, "kernel_path", 7), 2),
+    (lambda c: setattr(c, "n_experts", 300), 2),
+])
+def test_check_config(lib, mutate, code):
+    c = good()
+    mutate(c)
+    assert binding.check_config(c) == code
+
+
+def test_packed_bytes_is_the_top_width_only(lib):
+    rows, cols = 512, 256
+    a = binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (2, 3, 4, 8)), rows, cols)
+    b = binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (2, 4, 8)), rows, cols)
+    c = binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (8,)), rows, cols)
+    assert a == b == c
+    total, code, meta = a
+    assert code == rows * cols and meta == rows * (cols // 64) * 4 and total == 256 + code + meta
+    # a 4-bit top width stores half of that
+    assert binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (2, 3, 4)), rows, cols)[1] == rows * cols // 2
+    # rows are padded to the 64-row tile
+    assert binding.packed_bytes(good(), 100, 256)[1] == 128 * 256
+    with pytest.raises(binding.D2MoEError):
+        binding.packed_bytes(good(), 64, 100)
+
+
+def test_null_and_short_buffers_are_rejected_before_launch(lib):
+    c = good().c()
+    L = lib
+    # pack: NULL pointers
+    assert L.d2moe_pack_mwq(ctypes.byref(c), None, 64, 64, None, 0, None) == 1
+    # pack: short output, misaligned output (fake non-null pointers are never dereferenced)
+    assert L.d2moe_pack_mwq(ctypes.byref(c), 4096, 64, 64, 8192, 10, None) == 5
+    assert L.d2moe_pack_mwq(ctypes.byref(c), 4096, 64, 64, 8192 + 16, 1 << 20, None) == 3
+    # unpack: width outside [b1, top]
+    assert L.d2moe_unpack_codes(ctypes.byref(c), 4096, 64, 64, 1, 4096, None, None, None) == 3
+    # workspace query
+    assert binding.workspace_bytes(good(), 16) > 0
+    bad = good(); bad.top_k = 9
+    assert L.d2moe_workspace_bytes(ctypes.byref(bad.c()), 16) == 0
+    # route: both / neither of gate_w and logits
+    args_tail = [4096] * 6 + [None, 4096, 1 << 30, None]
+    assert L.d2moe_route(ctypes.byref(c), 4, 4096, None, None, None, 4096, *args_tail) == 1
+    assert L.d2moe_route(ctypes.byref(c), 4, 4096, 4096, 4096, None, 4096, *args_tail) == 1
+    assert L.d2moe_route(ctypes.byref(c), 4, 4096, 4096, None, None, None, *args_tail) == 1
+    # route: short workspace
+    assert L.d2moe_route(ctypes.byref(c), 4, 4096, 4096, None, None, 4096, *([4096] * 6), None, 4096, 16, None) == 5
+    # forward: T == 0 is a no-op, negative T is a shape error, missing expert pointer is NULL
+    assert L.d2moe_moe_forward(ctypes.byref(c), 0, None, None, None, None, None, None, None, 0, None) == 0
+    assert L.d2moe_moe_forward(ctypes.byref(c), -1, None, None, None, None, None, None, None, 0, None) == 3
+    ptrs = (ctypes.c_void_p * 12)(*([4096] * 11 + [None]))
+    rin = binding._RouteIn(4096, None, None, 4096)
+    assert L.d2moe_moe_forward(ctypes.byref(c), 4, 4096, ptrs, ctypes.byref(rin), None, 4096, None, 4096,
+                               1 << 30, None) == 1
+    ptrs = (ctypes.c_void_p * 12)(*([4096] * 12))
+    assert L.d2moe_moe_forward(ctypes.byref(c), 4, 4096, ptrs, ctypes.byref(rin), None, 4096, None, 4096,
+                               16, None) == 5
+    # stack layer: argument errors are found before the normalisation kernel would be launched
+    assert L.d2moe_stack_layer(ctypes.byref(c), 4, 4096, 4096, ctypes.c_float(1e-5), ptrs, ctypes.byref(rin),
+                               None, 4096, 16, None) == 5

@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer work (codes, routing indices, widths, permutation) is compared bit for bit; layer
+outputs within 1e-2 of the row's largest magnitude (fp32 accumulation, bf16 output)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2504_15299_b200 import synth
+from tests.helpers import OracleLayer, gpu_layer, max_norm_rel_err, np_f32
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2504_15299_b200 import binding, build
+    build.build_library()
+    binding.lib()
+    return binding
+
+
+def oracle_mods():
+    from oracle import moe, mwq, routing
+    return mwq, routing, moe
+
+
+# ------------------------------------------------------------------ pack / unpack
+@pytest.mark.parametrize("bits,g,rows,cols", [
+    ((2, 4, 8), 64, 512, 256), ((2, 3, 4, 8), 128, 256, 512), ((2, 3, 4), 128, 100, 256),
+    ((5, 6, 7, 8), 32, 64, 96), ((3, 5), 64, 130, 128), ((8,), 256, 64, 512), ((1, 2, 3), 32, 70, 64),
+    ((4, 8), 128, 192, 1408),
+])
+def test_pack_codes_bit_exact(B, bits, g, rows, cols):
+    mwq, _, _ = oracle_mods()
+    cfg = B.Config(cols, cols, 2, 1, g, bits)
+    W = synth.normal(11, 5, (rows, cols), 0.02, "cuda")
+    blob = B.pack_mwq(cfg, W)
+    q = mwq.quantize(np_f32(W), bits, g)
+    for b in range(bits[0], bits[-1] + 1):
+        codes, s1, lo = B.unpack_codes(cfg, blob, rows, cols, b)
+        assert np.array_equal(codes.cpu().numpy(), mwq.slice_code(q, b)), f"width {b}"
+    assert np.array_equal(np_f32(s1), q.s1) and np.array_equal(np_f32(lo), q.lo)
+
+
+def test_pack_degenerate_groups(B):
+    mwq, _, _ = oracle_mods()
+    cfg = B.Config(128, 128, 2, 1, 64, (2, 4, 8))
+    W = torch.zeros((64, 128), device="cuda")
+    W[1] = 0.03125
+    W[2, :64] = torch.linspace(-1, 1, 64, device="cuda")
+    W[3] = synth.normal(1, 1, (1, 128), 1e-6, "cuda")[0]          # tiny range: subnormal fp16 scale
+    blob = B.pack_mwq(cfg, W)
+    q = mwq.quantize(np_f32(W), (2, 4, 8), 64)
+    codes, s1, lo = B.unpack_codes(cfg, blob, 64, 128, 8)
+    assert np.array_equal(codes.cpu().numpy(), q.code)
+    assert np.array_equal(np_f32(s1), q.s1) and np.array_equal(np_f32(lo), q.lo)
+
+
+def test_pack_mixtral_matrix_sampled_rows(B):
+    """Full-size expert matrix (14336 x 4096, g = 128): the oracle regenerates and quantizes sampled
+    rows (first, last, tile edges, random) and every code, scale and offset of those rows must match."""
+    mwq, _, _ = oracle_mods()
+    wl = synth.WORKLOADS["mixtral_decode"]
+    cfg = B.Config.from_workload(wl)
+    rows, cols = synth.expert_matrix_shape(wl, 0)
+    W = synth.expert_matrix(wl, 3, 0, device="cuda")
+    blob = B.pack_mwq(cfg, W)
+    del W
+    r = np.random.default_rng(0)
+    sample = sorted(set([0, 63, 64, 127, 128, rows - 1, rows - 64] + r.integers(0, rows, 40).tolist()))
+    Wr = np_f32(synth.expert_matrix(wl, 3, 0, rows=torch.tensor(sample)))
+    q = mwq.quantize(Wr, wl.bits, wl.group_size)
+    for b in wl.bits:
+        codes, s1, lo = B.unpack_codes(cfg, blob, rows, cols, b)
+        assert np.array_equal(codes[sample].cpu().numpy(), mwq.slice_code(q, b))
+    assert np.array_equal(np_f32(s1[sample]), q.s1) and np.array_equal(np_f32(lo[sample]), q.lo)
+
+
+# ------------------------------------------------------------------ routing
+def check_route(B, cfg, x, *, gate_w=None, logits=None, bit_w=None, forced=None):
+    _, routing, _ = oracle_mods()
+    K = len(cfg.bits)
+    r = B.route(cfg, x, gate_w=gate_w, logits=logits, bit_w=bit_w, forced_bit_idx=forced)
+    torch.cuda.synchronize()
+    ref = routing.route(np_f32(x), E=cfg.n_experts, K=K, top_k=cfg.top_k, renormalize=bool(cfg.renormalize),
+                        gate_w=None if gate_w is None else np_f32(gate_w),
+                        logits=None if logits is None else np_f32(logits),
+                        bit_w=None if bit_w is None else np_f32(bit_w),
+                        forced_bit_idx=None if forced is None else forced.cpu().numpy())
+    assert np.array_equal(r.topk_idx.cpu().numpy(), ref.topk_idx)
+    assert np.array_equal(r.bit_idx.cpu().numpy(), ref.bit_idx)
+    assert np.array_equal(r.perm.cpu().numpy(), ref.grouping.perm)
+    assert np.array_equal(r.inv_perm.cpu().numpy(), ref.grouping.inv_perm)
+    assert np.array_equal(r.group_off.cpu().numpy(), ref.grouping.group_off)
+    assert np.allclose(r.topk_w.cpu().numpy(), ref.topk_w, rtol=1e-5, atol=1e-7)
+    assert int(r.device_status.item()) == 0
+    return r, ref
+
+
+@pytest.mark.parametrize("name,T", [("tiny", 16), ("mixtral_decode", 1), ("mixtral_decode", 64),
+                                    ("finegrained", 256)])
+def test_route_from_gate_weights(B, name, T):
+    wl = synth.WORKLOADS[name]
+    cfg = B.Config.from_workload(wl)
+    x = synth.tokens_bf16(wl, T, "cuda")
+    check_route(B, cfg, x, gate_w=synth.gate_weight_bf16(wl, "cuda"), forced=synth.forced_bit_idx(wl, T, "cuda"))
+
+
+def test_route_from_supplied_logits_prefill(B):
+    wl = synth.WORKLOADS["mixtral_prefill"]
+    cfg = B.Config.from_workload(wl)
+    T = 2048
+    x = synth.tokens_bf16(wl, T, "cuda")
+    r, ref = check_route(B, cfg, x, logits=synth.zipf_logits(wl, T, "cuda"),
+                         forced=synth.forced_bit_idx(wl, T, "cuda"))
+    load = ref.grouping.hist.sum(axis=1)
+    assert load[0] > 2 * load[-1]                       # the Zipf prior skews the expert loads
+
+
+def test_route_learned_bit_widths_and_no_renormalize(B):
+    wl = synth.WORKLOADS["mixtral_stack"]
+    cfg = B.Config.from_workload(wl)
+    cfg.renormalize = 0
+    x = synth.tokens_bf16(wl, 16, "cuda")
+    r, ref = check_route(B, cfg, x, gate_w=synth.gate_weight_bf16(wl, "cuda"),
+                         bit_w=synth.bit_router_weight_bf16(wl, "cuda"))
+    assert len(set(ref.bit_idx.reshape(-1).tolist())) > 1
+
+
+def test_route_ties_and_empty_groups(B):
+    cfg = B.Config(64, 64, 8, 3, 32, (2, 4, 8))
+    T = 5
+    x = synth.tokens_bf16(synth.WORKLOADS["tiny"], T, "cuda")[:, :64].contiguous()
+    logits = torch.zeros((T, 8), device="cuda")
+    logits[1, 5] = logits[1, 2] = 1.0
+    logits[2] = torch.tensor([0, 1, 1, 1, 1, 0, 0, 0.0])
+    forced = torch.zeros((T, 3), dtype=torch.int8, device="cuda")
+    r, ref = check_route(B, cfg, x, logits=logits, forced=forced)
+    assert r.topk_idx[0].tolist() == [0, 1, 2] and r.topk_idx[1].tolist() == [2, 5, 0]
+    assert r.topk_idx[2].tolist() == [1, 2, 3]
+
+
+def test_route_flags_nonfinite_logits_and_bad_width_index(B):
+    cfg = B.Config(64, 64, 4, 2, 32, (2, 4, 8))
+    x = torch.zeros((2, 64), dtype=torch.bfloat16, device="cuda")
+    logits = torch.zeros((2, 4), device="cuda")
+    logits[1, 2] = float("nan")
+    forced = torch.zeros((2, 2), dtype=torch.int8, device="cuda")
+    forced[0, 1] = 7
+    r = B.route(cfg, x, logits=logits, forced_bit_idx=forced)
+    torch.cuda.synchronize()
+    st = int(r.device_status.item())
+    assert st & B.DEV_NONFINITE and st & B.DEV_BAD_INDEX
+    assert int(r.group_off[-1].item()) == 4 and sorted(r.perm.tolist()) == [0, 1, 2, 3]
+
+
+# ------------------------------------------------------------------ whole layer
+def run_layer(B, cfg, wl, T, *, tokens=None, kernel_path=None, blobs=None):
+    _, routing, moe = oracle_mods()
+    if kernel_path is not None:
+        cfg.kernel_path = kernel_path
+    x = synth.tokens_bf16(wl, T, "cuda")
+    kw = {}
+    okw = {}
+    if wl.zipf_logits:
+        kw["logits"] = synth.zipf_logits(wl, T, "cuda")
+        okw["logits"] = np_f32(kw["logits"])
+    else:
+        kw["gate_w"] = synth.gate_weight_bf16(wl, "cuda")
+        okw["gate_w"] = np_f32(kw["gate_w"])
+    if wl.learned_bits:
+        kw["bit_w"] = synth.bit_router_weight_bf16(wl, "cuda")
+        okw["bit_w"] = np_f32(kw["bit_w"])
+    else:
+        kw["forced_bit_idx"] = synth.forced_bit_idx(wl, T, "cuda")
+        okw["forced_bit_idx"] = kw["forced_bit_idx"].cpu().numpy()
+    if blobs is None:
+        blobs = gpu_layer(B, cfg, wl)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = B.moe_forward(cfg, x, blobs, device_status=status, **kw)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rt = routing.route(np_f32(x), E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
+                       renormalize=bool(cfg.renormalize), **okw)
+    ol = OracleLayer(wl)
+    ref = moe.moe_layer(np_f32(x), rt, ol, wl.bits, wl.n_experts, wl.n_shared, tokens=tokens)
+    yg = np_f32(y)
+    errs = {t: max_norm_rel_err(yg[t], ref[t]) for t in ref}
+    return errs, y, blobs
+
+
+@pytest.mark.parametrize("path", [1])
+def test_layer_tiny(B, path):
+    wl = synth.WORKLOADS["tiny"]
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 16, kernel_path=path)
+    assert len(errs) == 16 and max(errs.values()) < TOL, errs
+
+
+def test_layer_finegrained_with_shared_experts_sampled_tokens(B):
+    wl = synth.WORKLOADS["finegrained"]
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 256, tokens=[0, 100, 255], kernel_path=1)
+    assert max(errs.values()) < TOL, errs
+
+
+def test_layer_empty_batch_is_a_noop(B):
+    wl = synth.WORKLOADS["tiny"]
+    cfg = B.Config.from_workload(wl)
+    x = torch.empty((0, wl.d_model), dtype=torch.bfloat16, device="cuda")
+    y = B.moe_forward(cfg, x, [x] * 12, gate_w=synth.gate_weight_bf16(wl, "cuda"),
+                      forced_bit_idx=torch.empty((0, 2), dtype=torch.int8, device="cuda"))
+    assert y.shape == (0, wl.d_model)
+
+
+def test_layer_with_precomputed_routing_matches_internal_routing(B):
+    wl = synth.WORKLOADS["tiny"]
+    cfg = B.Config.from_workload(wl, kernel_path=1)
+    x = synth.tokens_bf16(wl, 16, "cuda")
+    gw = synth.gate_weight_bf16(wl, "cuda")
+    fb = synth.forced_bit_idx(wl, 16, "cuda")
+    blobs = gpu_layer(B, cfg, wl)
+    y1 = B.moe_forward(cfg, x, blobs, gate_w=gw, forced_bit_idx=fb)
+    pre = B.route(cfg, x, gate_w=gw, forced_bit_idx=fb)
+    y2 = B.moe_forward(cfg, x, blobs, pre=pre)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+
+
+def test_stack_layer_tiny(B):
+    _, routing, moe = oracle_mods()
+    wl = synth.WORKLOADS["tiny"]
+    cfg = B.Config.from_workload(wl, kernel_path=1)
+    x = synth.tokens_bf16(wl, 16, "cuda")
+    x0 = np_f32(x).astype(np.float64)
+    gw = synth.gate_weight_bf16(wl, "cuda")
+    bw = bit_w = synth.bit_router_weight_bf16(wl, "cuda")
+    blobs = gpu_layer(B, cfg, wl)
+    xn = torch.empty_like(x)
+    B.stack_layer(cfg, x, xn, blobs, gate_w=gw, bit_w=bw)
+    torch.cuda.synchronize()
+    ol = OracleLayer(wl)
+
+    def moe_of(xnorm):
+        rt = routing.route(xnorm.astype(np.float32), E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
+                           renormalize=True, gate_w=np_f32(gw), bit_w=np_f32(bw))
+        out = moe.moe_layer(xnorm, rt, ol, wl.bits, wl.n_experts)
+        return np.stack([out[t] for t in range(16)])
+
+    ref = moe.stack_layer(x0, moe_of)
+    assert np.array_equal(np_f32(xn), moe.round_to_bf16(moe.rmsnorm(x0)))
+    for t in range(16):
+        assert max_norm_rel_err(np_f32(x)[t], ref[t]) < TOL
