@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the dual-routed MWQ MoE layer (one step = one pass of the whole hot path over one batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload mixtral_decode] [--tokens 64] [--path auto|cuda_core|tensor]
+
+Prints ONE JSON line.  N > 1 runs independent replicas, one process per GPU (launched by
+torch.distributed.run), no data-path collective; the barrier and the max-over-ranks timing use NCCL.
+`--impl reference` times the CPU oracle on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2504_15299_b200 import synth  # noqa: E402
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic bytes (what the method has to read at the routed widths)
+# ------------------------------------------------------------------------------------------------
+def matrix_bytes(rows, cols, g, bits_read):
+    return rows * cols * bits_read // 8 + rows * (cols // g) * 4
+
+
+def algorithmic_bytes(wl, T, group_off):
+    """Bytes per layer call from the realised routing: every plane of an active expert up to the
+    largest width routed to it is read once; plus activations in/out and the h round trip."""
+    K = len(wl.bits)
+    hist = [group_off[i + 1] - group_off[i] for i in range(wl.n_experts * K)]
+    gu = dn = 0
+    active = 0
+    for e in range(wl.n_experts + wl.n_shared):
+        if e < wl.n_experts:
+            ks = [kk for kk in range(K) if hist[e * K + kk] > 0]
+            if not ks:
+                continue
+            b = wl.bits[max(ks)]
+        else:
+            b = wl.bits[-1]
+        active += 1
+        gu += 2 * matrix_bytes(wl.d_ffn, wl.d_model, wl.group_size, b)
+        dn += matrix_bytes(wl.d_model, wl.d_ffn, wl.group_size, b)
+    A_tot = T * (wl.top_k + wl.n_shared)
+    io_gu = A_tot * wl.d_model * 2 + A_tot * wl.d_ffn * 2       # gathered x in, h out (16-bit)
+    io_dn = A_tot * wl.d_ffn * 2 + A_tot * wl.d_model * 4       # h in, expert outputs out (fp32)
+    io_layer = 2 * T * wl.d_model * 2 + T * wl.top_k * 17
+    return {"gate_up": gu + io_gu, "down": dn + io_dn, "layer": gu + dn + io_layer, "active_experts": active}
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        try:
+            sm, mx, reasons = [], [], set()
+            for line in open(self.path):
+                f = [s.strip() for s in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            if sm:
+                sm.sort()
+                out = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                       "samples": len(sm)}
+            os.unlink(self.path)
+        except Exception:
+            pass
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# oracle legs (CPU)
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    """The oracle on a bounded sample: the first `n_tok` tokens of the batch through routing,
+    dequantization at the routed widths, the expert FFN restricted to the first `n_hidden_groups`
+    groups of hidden units (the FFN cost is linear in the hidden units: each contributes one term
+    of the down projection), and the combine.  Time is scaled by F / hidden units used."""
+
+    def __init__(self, wl, T, n_tok, n_hidden_groups, device_for_inputs="cpu"):
+        import numpy as np
+        from oracle import mwq, routing
+        self.np, self.mwq, self.routing = np, mwq, routing
+        self.wl, self.T, self.n_tok = wl, T, n_tok
+        g = wl.group_size
+        self.hid = min(wl.d_ffn, n_hidden_groups * g)
+        x = synth.tokens_bf16(wl, T, device_for_inputs)
+        self.x = x.to("cpu", torch.float32).numpy()
+        self.gw = synth.gate_weight_bf16(wl, "cpu").to(torch.float32).numpy()
+        self.fb = synth.forced_bit_idx(wl, T, "cpu").numpy()
+        rt = routing.route(self.x, E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
+                           renormalize=bool(wl.renormalize), gate_w=self.gw, forced_bit_idx=self.fb)
+        experts = sorted({int(e) for t in range(n_tok) for e in rt.topk_idx[t]}) + \
+            [wl.n_experts + s for s in range(wl.n_shared)]
+        sub = torch.arange(self.hid)
+        self.packed = {}
+        for e in experts:          # setup (offline quantization), not timed
+            Wg = synth.expert_matrix(wl, e, 0, device_for_inputs, rows=sub).cpu().numpy()
+            Wu = synth.expert_matrix(wl, e, 1, device_for_inputs, rows=sub).cpu().numpy()
+            # columns 0..hid-1 of the [d, F] down projection (whole groups along F)
+            Wd = synth.expert_matrix(wl, e, 2, device_for_inputs, cols=sub).cpu().numpy()
+            self.packed[e] = tuple(mwq.quantize(W, wl.bits, g) for W in (Wg, Wu, Wd))
+
+    def step(self):
+        """One timed pass; returns (seconds, scale factor to the full FFN)."""
+        from oracle import moe
+        wl = self.wl
+        t0 = time.perf_counter()
+        rt = self.routing.route(self.x, E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
+                                renormalize=bool(wl.renormalize), gate_w=self.gw, forced_bit_idx=self.fb)
+        moe.moe_layer(self.x, rt, lambda e: self.packed[e], wl.bits, wl.n_experts, wl.n_shared,
+                      tokens=range(self.n_tok))
+        dt = time.perf_counter() - t0
+        return dt, wl.d_ffn / self.hid
+
+
+def oracle_tokens_per_s(wl, T, n_tok, n_hidden_groups, steps, warmup, device_for_inputs="cpu"):
+    s = OracleSample(wl, T, n_tok, n_hidden_groups, device_for_inputs)
+    for _ in range(warmup):
+        s.step()
+    tot = 0.0
+    for _ in range(max(steps, 1)):
+        dt, scale = s.step()
+        tot += dt * scale
+    per_step = tot / max(steps, 1)
+    return n_tok / per_step, per_step, s.hid
+
+
+def used_threads():
+    try:
+        import threadpoolctl
+        n = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = synth.WORKLOADS[args.workload]
+    T = args.tokens
+    total_steps = args.steps + args.warmup
+    # size the sample so the whole run stays within ~2.5 minutes: calibrate on one hidden group
+    t0 = time.perf_counter()
+    v, per, _ = oracle_tokens_per_s(wl, T, 1, 1, 1, 0)
+    calib = time.perf_counter() - t0
+    groups = 1
+    budget = 150.0 / max(total_steps, 1)
+    while groups < 8 and calib * groups * 2 < budget * 0.5:
+        groups *= 2
+    value, per_step, hid = oracle_tokens_per_s(wl, T, 1, groups, args.steps, args.warmup)
+    cores = used_threads()
+    sample = (f"first token of the T={T} batch, all its experts at the routed widths, hidden units "
+              f"0..{hid - 1} of {wl.d_ffn} per expert, time scaled by {wl.d_ffn}/{hid} (extrapolated)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(wl, T, "cpu oracle"),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(wl, T, path):
+    return {"workload": f"{wl.name} T={T}: d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} top{wl.top_k} "
+                        f"g={wl.group_size} bits={list(wl.bits)} p={list(wl.bit_probs)}",
+            "tokens_per_step": T, "kernel_path": path,
+            "l2": "inputs larger than L2: each step streams the routed planes of every active expert "
+                  "(>1 GB per layer call against a 126 MB L2); four token batches are rotated"}
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2504_15299_b200 import binding as B, build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build_library()
+    if dist:
+        dist.barrier()
+    B.lib()
+
+    wl = synth.WORKLOADS[args.workload]
+    T = args.tokens
+    path = {"auto": B.PATH_AUTO, "cuda_core": B.PATH_CUDA_CORE, "tensor": B.PATH_TENSOR}[args.path]
+    cfg = B.Config.from_workload(wl, kernel_path=path)
+
+    blobs = []
+    for e in range(wl.n_experts + wl.n_shared):
+        for m in range(3):
+            W = synth.expert_matrix(wl, e, m, device=dev)
+            blobs.append(B.pack_mwq(cfg, W))
+            del W
+    gw = synth.gate_weight_bf16(wl, dev)
+    n_batches = 4
+    xs = [synth.tokens_bf16(wl, T, dev, step=rank * 100 + i) for i in range(n_batches)]
+    fbs = [synth.categorical(wl.seed + rank * 100 + i, synth.TID_FORCED_BITS, (T, wl.top_k), wl.bit_probs, dev)
+           for i in range(n_batches)]
+    logits = [synth.zipf_logits(wl, T, dev) for _ in range(n_batches)] if wl.zipf_logits else None
+    ws = torch.empty(B.workspace_bytes(cfg, T), dtype=torch.uint8, device=dev)
+    y = torch.empty_like(xs[0])
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def kw(i):
+        d = {"forced_bit_idx": fbs[i]}
+        if logits is not None:
+            d["logits"] = logits[i]
+        else:
+            d["gate_w"] = gw
+        return d
+
+    # realised routing of each batch -> algorithmic bytes
+    alg = []
+    for i in range(n_batches):
+        r = B.route(cfg, xs[i], workspace=ws, **kw(i))
+        torch.cuda.synchronize()
+        alg.append(algorithmic_bytes(wl, T, r.group_off.cpu().tolist()))
+
+    def step(i, events=None):
+        B.moe_forward(cfg, xs[i % n_batches], blobs, y=y, workspace=ws, device_status=status,
+                      stage_events=events, **kw(i % n_batches))
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    sync_all()
+
+    # ---- timed region: K steps, device time, max over ranks ----
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    stream = torch.cuda.current_stream()
+    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(B.N_STAGES + 1)] for _ in range(args.steps)]
+    for evs in stage_ev:
+        for ev in evs:
+            ev.record(stream)            # creates the handle
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i, stage_ev[i])
+    e1.record(stream)
+    sync_all()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    if dist:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_per_step = ms_total / args.steps
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    stage_ms = [sum(stage_ev[i][s].elapsed_time(stage_ev[i][s + 1]) for i in range(args.steps)) / args.steps
+                for s in range(B.N_STAGES)]
+
+    # ---- end to end: pinned host inputs -> device, layer, result back to the host, every step ----
+    hx = [x.cpu().pin_memory() for x in xs]
+    hfb = [f.cpu().pin_memory() for f in fbs]
+    hy = torch.empty_like(hx[0]).pin_memory()
+    dx, dfb = torch.empty_like(xs[0]), torch.empty_like(fbs[0])
+
+    def e2e_step(i):
+        j = i % n_batches
+        dx.copy_(hx[j], non_blocking=True)
+        dfb.copy_(hfb[j], non_blocking=True)
+        d = {"forced_bit_idx": dfb}
+        if logits is not None:
+            d["logits"] = logits[j]
+        else:
+            d["gate_w"] = gw
+        B.moe_forward(cfg, dx, blobs, y=y, workspace=ws, device_status=status, **d)
+        hy.copy_(y, non_blocking=True)
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    sync_all()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(args.steps):
+        e2e_step(i)
+    f1.record(stream)
+    sync_all()
+    e2e_ms = f0.elapsed_time(f1)
+    if dist:
+        tt = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_ms /= args.steps
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    used = [alg[i % n_batches] for i in range(args.steps)]
+    stage_names = B.STAGE_NAMES
+    dom = max(range(B.N_STAGES), key=lambda s: stage_ms[s])
+    dom_name = stage_names[dom]
+    dom_bytes = sum(u.get(dom_name, u["layer"]) for u in used) / len(used)
+    layer_bytes = sum(u["layer"] for u in used) / len(used)
+    achieved = dom_bytes / (stage_ms[dom] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "algorithmic_bytes_per_launch": dom_bytes,
+                "stage_ms": dict(zip(stage_names, stage_ms)),
+                "layer": {"algorithmic_bytes": layer_bytes,
+                          "achieved_gbs": layer_bytes / (ms_per_step * 1e-3) / 1e9,
+                          "frac": layer_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            tr = json.load(open(traffic_file))
+            key = f"{args.workload}:T{T}:{dom_name}:{args.path}"
+            if key in tr:
+                roofline["traffic"] = tr[key]
+        except Exception:
+            pass
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, per, hid = oracle_tokens_per_s(wl, T, 1, 2, 2, 0, device_for_inputs=dev)
+        cpu = {"value": v, "unit": UNIT, "cores": used_threads(), "kind": "oracle",
+               "sample": f"first token of the batch, all its experts at the routed widths, hidden units "
+                         f"0..{hid - 1} of {wl.d_ffn} per expert, time scaled by {wl.d_ffn}/{hid} "
+                         f"(extrapolated); 2 passes"}
+
+    line = {"metric": METRIC, "value": T * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+            "data": "synthetic", "config": workload_config(wl, T, args.path),
+            "clocks": clocks,
+            "e2e": {"value": T * world / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": hx[0].numel() * 2 + hfb[0].numel(),
+                    "d2h_bytes_per_step": hy.numel() * 2},
+            "gpu_launches": B.forward_launch_count(cfg, T) * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mixtral_decode", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=64)
+    ap.add_argument("--path", default="auto", choices=["auto", "cuda_core", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -160,6 +160,24 @@ d2moe_status d2moe_moe_forward(const d2moe_config* cfg, int64_t T, const void* x
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * d2moe_moe_forward with timing marks for profiling: `stage_events` is a HOST array of
+ * D2MOE_N_STAGES + 1 cudaEvent_t handles created by the caller with timing enabled; the call records
+ * event i on `stream` before stage i and the last one after the final stage, so the caller can read
+ * each stage's device time with cudaEventElapsedTime after synchronising.  Stages: 0 routing and
+ * grouping (nothing when `pre` is given), 1 gate/up projection + SwiGLU, 2 down projection,
+ * 3 weighted combine.  Results are identical to d2moe_moe_forward.
+ */
+#define D2MOE_N_STAGES 4
+d2moe_status d2moe_moe_forward_events(const d2moe_config* cfg, int64_t T, const void* x_bf16,
+                                      const void* const* expert_w, const d2moe_route_in* in,
+                                      const d2moe_route_out* pre, void* y_bf16, int32_t* device_status,
+                                      void* workspace, size_t workspace_bytes, void* stream,
+                                      void* const* stage_events);
+
+/* Number of kernel launches one d2moe_moe_forward call enqueues for T tokens (0 on a bad config). */
+int d2moe_forward_launch_count(const d2moe_config* cfg, int64_t T, int routing_precomputed);
+
+/*
  * One layer of the FFN-only stack used by the multi-layer benchmark configuration (not in the
  * paper): x <- bf16( x + MoE( bf16( x / sqrt(mean(x^2) + eps) ) ) ), unit gain.  x_bf16 is updated
  * in place; xn_bf16 is a caller-provided bf16 [T, d_model] scratch that receives the normalised

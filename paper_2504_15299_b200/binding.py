@@ -49,7 +49,7 @@ _lib = None
 
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
-           "d2moe_stack_layer"]
+           "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count"]
 
 
 def lib() -> ctypes.CDLL:
@@ -73,6 +73,9 @@ def lib() -> ctypes.CDLL:
     L.d2moe_route.argtypes = [cfgp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.d2moe_moe_forward.argtypes = [cfgp, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(_RouteIn),
                                     ctypes.POINTER(_RouteOut), vp, vp, vp, sz, vp]
+    L.d2moe_moe_forward_events.argtypes = [cfgp, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(_RouteIn),
+                                           ctypes.POINTER(_RouteOut), vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
+    L.d2moe_forward_launch_count.argtypes = [cfgp, i64, ctypes.c_int]
     L.d2moe_stack_layer.argtypes = [cfgp, i64, vp, vp, ctypes.c_float, ctypes.POINTER(vp),
                                     ctypes.POINTER(_RouteIn), vp, vp, sz, vp]
     for name in EXPORTS:
@@ -215,11 +218,22 @@ def _expert_ptr_array(expert_w: Sequence[torch.Tensor]):
     return arr
 
 
+N_STAGES = 4
+STAGE_NAMES = ("route", "gate_up", "down", "combine")
+
+
+def forward_launch_count(cfg: Config, T: int, routing_precomputed: bool = False) -> int:
+    return lib().d2moe_forward_launch_count(ctypes.byref(cfg.c()), T, int(routing_precomputed))
+
+
 def moe_forward(cfg: Config, x: torch.Tensor, expert_w: Sequence[torch.Tensor], *, gate_w=None, logits=None,
                 bit_w=None, forced_bit_idx=None, pre: Optional[RouteResult] = None,
                 y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                device_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """One dual-routed MWQ MoE layer.  expert_w: packed blobs, order [expert][gate, up, down]."""
+                device_status: Optional[torch.Tensor] = None, stream=None,
+                stage_events: Optional[Sequence[torch.cuda.Event]] = None) -> torch.Tensor:
+    """One dual-routed MWQ MoE layer.  expert_w: packed blobs, order [expert][gate, up, down].
+    stage_events: optional N_STAGES+1 torch.cuda.Event(enable_timing=True), each recorded once before
+    (so that its handle exists); the library records them around its stages."""
     assert x.is_cuda and x.dtype == torch.bfloat16
     T = x.shape[0]
     if y is None:
@@ -228,6 +242,14 @@ def moe_forward(cfg: Config, x: torch.Tensor, expert_w: Sequence[torch.Tensor], 
         workspace = torch.empty(workspace_bytes(cfg, max(T, 1)), dtype=torch.uint8, device=x.device)
     rin = _RouteIn(_ptr(gate_w), _ptr(logits), _ptr(bit_w), _ptr(forced_bit_idx))
     rout = pre.c() if pre is not None else None
+    if stage_events is not None:
+        assert len(stage_events) == N_STAGES + 1
+        evs = (ctypes.c_void_p * (N_STAGES + 1))(*[e.cuda_event for e in stage_events])
+        _check(lib().d2moe_moe_forward_events(ctypes.byref(cfg.c()), T, _ptr(x), _expert_ptr_array(expert_w),
+                                              ctypes.byref(rin), ctypes.byref(rout) if rout is not None else None,
+                                              _ptr(y), _ptr(device_status), _ptr(workspace), workspace.numel(),
+                                              _stream(stream), evs), "d2moe_moe_forward_events")
+        return y
     _check(lib().d2moe_moe_forward(ctypes.byref(cfg.c()), T, _ptr(x), _expert_ptr_array(expert_w),
                                    ctypes.byref(rin), ctypes.byref(rout) if rout is not None else None,
                                    _ptr(y), _ptr(device_status), _ptr(workspace), workspace.numel(),

@@ -199,7 +199,7 @@ static d2moe_status validate_forward(const d2moe_config* c, int64_t T, const voi
 static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x, const void* const* expert_w,
                                  const d2moe_route_in* in, const d2moe_route_out* pre,
                                  const void* residual, void* y, int32_t* device_status, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t st) {
+                                 size_t workspace_bytes, cudaStream_t st, void* const* ev = nullptr) {
     d2moe_status s = validate_forward(c, T, x, expert_w, in, pre, y, workspace, workspace_bytes);
     if (s != D2MOE_OK || T == 0) return s;
     const int n_exp = c->n_experts + c->n_shared;
@@ -211,6 +211,8 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     uint8_t* w = (uint8_t*)workspace;
     RouteBufs R;
     cudaError_t e;
+    auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
+    mark(0);
     if (pre) {
         R = RouteBufs{(int32_t*)pre->topk_idx, (float*)pre->topk_w, (int8_t*)pre->bit_idx,
                       (int32_t*)pre->perm, (int32_t*)pre->inv_perm, (int32_t*)pre->group_off};
@@ -234,9 +236,15 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     if (c->kernel_path == D2MOE_PATH_TENSOR) return D2MOE_ERR_UNSUPPORTED;
     float* hbuf = (float*)(w + ws.off_h);
     float* obuf = (float*)(w + ws.off_o);
-    e = launch_ffn_cuda_core(D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, hbuf, obuf, device_status, st);
+    mark(1);
+    e = launch_gateup_cuda_core(D, Lgu, P, (const __nv_bfloat16*)x, R, hbuf, device_status, st);
     if (e != cudaSuccess) return D2MOE_ERR_CUDA;
+    mark(2);
+    e = launch_down_cuda_core(D, Ld, P, R, hbuf, obuf, device_status, st);
+    if (e != cudaSuccess) return D2MOE_ERR_CUDA;
+    mark(3);
     e = launch_combine(D, R, obuf, 1, (const __nv_bfloat16*)residual, (__nv_bfloat16*)y, st);
+    mark(4);
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
 
@@ -246,6 +254,24 @@ extern "C" d2moe_status d2moe_moe_forward(const d2moe_config* c, int64_t T, cons
                                           void* workspace, size_t workspace_bytes, void* stream) {
     return forward_impl(c, T, x, expert_w, in, pre, nullptr, y, device_status, workspace, workspace_bytes,
                         (cudaStream_t)stream);
+}
+
+extern "C" d2moe_status d2moe_moe_forward_events(const d2moe_config* c, int64_t T, const void* x,
+                                                 const void* const* expert_w, const d2moe_route_in* in,
+                                                 const d2moe_route_out* pre, void* y, int32_t* device_status,
+                                                 void* workspace, size_t workspace_bytes, void* stream,
+                                                 void* const* stage_events) {
+    if (!stage_events) return D2MOE_ERR_NULL;
+    for (int i = 0; i <= D2MOE_N_STAGES; ++i)
+        if (!stage_events[i]) return D2MOE_ERR_NULL;
+    return forward_impl(c, T, x, expert_w, in, pre, nullptr, y, device_status, workspace, workspace_bytes,
+                        (cudaStream_t)stream, stage_events);
+}
+
+extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int routing_precomputed) {
+    if (d2moe_check_config(c) != D2MOE_OK || T <= 0) return 0;
+    const int route = routing_precomputed ? 0 : 4;     // route, count, scan, scatter
+    return route + 3;                                   // gate/up, down, combine
 }
 
 extern "C" d2moe_status d2moe_stack_layer(const d2moe_config* c, int64_t T, void* x, void* xn, float eps,

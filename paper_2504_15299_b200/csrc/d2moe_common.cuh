@@ -138,9 +138,12 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
                          int32_t* device_status, cudaStream_t st);
 
 // kernels_ffn_cc.cu  (plain CUDA-core path)
-cudaError_t launch_ffn_cuda_core(const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
-                                 const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R,
-                                 float* hbuf, float* obuf, int32_t* device_status, cudaStream_t st);
+cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, const ExpertPtrs& P,
+                                    const __nv_bfloat16* x, const RouteBufs& R, float* hbuf,
+                                    int32_t* device_status, cudaStream_t st);
+cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const ExpertPtrs& P,
+                                  const RouteBufs& R, const float* hbuf, float* obuf,
+                                  int32_t* device_status, cudaStream_t st);
 cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* obuf, int n_split,
                            const __nv_bfloat16* residual, __nv_bfloat16* y, cudaStream_t st);
 cudaError_t launch_rmsnorm(int T, int d, float eps, const __nv_bfloat16* x, __nv_bfloat16* xn, cudaStream_t st);

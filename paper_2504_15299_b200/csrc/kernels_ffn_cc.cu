@@ -151,12 +151,19 @@ rmsnorm_kernel(int d, double eps, const __nv_bfloat16* __restrict__ x, __nv_bflo
 
 }  // namespace
 
-cudaError_t launch_ffn_cuda_core(const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
-                                 const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R,
-                                 float* hbuf, float* obuf, int32_t* device_status, cudaStream_t st) {
+cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, const ExpertPtrs& P,
+                                    const __nv_bfloat16* x, const RouteBufs& R, float* hbuf,
+                                    int32_t* device_status, cudaStream_t st) {
     if (D.A_tot == 0) return cudaSuccess;
     dim3 g1((D.F + 7) / 8, D.A_tot);
     gateup_cc_kernel<<<g1, 256, 0, st>>>(D, Lgu, P, x, R, hbuf, device_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const ExpertPtrs& P,
+                                  const RouteBufs& R, const float* hbuf, float* obuf,
+                                  int32_t* device_status, cudaStream_t st) {
+    if (D.A_tot == 0) return cudaSuccess;
     dim3 g2((D.d + 7) / 8, D.A_tot);
     down_cc_kernel<<<g2, 256, 0, st>>>(D, Ld, P, R, hbuf, obuf, device_status);
     return cudaGetLastError();

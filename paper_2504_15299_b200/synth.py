@@ -91,24 +91,29 @@ def _normal_edges(device) -> torch.Tensor:
     return _EDGE_CACHE[key]
 
 
-def _flat_index(shape: Sequence[int], rows: Optional[torch.Tensor], device) -> Tuple[torch.Tensor, Tuple[int, ...]]:
-    """Flat indices of the whole tensor, or of the listed rows of a 2-D tensor."""
-    if rows is None:
+def _flat_index(shape: Sequence[int], rows, cols, device) -> Tuple[torch.Tensor, Tuple[int, ...]]:
+    """Flat indices of the whole tensor, or of the listed rows / columns of a 2-D tensor."""
+    if rows is None and cols is None:
         n = 1
         for s in shape:
             n *= int(s)
         return torch.arange(n, dtype=torch.int64, device=device), tuple(int(s) for s in shape)
-    assert len(shape) == 2, "row sampling is for 2-D tensors"
-    rows = torch.as_tensor(rows, dtype=torch.int64, device=device)
-    cols = int(shape[1])
-    idx = rows[:, None] * cols + torch.arange(cols, dtype=torch.int64, device=device)[None, :]
-    return idx.reshape(-1), (int(rows.numel()), cols)
+    assert len(shape) == 2, "row / column sampling is for 2-D tensors"
+    n_cols = int(shape[1])
+    rows = torch.arange(int(shape[0]), dtype=torch.int64, device=device) if rows is None else \
+        torch.as_tensor(rows, dtype=torch.int64, device=device)
+    cols = torch.arange(n_cols, dtype=torch.int64, device=device) if cols is None else \
+        torch.as_tensor(cols, dtype=torch.int64, device=device)
+    idx = rows[:, None] * n_cols + cols[None, :]
+    return idx.reshape(-1), (int(rows.numel()), int(cols.numel()))
 
 
 def normal(seed: int, tensor_id: int, shape: Sequence[int], sigma: float = 1.0,
-           device="cpu", rows: Optional[torch.Tensor] = None, chunk: int = 1 << 24) -> torch.Tensor:
-    """fp32 tensor ~ "N(0, sigma)" as defined in the module docstring."""
-    idx_all, out_shape = _flat_index(shape, rows, device)
+           device="cpu", rows: Optional[torch.Tensor] = None, cols: Optional[torch.Tensor] = None,
+           chunk: int = 1 << 24) -> torch.Tensor:
+    """fp32 tensor ~ "N(0, sigma)" as defined in the module docstring; ``rows`` / ``cols`` select a
+    sub-matrix of a 2-D tensor (same values as the corresponding entries of the full tensor)."""
+    idx_all, out_shape = _flat_index(shape, rows, cols, device)
     edges = _normal_edges(device)
     out = torch.empty(idx_all.numel(), dtype=torch.float32, device=device)
     for s in range(0, idx_all.numel(), chunk):
@@ -125,7 +130,7 @@ def normal(seed: int, tensor_id: int, shape: Sequence[int], sigma: float = 1.0,
 
 
 def uniform24(seed: int, tensor_id: int, shape: Sequence[int], device="cpu") -> torch.Tensor:
-    idx, out_shape = _flat_index(shape, None, device)
+    idx, out_shape = _flat_index(shape, None, None, device)
     return _lsr(random_bits(seed, tensor_id, idx), 40).reshape(out_shape)
 
 
@@ -200,10 +205,10 @@ def expert_matrix_shape(wl: Workload, m: int) -> Tuple[int, int]:
 
 
 def expert_matrix(wl: Workload, e: int, m: int, device="cpu", layer: int = 0,
-                  rows: Optional[torch.Tensor] = None) -> torch.Tensor:
+                  rows: Optional[torch.Tensor] = None, cols: Optional[torch.Tensor] = None) -> torch.Tensor:
     """fp32 weights ~N(0, sigma_w) of expert ``e`` (shared experts follow the routed ones)."""
     return normal(wl.seed + layer, TID_EXPERT0 + 3 * e + m, expert_matrix_shape(wl, m),
-                  wl.sigma_w, device, rows)
+                  wl.sigma_w, device, rows, cols)
 
 
 def tokens_bf16(wl: Workload, T: int, device="cpu", step: int = 0) -> torch.Tensor:
