@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checks, workspace carving, launches.
 #include "d2moe_common.cuh"
+#include "kernels_ffn_tc.cuh"
 
 #include <string.h>
 
@@ -102,6 +103,11 @@ extern "C" d2moe_status d2moe_unpack_codes(const d2moe_config* c, const void* pa
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
 
+// AUTO takes the tensor-core path whenever the shape allows it; TENSOR insists on it.
+static bool use_tensor_path(const d2moe_config* c) {
+    return c->kernel_path != D2MOE_PATH_CUDA_CORE && tc_path_supported(c);
+}
+
 void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
     const size_t A = (size_t)T * c->top_k;
     const size_t A_tot = A + (size_t)T * c->n_shared;
@@ -118,8 +124,22 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
     ws->off_perm = take(A * 4);
     ws->off_inv_perm = take(A * 4);
     ws->off_group_off = take((n_keys + 1) * 4);
-    ws->off_h = take(A_tot * (size_t)c->d_ffn * 4);
-    ws->off_o = take(A_tot * (size_t)c->d_model * 4);
+    if (use_tensor_path(c)) {
+        TcPlan pl;
+        tc_plan(c, T, &pl);
+        ws->off_units = take((size_t)pl.max_units * sizeof(TcUnit));
+        ws->off_n_units = take(256);
+        ws->off_pad_off = take((n_keys + c->n_shared + 1) * 4);
+        ws->off_row_map = take(A_tot * 4);
+        ws->off_src_token = take((size_t)pl.R_alloc * 4);
+        ws->off_xp16 = take((size_t)pl.R_alloc * c->d_model * 2);
+        ws->off_h = take((size_t)pl.R_alloc * c->d_ffn * 2);
+        ws->off_o = take((size_t)pl.n_split * pl.R_alloc * c->d_model * 4);
+    } else {
+        ws->off_units = ws->off_n_units = ws->off_pad_off = ws->off_row_map = ws->off_src_token = ws->off_xp16 = 0;
+        ws->off_h = take(A_tot * (size_t)c->d_ffn * 4);
+        ws->off_o = take(A_tot * (size_t)c->d_model * 4);
+    }
     ws->total = off;
 }
 
@@ -190,6 +210,7 @@ static d2moe_status validate_forward(const d2moe_config* c, int64_t T, const voi
         s = check_route_inputs(in->gate_w_bf16, in->logits, in->bit_w_bf16, in->forced_bit_idx);
         if (s != D2MOE_OK) return s;
     }
+    if (c->kernel_path == D2MOE_PATH_TENSOR && !tc_path_supported(c)) return D2MOE_ERR_UNSUPPORTED;
     Workspace ws;
     d2moe_carve_workspace(c, T, &ws);
     if (workspace_bytes < ws.total) return D2MOE_ERR_WORKSPACE;
@@ -233,7 +254,22 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     d2moe_make_layout(Lgu, c->bits, c->n_bits, c->group_size, c->d_ffn, c->d_model);
     d2moe_make_layout(Ld, c->bits, c->n_bits, c->group_size, c->d_model, c->d_ffn);
 
-    if (c->kernel_path == D2MOE_PATH_TENSOR) return D2MOE_ERR_UNSUPPORTED;
+    if (use_tensor_path(c)) {
+        TcPlan pl;
+        tc_plan(c, T, &pl);
+        TcBuffers B;
+        B.units = (TcUnit*)(w + ws.off_units); B.n_units = (int*)(w + ws.off_n_units);
+        B.pad_off = (int32_t*)(w + ws.off_pad_off); B.row_map = (int32_t*)(w + ws.off_row_map);
+        B.src_token = (int32_t*)(w + ws.off_src_token);
+        B.xp16 = (__half*)(w + ws.off_xp16); B.h16 = (__half*)(w + ws.off_h); B.o32 = (float*)(w + ws.off_o);
+        e = launch_ffn_tensor(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev);
+        if (e != cudaSuccess) return D2MOE_ERR_CUDA;
+        mark(3);
+        e = launch_combine(D, R, B.o32, pl.n_split, (size_t)pl.R_alloc * D.d, B.row_map,
+                           (const __nv_bfloat16*)residual, (__nv_bfloat16*)y, st);
+        mark(4);
+        return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+    }
     float* hbuf = (float*)(w + ws.off_h);
     float* obuf = (float*)(w + ws.off_o);
     mark(1);
@@ -243,7 +279,8 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     e = launch_down_cuda_core(D, Ld, P, R, hbuf, obuf, device_status, st);
     if (e != cudaSuccess) return D2MOE_ERR_CUDA;
     mark(3);
-    e = launch_combine(D, R, obuf, 1, (const __nv_bfloat16*)residual, (__nv_bfloat16*)y, st);
+    e = launch_combine(D, R, obuf, 1, (size_t)D.A_tot * D.d, nullptr, (const __nv_bfloat16*)residual,
+                       (__nv_bfloat16*)y, st);
     mark(4);
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
@@ -271,6 +308,7 @@ extern "C" d2moe_status d2moe_moe_forward_events(const d2moe_config* c, int64_t 
 extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int routing_precomputed) {
     if (d2moe_check_config(c) != D2MOE_OK || T <= 0) return 0;
     const int route = routing_precomputed ? 0 : 4;     // route, count, scan, scatter
+    if (use_tensor_path(c)) return route + 5;           // unit build, gather, gate/up, down, combine
     return route + 3;                                   // gate/up, down, combine
 }
 

@@ -48,7 +48,8 @@ struct PackHeader {
     int32_t rows, cols, g, n_bits;
     int32_t bits[8];
     uint32_t s1_max_bits;          // bit pattern of the largest fp32 s1 in the matrix
-    uint32_t pad[49];
+    uint32_t wabs_max_bits;        // bit pattern of the largest |W| in the matrix
+    uint32_t pad[48];
 };
 static_assert(sizeof(PackHeader) == D2MOE_HEADER_BYTES, "header size");
 
@@ -121,6 +122,7 @@ struct Workspace {
     size_t off_logits, off_keys, off_hist;
     size_t off_topk_idx, off_topk_w, off_bit_idx, off_perm, off_inv_perm, off_group_off;
     size_t off_h, off_o, off_status;
+    size_t off_units, off_n_units, off_pad_off, off_row_map, off_src_token, off_xp16;   // tensor-core path
 };
 
 void d2moe_carve_workspace(const d2moe_config* cfg, long long max_tokens, Workspace* ws);
@@ -145,5 +147,6 @@ cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const 
                                   const RouteBufs& R, const float* hbuf, float* obuf,
                                   int32_t* device_status, cudaStream_t st);
 cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* obuf, int n_split,
-                           const __nv_bfloat16* residual, __nv_bfloat16* y, cudaStream_t st);
+                           size_t split_stride, const int32_t* row_map, const __nv_bfloat16* residual,
+                           __nv_bfloat16* y, cudaStream_t st);
 cudaError_t launch_rmsnorm(int T, int d, float eps, const __nv_bfloat16* x, __nv_bfloat16* xn, cudaStream_t st);

@@ -170,10 +170,11 @@ cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const 
 }
 
 cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* obuf, int n_split,
-                           const __nv_bfloat16* residual, __nv_bfloat16* y, cudaStream_t st) {
+                           size_t split_stride, const int32_t* row_map, const __nv_bfloat16* residual,
+                           __nv_bfloat16* y, cudaStream_t st) {
     if (D.T == 0) return cudaSuccess;
     dim3 grid((D.d + 255) / 256, D.T);
-    combine_kernel<<<grid, 256, 0, st>>>(D, R, obuf, n_split, (size_t)D.A_tot * D.d, nullptr, residual, y);
+    combine_kernel<<<grid, 256, 0, st>>>(D, R, obuf, n_split, split_stride, row_map, residual, y);
     return cudaGetLastError();
 }
 

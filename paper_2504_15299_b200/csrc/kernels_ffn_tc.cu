@@ -1,0 +1,727 @@
+// Grouped dequant-GEMM on the 5th-generation tensor cores (tcgen05 + TMEM) for the expert FFN.
+//
+// One CTA computes, for one (unit, 128-row tile) pair, D[128 weight rows, N tokens] over a range of
+// K-groups.  A "unit" is up to n_cap consecutive columns (tokens) of one expert in the padded,
+// (expert, width)-sorted activation buffer; it holds one piece per routed width, each padded to a
+// multiple of 16 columns.  Weight rows sit on the MMA's M side (TMEM lanes), tokens on N.
+//
+// Per K-group (g input columns) the four dequant warps own one weight row each (thread = row = TMEM
+// lane).  A thread reads its row's packed segments from shared memory and builds the fp16 weights
+// width by width, in registers, using the additivity of the nested code (Section 3.3.1,
+// W_hat_{b_k} = W_hat_{b_1} + sum of the residual terms):
+//     U_0  = (lo - s1/2) + s1 * v_0                       v_j = value of segment j
+//     U_j  = U_{j-1} + M_j * v_j,   M_j = s1 / 2^(bits[j]-bits[0])
+//     W_hat at width bits[j] = U_j + M_j / 2
+// Each step is one AND (isolates a code pair inside the fp16 subnormal range, where a bit pattern
+// v << p is the value v * 2^(p-24)) and one packed half-precision FMA with a pre-scaled multiplier.
+// Every width that has tokens in the unit gets its tile written to TMEM (tcgen05.st) and one
+// tcgen05.mma (A from TMEM, B = the tokens of that width from shared memory) accumulates it into
+// the D columns of those tokens, so each packed byte is read once from HBM however many widths
+// use it (the plane reuse of Section 3.4), and each token is multiplied exactly once.
+// All tiles carry a common power-of-two factor 2^-S (S per matrix, from the largest scale seen at
+// pack time) so that the multipliers stay inside fp16 range; the epilogue multiplies by 2^S.
+//
+// Warp roles (224 threads, 2 CTAs per SM): 0-3 dequant + epilogue, 4 weight producer (bulk async
+// copies of packed blocks, HBM -> shared), 5 activation producer (TMA tensor loads, 128B swizzle),
+// 6 MMA issuer.  Every wait is bounded: on expiry the CTA raises D2MOE_DEV_TIMEOUT, stops
+// waiting, drains and exits.
+#include "d2moe_common.cuh"
+#include "kernels_ffn_tc.cuh"
+
+#include <cuda.h>
+
+namespace {
+
+constexpr int TC_THREADS = 224;
+constexpr int WARP_WPROD = 4, WARP_BPROD = 5, WARP_MMA = 6;
+constexpr int TMEM_COLS = 256;
+constexpr int D_COLS = 128;            // accumulator columns (n_cap <= 128)
+constexpr int A_SLOTS = 2;
+constexpr int NSB = 2;                 // activation ring depth
+constexpr int MAX_NSW = 8;             // weight ring depth (upper bound)
+constexpr int EPI_STRIDE = 17;
+
+struct TmaMaps { CUtensorMap m[5]; };  // box heights 16, 32, 64, 128, 256
+
+struct TcParams {
+    MoeDims D;
+    PackLayout L;
+    ExpertPtrs P;
+    int mode;                 // 0: gate/up + SwiGLU -> hbuf;  1: down -> obuf
+    int n_cap, n_row_tiles, n_split, groups_per_split, nsw;
+    const TcUnit* units;
+    const int* n_units;
+    __half* hbuf;             // [R, F]
+    float* obuf;              // [n_split][R, d]
+    long long R_alloc;
+    int32_t* status;
+    int smem_w_off, smem_epi_off, smem_bar_off;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  `abort_flag` (shared) is set by the first wait that runs out (about one second);
+// once it is set no wait blocks any more, so the CTA drains and exits instead of hanging.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          bool drain = false) {
+    if (mbar_try(bar, parity)) return;
+    unsigned long long t0 = 0;
+    for (unsigned spin = 0;; ++spin) {
+        if (mbar_try(bar, parity)) return;
+        if ((spin & 255u) == 255u) {
+            if (*abort_flag && !drain) return;      // a drain wait keeps its own one-second limit
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 1000000000ull) {
+                *abort_flag = 1;
+                if (status) atomicOr(status, D2MOE_DEV_TIMEOUT);
+                return;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]; fp16 inputs, fp32 accumulation
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                   "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled shared-memory operand: 8-row atoms of 1024 bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);         // start address
+    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset: next 8-row atom
+    d |= (uint64_t)1 << 46;                           // descriptor version
+    d |= (uint64_t)2 << 61;                           // 128B swizzle
+    return d;
+}
+// fp16 x fp16 -> fp32, A and B K-major, M = 128
+__device__ __forceinline__ uint32_t instr_desc_f16(int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ __half2 h2dup(float v) { return __float2half2_rn(v); }
+__device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+__device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
+// exponent S of the common factor 2^-S from the header of a packed matrix
+__device__ __forceinline__ int matrix_exponent(const uint8_t* packed) {
+    const PackHeader* h = reinterpret_cast<const PackHeader*>(packed);
+    const float s1max = __uint_as_float(h->s1_max_bits);
+    const float wabs = __uint_as_float(h->wabs_max_bits) + 4.0f * s1max;
+    int e1, e2;
+    frexpf(s1max, &e1);            // s1max = m * 2^e1, 0.5 <= m < 1  =>  s1max <= 2^e1
+    frexpf(wabs, &e2);
+    int S = e1 + 9;                // s1max * 2^(24 - S) <= 2^15
+    if (e2 - 15 > S) S = e2 - 15;  // |tile| <= 2^15
+    return S;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dequantization of one segment of one row into the running tile.
+//   seg     shared-memory address of the segment inside the block (this row's chunks are at
+//           (c*64 + rr)*cs)
+//   acc     running tile U (GS/2 half2 registers: register i = elements 2i, 2i+1 of the group)
+//   m0      multiplier for a code at bit position 0: M_j * 2^(24 - S); position p uses m0 * 2^-p
+//   FIRST   segment 0: the addend is u0 = (lo - s1/2) * 2^-S instead of acc
+// ------------------------------------------------------------------------------------------------
+template <int GS, int SW, bool FIRST>
+__device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, __half2 (&acc)[GS / 2], __half2 m0, __half2 u0) {
+    constexpr int ROW_BYTES = GS * SW / 8;
+    constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
+    constexpr int NCHUNK = ROW_BYTES / CS;
+    constexpr int WPC = CS / 4;                 // words per chunk
+    constexpr int PER = 16 / SW;                // registers per word
+    constexpr int NPOS = 8 / SW;                // distinct bit positions per byte lane
+    constexpr uint32_t FIELD = ((1u << SW) - 1u) * 0x00010001u;
+    __half2 mult[NPOS];
+    mult[0] = m0;
+    const __half2 step = __float2half2_rn(1.0f / (float)(1 << SW));     // exact power of two
+#pragma unroll
+    for (int q = 1; q < NPOS; ++q) mult[q] = __hmul2(mult[q - 1], step);
+#pragma unroll
+    for (int c = 0; c < NCHUNK; ++c) {
+        uint32_t w[WPC];
+        const uint32_t addr = seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS);
+        if constexpr (WPC == 4) {
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+        } else if constexpr (WPC == 2) {
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr));
+        } else {
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[0]) : "r"(addr));
+        }
+#pragma unroll
+        for (int q = 0; q < WPC; ++q) {
+            const int m = c * WPC + q;
+            const uint32_t lo8 = w[q], hi8 = w[q] >> 8;
+#pragma unroll
+            for (int e = 0; e < PER; ++e) {
+                const int pos = (e % NPOS) * SW;
+                const uint32_t src = e < NPOS ? lo8 : hi8;
+                const __half2 code = as_h2(src & (FIELD << pos));
+                const int i = m * PER + e;
+                acc[i] = __hfma2(code, mult[e % NPOS], FIRST ? u0 : acc[i]);
+            }
+        }
+    }
+}
+
+template <int GS, bool FIRST>
+__device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, __half2 (&acc)[GS / 2], __half2 m0, __half2 u0) {
+    switch (sw) {
+        case 1: dequant_segment<GS, 1, FIRST>(seg, rr, acc, m0, u0); break;
+        case 2: dequant_segment<GS, 2, FIRST>(seg, rr, acc, m0, u0); break;
+        case 4: dequant_segment<GS, 4, FIRST>(seg, rr, acc, m0, u0); break;
+        default: dequant_segment<GS, 8, FIRST>(seg, rr, acc, m0, u0); break;
+    }
+}
+
+struct ItemInfo {
+    int unit, tile, split, g0, g1;
+};
+
+__device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
+    ItemInfo it;
+    const int per_unit = p.n_row_tiles * p.n_split;
+    it.unit = item / per_unit;
+    const int rem = item - it.unit * per_unit;
+    it.tile = rem / p.n_split;
+    it.split = rem - it.tile * p.n_split;
+    it.g0 = it.split * p.groups_per_split;
+    it.g1 = min(p.L.n_groups, it.g0 + p.groups_per_split);
+    return it;
+}
+
+// ------------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------------
+template <int GS>
+__global__ void __launch_bounds__(TC_THREADS, 2)
+ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMaps maps) {
+    extern __shared__ uint8_t smem_raw[];
+    // shared layout (from a 1024-byte boundary, which the 128B-swizzled operand tiles need):
+    // [activation ring: NSB x n_cap*GS*2] [weight ring: nsw x 2 blocks] [epilogue] [barriers]
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t b_slot_bytes = (uint32_t)p.n_cap * GS * 2;
+    const uint32_t w_slot_bytes = 2u * (uint32_t)p.L.block_bytes;
+    const uint32_t bbuf = smem_base;
+    const uint32_t wbuf = smem_base + p.smem_w_off;
+    float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.smem_bar_off);
+    // barrier indices
+    const uint32_t bar0 = smem_u32(bars);
+    auto W_FULL = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    auto W_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(MAX_NSW + i); };
+    auto B_FULL = [&](int i) { return bar0 + 8u * (uint32_t)(2 * MAX_NSW + i); };
+    auto B_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(2 * MAX_NSW + NSB + i); };
+    auto A_FULL = [&](int i) { return bar0 + 8u * (uint32_t)(2 * MAX_NSW + 2 * NSB + i); };
+    auto A_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(2 * MAX_NSW + 2 * NSB + A_SLOTS + i); };
+    const uint32_t D_FULL = bar0 + 8u * (uint32_t)(2 * MAX_NSW + 2 * NSB + 2 * A_SLOTS);
+    const uint32_t D_EMPTY = D_FULL + 8u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_NSW + 2 * NSB + 2 * A_SLOTS + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 128); }
+        for (int i = 0; i < NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 1); }
+        for (int i = 0; i < A_SLOTS; ++i) { mbar_init(A_FULL(i), 128); mbar_init(A_EMPTY(i), 1); }
+        mbar_init(D_FULL, 1);
+        mbar_init(D_EMPTY, 128);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == WARP_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t d_tmem = tmem_base;                       // columns [0, 128)
+    const uint32_t a_tmem = tmem_base + D_COLS;              // A_SLOTS tiles of GS/2 columns
+
+    const int n_units = *p.n_units;
+    const int total_items = n_units * p.n_row_tiles * p.n_split;
+    const int nsw = p.nsw;
+
+    if (warp == WARP_WPROD) {
+        // ---------------- weight producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+                const ItemInfo ii = decode_item(p, item);
+                const TcUnit* u = p.units + ii.unit;
+                const int e = u->e, kmax = u->kmax;
+                const uint32_t bytes = (uint32_t)p.L.seg_off[kmax + 1];
+                const uint8_t *m0, *m1;
+                int rt0, rt1;
+                if (p.mode == 0) { m0 = p.P.w[3 * e + 0]; m1 = p.P.w[3 * e + 1]; rt0 = rt1 = ii.tile; }
+                else { m0 = m1 = p.P.w[3 * e + 2]; rt0 = 2 * ii.tile; rt1 = 2 * ii.tile + 1; }
+                for (int G = ii.g0; G < ii.g1; ++G, ++it) {
+                    const int s = it % nsw;
+                    mbar_wait(W_EMPTY(s), ((it / nsw) & 1) ^ 1, abort_flag, p.status);
+                    mbar_expect_tx(W_FULL(s), 2 * bytes);
+                    const uint32_t dst = wbuf + s * w_slot_bytes;
+                    bulk_g2s(dst, m0 + d2moe_block_offset(p.L, rt0, G), bytes, W_FULL(s));
+                    bulk_g2s(dst + p.L.block_bytes, m1 + d2moe_block_offset(p.L, rt1, G), bytes, W_FULL(s));
+                }
+            }
+            // drain: every copy issued must have landed before the CTA may exit
+            for (int s = 0; s < nsw && s < (int)it; ++s) {
+                const uint32_t last = it - 1 - ((it - 1 - s) % nsw + nsw) % nsw;   // last iteration that used slot s
+                mbar_wait(W_FULL(s), (last / nsw) & 1, abort_flag, p.status, true);
+            }
+        }
+    } else if (warp == WARP_BPROD) {
+        // ---------------- activation producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+                const ItemInfo ii = decode_item(p, item);
+                const TcUnit* u = p.units + ii.unit;
+                const int ncols = u->ncols;
+                int mi = 0, box = 16;
+                while (box < ncols) { box <<= 1; ++mi; }
+                const uint32_t bytes = (uint32_t)box * 128u * (GS / 64);
+                for (int G = ii.g0; G < ii.g1; ++G, ++it) {
+                    const int s = it % NSB;
+                    mbar_wait(B_EMPTY(s), ((it / NSB) & 1) ^ 1, abort_flag, p.status);
+                    mbar_expect_tx(B_FULL(s), bytes);
+                    const uint32_t dst = bbuf + s * b_slot_bytes;
+#pragma unroll
+                    for (int h = 0; h < GS / 64; ++h)
+                        tma_load_2d(dst + h * (uint32_t)p.n_cap * 128u, &maps.m[mi], G * GS + h * 64, u->row0, B_FULL(s));
+                }
+            }
+            for (int s = 0; s < NSB && s < (int)it; ++s) {
+                const uint32_t last = it - 1 - ((it - 1 - s) % NSB + NSB) % NSB;
+                mbar_wait(B_FULL(s), (last / NSB) & 1, abort_flag, p.status, true);
+            }
+        }
+    } else if (warp == WARP_MMA) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            uint32_t it = 0, at = 0, ic = 0;
+            for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
+                const ItemInfo ii = decode_item(p, item);
+                const TcUnit* u = p.units + ii.unit;
+                const int kmax = u->kmax;
+                mbar_wait(D_EMPTY, (ic & 1) ^ 1, abort_flag, p.status);
+                tc_fence_after();
+                for (int G = ii.g0; G < ii.g1; ++G, ++it) {
+                    const int s = it % NSB;
+                    mbar_wait(B_FULL(s), (it / NSB) & 1, abort_flag, p.status);
+                    const uint32_t bsl = bbuf + s * b_slot_bytes;
+                    for (int kk = 0; kk <= kmax; ++kk) {
+                        const int cnt = u->cnt[kk];
+                        if (cnt == 0) continue;
+                        const int slot = at % A_SLOTS;
+                        mbar_wait(A_FULL(slot), (at / A_SLOTS) & 1, abort_flag, p.status);
+                        tc_fence_after();
+                        const uint32_t idesc = instr_desc_f16(cnt);
+                        const int col0 = u->col0[kk];
+#pragma unroll
+                        for (int j = 0; j < GS / 16; ++j) {
+                            const uint32_t a_addr = a_tmem + slot * (GS / 2) + j * 8;
+                            const uint32_t b_addr = bsl + (j >> 2) * (uint32_t)p.n_cap * 128u + (uint32_t)col0 * 128u + (j & 3) * 32u;
+                            tc_mma_ts(d_tmem + col0, a_addr, smem_desc_sw128(b_addr), idesc,
+                                      (G != ii.g0 || j != 0) ? 1u : 0u);
+                        }
+                        tc_commit(A_EMPTY(slot));
+                        ++at;
+                    }
+                    tc_commit(B_EMPTY(s));
+                }
+                tc_commit(D_FULL);
+            }
+            // all MMAs must be complete before TMEM is freed
+            if (ic > 0) mbar_wait(D_FULL, (ic - 1) & 1, abort_flag, p.status, true);
+        }
+    } else {
+        // ---------------- dequant + epilogue warps ----------------
+        const int r = threadIdx.x;               // row of the tile = TMEM lane
+        const int blk = r >> 6, rr = r & 63;
+        const uint32_t lane_addr = ((uint32_t)(warp * 32)) << 16;
+        uint32_t it = 0, at = 0, ic = 0;
+        __half2 acc[GS / 2];
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
+            const ItemInfo ii = decode_item(p, item);
+            const TcUnit* u = p.units + ii.unit;
+            const int e = u->e, kmax = u->kmax;
+            const uint8_t* mat = p.mode == 0 ? p.P.w[3 * e + blk] : p.P.w[3 * e + 2];
+            const int S = matrix_exponent(mat);
+            const float two_mS = exp2f((float)-S);
+            unsigned present = 0;
+            for (int kk = 0; kk <= kmax; ++kk) present |= (u->cnt[kk] > 0 ? 1u : 0u) << kk;
+
+            for (int G = ii.g0; G < ii.g1; ++G, ++it) {
+                const int s = it % nsw;
+                mbar_wait(W_FULL(s), (it / nsw) & 1, abort_flag, p.status);
+                const uint32_t wb = wbuf + s * w_slot_bytes + blk * p.L.block_bytes;
+                uint32_t meta;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
+                const __half2 mh = as_h2(meta);
+                const float s1 = __low2float(mh), lo = __high2float(mh);
+                const __half2 u0 = h2dup((lo - 0.5f * s1) * two_mS);
+#pragma unroll 1
+                for (int kk = 0; kk <= kmax; ++kk) {
+                    const int sw = p.L.seg_sw[kk];
+                    // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
+                    const float Mk = s1 * exp2f((float)(-(p.D.bits[kk] - p.D.bits[0]))) * two_mS;
+                    const __half2 m0 = h2dup(Mk * 16777216.0f);
+                    const uint32_t seg = wb + (uint32_t)p.L.seg_off[kk];
+                    if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, acc, m0, u0);
+                    else dequant_dispatch<GS, false>(sw, seg, rr, acc, m0, u0);
+                    if ((present >> kk) & 1u) {
+                        const int slot = at % A_SLOTS;
+                        mbar_wait(A_EMPTY(slot), ((at / A_SLOTS) & 1) ^ 1, abort_flag, p.status);
+                        tc_fence_after();
+                        const __half2 half_m = h2dup(0.5f * Mk);
+                        const uint32_t dst = a_tmem + slot * (GS / 2) + lane_addr;
+#pragma unroll
+                        for (int c = 0; c < GS / 32; ++c) {
+                            uint32_t v[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[j] = as_u32(__hadd2(acc[c * 16 + j], half_m));
+                            tc_st16(dst + c * 16, v);
+                        }
+                        tc_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(A_FULL(slot));
+                        ++at;
+                    }
+                }
+                mbar_arrive(W_EMPTY(s));
+            }
+
+            // ---- epilogue: D (128 rows x ncols) -> global ----
+            mbar_wait(D_FULL, ic & 1, abort_flag, p.status);
+            tc_fence_after();
+            const float two_S = exp2f((float)S);
+            const int ncols = u->ncols;
+            for (int c0 = 0; c0 < ncols; c0 += 16) {
+                int nreal = 0;
+                for (int kk = 0; kk <= kmax; ++kk) {
+                    const int rel = c0 - u->col0[kk];
+                    if (u->cnt[kk] > 0 && rel >= 0 && rel < u->cnt[kk]) nreal = min(16, max(0, u->real[kk] - rel));
+                }
+                if (nreal == 0) continue;            // padding columns only (uniform across the CTA)
+                uint32_t v[16];
+                tc_ld16(d_tmem + lane_addr + c0, v);
+                tc_wait_ld();
+                const long long grow = u->row0 + c0;
+                if (p.mode == 0) {
+                    if (blk == 1) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) epi[rr * EPI_STRIDE + j] = __uint_as_float(v[j]) * two_S;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (blk == 0) {
+                        __half* dst = p.hbuf + grow * p.D.F + (long long)ii.tile * 64 + rr;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (j < nreal) {
+                                const float g = __uint_as_float(v[j]) * two_S;
+                                const float up = epi[rr * EPI_STRIDE + j];
+                                dst[(long long)j * p.D.F] = __float2half_rn(g / (1.0f + __expf(-g)) * up);
+                            }
+                        }
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                } else {
+                    float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + r;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (j < nreal) dst[(long long)j * p.D.d] = __uint_as_float(v[j]) * two_S;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(D_EMPTY);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == WARP_MMA) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Unit construction and activation gather
+// ------------------------------------------------------------------------------------------------
+// One block.  Pads every (expert, width) group to a multiple of 16 rows, lays the groups out
+// contiguously (routed experts, then shared experts), cuts each expert's range into units of at
+// most n_cap rows, and records for every assignment its padded row.
+__global__ void __launch_bounds__(256)
+tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, int32_t* pad_off,
+               int32_t* row_map, int32_t* src_token, int max_units) {
+    __shared__ int s_total_rows, s_n_units;
+    const int n_keys = D.E * D.K + D.n_shared;
+    // 1. padded offsets (one warp scans)
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int base = 0; base < n_keys; base += 32) {
+            const int i = base + lane;
+            int n = 0;
+            if (i < D.E * D.K) n = R.group_off[i + 1] - R.group_off[i];
+            else if (i < n_keys) n = D.T;
+            const int v = (n + 15) & ~15;
+            int incl = v;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (i < n_keys) pad_off[i] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) { pad_off[n_keys] = carry; s_total_rows = carry; }
+    }
+    __syncthreads();
+    const int total_rows = s_total_rows;
+    // 2. source token of every padded row (-1 = padding)
+    for (int i = threadIdx.x; i < total_rows; i += blockDim.x) src_token[i] = -1;
+    __syncthreads();
+    for (int a = threadIdx.x; a < D.A; a += blockDim.x) {
+        const int pos = R.inv_perm[a];
+        const int e = R.topk_idx[a], kk = R.bit_idx[a];
+        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) { row_map[a] = 0; continue; }
+        const int key = e * D.K + kk;
+        const int row = pad_off[key] + (pos - R.group_off[key]);
+        row_map[a] = row;
+        if (row >= 0 && row < total_rows) src_token[row] = a / D.k;
+    }
+    for (int i = threadIdx.x; i < D.n_shared * D.T; i += blockDim.x) {
+        const int s = i / D.T, t = i - s * D.T;
+        const int row = pad_off[D.E * D.K + s] + t;
+        row_map[D.A + i] = row;
+        src_token[row] = t;
+    }
+    // 3. units (serial over experts: at most a few hundred)
+    if (threadIdx.x == 0) {
+        int nu = 0;
+        for (int e = 0; e < D.E + D.n_shared; ++e) {
+            const int key0 = e < D.E ? e * D.K : D.E * D.K + (e - D.E);
+            const int key1 = e < D.E ? key0 + D.K : key0 + 1;
+            const int p0 = pad_off[key0], p1 = pad_off[key1];
+            for (int start = p0; start < p1 && nu < max_units; start += n_cap) {
+                const int end = min(p1, start + n_cap);
+                TcUnit u;
+                u.e = e; u.row0 = start; u.ncols = end - start; u.kmax = 0;
+                for (int kk = 0; kk < 8; ++kk) { u.col0[kk] = 0; u.cnt[kk] = 0; u.real[kk] = 0; }
+                for (int key = key0; key < key1; ++key) {
+                    const int kk = e < D.E ? key - key0 : D.K - 1;
+                    const int a0 = pad_off[key], a1 = pad_off[key + 1];
+                    const int n_real = e < D.E ? R.group_off[key + 1] - R.group_off[key] : D.T;
+                    const int lo = max(a0, start), hi = min(a1, end);
+                    if (hi <= lo) continue;
+                    u.col0[kk] = lo - start;
+                    u.cnt[kk] = hi - lo;
+                    u.real[kk] = max(0, min(hi, a0 + n_real) - lo);
+                    u.kmax = kk;
+                }
+                units[nu++] = u;
+            }
+        }
+        *n_units = nu;
+        s_n_units = nu;
+    }
+}
+
+// xp16[row, :] = fp16(x[src_token[row], :]) for the real rows (padding rows are never consumed:
+// a D column depends only on its own token row).
+__global__ void __launch_bounds__(256)
+tc_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ src_token,
+                 const int32_t* __restrict__ pad_off, int n_keys, __half* __restrict__ xp16) {
+    const int total_rows = pad_off[n_keys];
+    for (int row = blockIdx.x; row < total_rows; row += gridDim.x) {
+        const int t = src_token[row];
+        if (t < 0) continue;
+        const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(x + (size_t)t * d);
+        __half2* dst = reinterpret_cast<__half2*>(xp16 + (size_t)row * d);
+        for (int i = threadIdx.x; i < d / 2; i += blockDim.x) {
+            const float2 f = __bfloat1622float2(src[i]);
+            dst[i] = __floats2half2_rn(f.x, f.y);
+        }
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    return fn;
+}
+
+bool make_maps(TmaMaps* maps, void* base, long long rows, long long cols) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    for (int i = 0; i < 5; ++i) {
+        cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)(16 << i)};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&maps->m[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    return true;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+bool tc_path_supported(const d2moe_config* c) {
+    if (c->group_size != 64 && c->group_size != 128) return false;
+    if (c->d_ffn % 64 || c->d_model % 128) return false;
+    return true;
+}
+
+void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
+    const long long A = T * c->top_k, A_tot = A + T * c->n_shared;
+    const long long avg = (A + c->n_experts - 1) / c->n_experts;
+    pl->n_cap = (avg <= 24) ? 64 : 128;
+    const long long n_pieces = (long long)c->n_experts * c->n_bits + c->n_shared;
+    long long pad_rows = A_tot + 15 * (n_pieces < A_tot ? n_pieces : A_tot);
+    pl->R_alloc = ((pad_rows + 255) / 256) * 256 + 256;
+    pl->max_units = (int)(c->n_experts + c->n_shared + pl->R_alloc / pl->n_cap + 1);
+    // split-K of the down projection: aim for >= 4 work items per resident CTA (2 per SM, 148 SMs)
+    const long long units_est = (c->n_experts < A ? c->n_experts : A) + (long long)c->n_shared * ((T + pl->n_cap - 1) / pl->n_cap);
+    const long long tiles = c->d_model / 128;
+    const int n_groups = c->d_ffn / c->group_size;
+    long long want = (4 * 296 + units_est * tiles - 1) / (units_est * tiles);
+    if (want < 1) want = 1;
+    if (want > 8) want = 8;
+    if (want > n_groups / 4) want = n_groups / 4 > 0 ? n_groups / 4 : 1;
+    pl->groups_per_split = (int)((n_groups + want - 1) / want);
+    pl->n_split = (n_groups + pl->groups_per_split - 1) / pl->groups_per_split;
+}
+
+cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                              const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
+                              const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
+    auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
+    const int n_keys = D.E * D.K + D.n_shared;
+    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units);
+    tc_gather_kernel<<<296, 256, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16);
+
+    TmaMaps maps_x, maps_h;
+    if (!make_maps(&maps_x, B.xp16, pl.R_alloc, D.d) || !make_maps(&maps_h, B.h16, pl.R_alloc, D.F))
+        return cudaErrorNotSupported;
+
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+
+    for (int mode = 0; mode < 2; ++mode) {
+        TcParams p;
+        p.D = D; p.L = mode == 0 ? Lgu : Ld; p.P = P; p.mode = mode;
+        p.n_cap = pl.n_cap;
+        p.n_row_tiles = mode == 0 ? D.F / 64 : D.d / 128;
+        p.n_split = mode == 0 ? 1 : pl.n_split;
+        p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
+        p.units = B.units; p.n_units = B.n_units;
+        p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
+        const int b_bytes = NSB * pl.n_cap * D.g * 2;
+        const int w_slot = 2 * p.L.block_bytes;
+        const int epi_bytes = 64 * EPI_STRIDE * 4;
+        const int bar_bytes = 512;
+        const int budget = 112 * 1024;
+        int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
+        if (nsw > MAX_NSW) nsw = MAX_NSW;
+        if (nsw < 2) return cudaErrorInvalidConfiguration;
+        p.nsw = nsw;
+        p.smem_w_off = b_bytes;
+        p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
+        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;   // + slack for the 1024-byte alignment
+        mark(mode == 0 ? 1 : 2);
+        cudaError_t e;
+        if (D.g == 128) {
+            e = cudaFuncSetAttribute(ffn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (e != cudaSuccess) return e;
+            ffn_tc_kernel<128><<<2 * sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+        } else {
+            e = cudaFuncSetAttribute(ffn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (e != cudaSuccess) return e;
+            ffn_tc_kernel<64><<<2 * sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+        }
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}

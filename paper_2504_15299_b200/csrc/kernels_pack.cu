@@ -12,7 +12,7 @@ __global__ void pack_header_kernel(PackHeader* h, PackLayout L, int n_bits,
         h->rows = L.rows; h->cols = L.cols; h->g = L.g; h->n_bits = n_bits;
         int b[8] = {b0, b1, b2, b3, b4, b5, b6, b7};
         for (int i = 0; i < 8; ++i) h->bits[i] = b[i];
-        // s1_max_bits was zeroed by the memset that precedes this kernel
+        // s1_max_bits and wabs_max_bits were zeroed by the memset that precedes this kernel
     }
 }
 
@@ -29,7 +29,7 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
     uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float levels = (float)((1 << L.b1) - 1);
-    unsigned s1_max_local = 0;
+    unsigned s1_max_local = 0, wabs_max_local = 0;
 
     for (int r = warp; r < D2MOE_TILE_ROWS; r += PACK_THREADS / 32) {
         const long long row = (long long)rt * D2MOE_TILE_ROWS + r;
@@ -71,10 +71,13 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
             __half2 m = __halves2half2(s1_h, lo_h);          // low half = s1, high half = lo
             reinterpret_cast<__half2*>(blk)[r] = m;
             s1_max_local = max(s1_max_local, __float_as_uint(s1));
+            wabs_max_local = max(wabs_max_local, __float_as_uint(fmaxf(fabsf(wmin), fabsf(wmax))));
         }
     }
-    if (lane == 0 && s1_max_local)
+    if (lane == 0 && s1_max_local) {
         atomicMax(&reinterpret_cast<PackHeader*>(packed)->s1_max_bits, s1_max_local);
+        atomicMax(&reinterpret_cast<PackHeader*>(packed)->wabs_max_bits, wabs_max_local);
+    }
     __syncthreads();
 
     for (int j = 0; j < L.n_seg; ++j) {

@@ -191,16 +191,59 @@ def run_layer(B, cfg, wl, T, *, tokens=None, kernel_path=None, blobs=None):
     return errs, y, blobs
 
 
-@pytest.mark.parametrize("path", [1])
+@pytest.mark.parametrize("path", [1, 2])
 def test_layer_tiny(B, path):
     wl = synth.WORKLOADS["tiny"]
     errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 16, kernel_path=path)
     assert len(errs) == 16 and max(errs.values()) < TOL, errs
 
 
-def test_layer_finegrained_with_shared_experts_sampled_tokens(B):
+@pytest.mark.parametrize("path", [1, 2])
+def test_layer_finegrained_with_shared_experts_sampled_tokens(B, path):
     wl = synth.WORKLOADS["finegrained"]
-    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 256, tokens=[0, 100, 255], kernel_path=1)
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 256, tokens=[0, 100, 255], kernel_path=path)
+    assert max(errs.values()) < TOL, errs
+
+
+def cross_check_paths(B, wl, T, blobs=None):
+    """Tensor-core path against the CUDA-core path on the same device inputs (all tokens)."""
+    x = synth.tokens_bf16(wl, T, "cuda")
+    kw = {"forced_bit_idx": synth.forced_bit_idx(wl, T, "cuda")}
+    if wl.zipf_logits:
+        kw["logits"] = synth.zipf_logits(wl, T, "cuda")
+    else:
+        kw["gate_w"] = synth.gate_weight_bf16(wl, "cuda")
+    cfg_cc = B.Config.from_workload(wl, kernel_path=1)
+    cfg_tc = B.Config.from_workload(wl, kernel_path=2)
+    if blobs is None:
+        blobs = gpu_layer(B, cfg_cc, wl)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_cc = B.moe_forward(cfg_cc, x, blobs, device_status=st, **kw).float()
+    y_tc = B.moe_forward(cfg_tc, x, blobs, device_status=st, **kw).float()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    err = (y_cc - y_tc).abs().amax(dim=1) / y_cc.abs().amax(dim=1)
+    return float(err.max().item()), blobs
+
+
+@pytest.fixture(scope="module")
+def mixtral_blobs(B):
+    wl = synth.WORKLOADS["mixtral_decode"]
+    return gpu_layer(B, B.Config.from_workload(wl), wl)
+
+
+@pytest.mark.parametrize("T", [1, 8, 32, 64])
+def test_mixtral_decode_tensor_path_matches_cuda_core_path(B, mixtral_blobs, T):
+    wl = synth.WORKLOADS["mixtral_decode"]
+    err, _ = cross_check_paths(B, wl, T, mixtral_blobs)
+    assert err < TOL, err
+
+
+def test_mixtral_decode_sampled_tokens_against_oracle(B, mixtral_blobs):
+    """Full-size decode layer in the benchmark's configuration (T = 64, tensor-core path): the oracle
+    recomputes one sampled token end to end (two experts, each regenerated and quantized on the CPU)."""
+    wl = synth.WORKLOADS["mixtral_decode"]
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 64, tokens=[37], kernel_path=0, blobs=mixtral_blobs)
     assert max(errs.values()) < TOL, errs
 
 
