@@ -14,7 +14,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libd2moe.so")
+LIB_PATH = os.environ.get("D2MOE_LIB_PATH") or os.path.join(_HERE, "libd2moe.so")
 
 PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR = 0, 1, 2
 

@@ -262,7 +262,8 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
         B.pad_off = (int32_t*)(w + ws.off_pad_off); B.row_map = (int32_t*)(w + ws.off_row_map);
         B.src_token = (int32_t*)(w + ws.off_src_token);
         B.xp16 = (__half*)(w + ws.off_xp16); B.h16 = (__half*)(w + ws.off_h); B.o32 = (float*)(w + ws.off_o);
-        e = launch_ffn_tensor(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev);
+        e = pl.decode ? launch_ffn_decode(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev)
+                      : launch_ffn_tensor(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev);
         if (e != cudaSuccess) return D2MOE_ERR_CUDA;
         mark(3);
         e = launch_combine(D, R, B.o32, pl.n_split, (size_t)pl.R_alloc * D.d, B.row_map,

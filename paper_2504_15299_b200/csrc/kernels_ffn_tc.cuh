@@ -14,6 +14,8 @@ struct TcUnit {
 };
 
 struct TcPlan {
+    int decode;             // 1: memory-bound decode kernel (tokens sorted widest first, one tile per
+                            //    segment); 0: grouped dequant-GEMM (one tile per width, any load)
     int n_cap;              // columns per unit
     long long R_alloc;      // rows of the padded activation buffers
     int max_units;
@@ -30,5 +32,8 @@ struct TcBuffers {
 bool tc_path_supported(const d2moe_config* c);
 void tc_plan(const d2moe_config* c, long long T, TcPlan* pl);
 cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                              const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
+                              const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
+cudaError_t launch_ffn_decode(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                               const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
                               const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
