@@ -25,10 +25,10 @@
 // 2^-S (S per matrix, from the largest scale seen at pack time) so the multipliers stay in fp16
 // range; the epilogue multiplies by 2^S.
 //
-// CTA = 384 threads, 2 CTAs per SM: warps 0-3 and 4-7 are two dequant warpgroups that take
-// alternate K-groups (each with its own two 32-column operand slots in TMEM), warp 8 streams packed
-// blocks (cp.async.bulk), warp 9 streams activation tiles (TMA, 128B swizzle), warps 10 and 11 issue
-// the MMAs (even / odd segments).  TMEM per CTA: 128 accumulator columns (K segments x n_cap tokens) + 4 x 32 operand columns.
+// CTA = 384 threads, 2 CTAs per SM: warps 0-3 and 4-7 are two dequant warpgroups; warpgroup w takes
+// the segments w, w+2, ... of every K-group and owns two 32-column operand slots in TMEM that
+// alternate; warp 8 streams packed blocks (cp.async.bulk), warp 9 streams activation tiles (TMA,
+// 128B swizzle), warps 10 and 11 issue the MMAs of warpgroup 0 and 1.  TMEM per CTA: 128 accumulator columns (K segments x n_cap tokens) + 4 x 32 operand columns.
 // Every wait is bounded; on expiry the CTA raises D2MOE_DEV_TIMEOUT, stops waiting, drains, exits.
 #include "d2moe_common.cuh"
 #include "kernels_ffn_tc.cuh"
@@ -92,8 +92,16 @@ __device__ __forceinline__ DecItem dec_item(const DecParams& p, int item) {
 // 64 consecutive codes (elements 64h .. 64h+63 of the group) of one segment of one row ->
 // 32 half2 registers tile[i] = code pair * multiplier + addend, written to TMEM columns
 // [taddr, taddr + 32).   m0: multiplier of a code at bit position 0; position p uses m0 * 2^-p.
+template <int SW>
+__device__ __forceinline__ void make_multipliers(__half2 m0, __half2 (&mult)[8]) {
+    mult[0] = m0;
+    const __half2 step = __float2half2_rn(1.0f / (float)(1 << SW));
+#pragma unroll
+    for (int q = 1; q < 8 / SW; ++q) mult[q] = __hmul2(mult[q - 1], step);
+}
+
 template <int GS, int SW>
-__device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, __half2 m0, __half2 addend, uint32_t taddr) {
+__device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, const __half2 (&mult)[8], __half2 addend, uint32_t taddr) {
     constexpr int ROW_BYTES = GS * SW / 8;
     constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;      // chunk size of the packed layout
     constexpr int HALF_BYTES = 8 * SW;                       // bytes of 64 codes
@@ -103,11 +111,6 @@ __device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, _
     constexpr int PER = 16 / SW;                             // registers per word
     constexpr int NPOS = 8 / SW;                             // distinct bit positions per byte lane
     constexpr uint32_t FIELD = ((1u << SW) - 1u) * 0x00010001u;
-    __half2 mult[NPOS];
-    mult[0] = m0;
-    const __half2 step = __float2half2_rn(1.0f / (float)(1 << SW));
-#pragma unroll
-    for (int q = 1; q < NPOS; ++q) mult[q] = __hmul2(mult[q - 1], step);
 
     uint32_t out[32];
 #pragma unroll
@@ -144,15 +147,72 @@ __device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, _
 
 template <int GS>
 __device__ __forceinline__ void dequant_half_dispatch(int sw, uint32_t seg, int rr, int h, __half2 m0, __half2 addend, uint32_t taddr) {
+    __half2 mult[8];
     switch (sw) {
-        case 1: dequant_half_tile<GS, 1>(seg, rr, h, m0, addend, taddr); break;
-        case 2: dequant_half_tile<GS, 2>(seg, rr, h, m0, addend, taddr); break;
-        case 4: dequant_half_tile<GS, 4>(seg, rr, h, m0, addend, taddr); break;
-        default: dequant_half_tile<GS, 8>(seg, rr, h, m0, addend, taddr); break;
+        case 1: make_multipliers<1>(m0, mult); dequant_half_tile<GS, 1>(seg, rr, h, mult, addend, taddr); break;
+        case 2: make_multipliers<2>(m0, mult); dequant_half_tile<GS, 2>(seg, rr, h, mult, addend, taddr); break;
+        case 4: make_multipliers<4>(m0, mult); dequant_half_tile<GS, 4>(seg, rr, h, mult, addend, taddr); break;
+        default: make_multipliers<8>(m0, mult); dequant_half_tile<GS, 8>(seg, rr, h, mult, addend, taddr); break;
     }
 }
 
-template <int GS>
+// Compile-time description of a width list whose segments are stored exactly (widths 1, 2, 4, 8):
+// nibble j of SWPACK is the width of segment j.  SWPACK == 0 selects the run-time path.
+template <int SWPACK>
+struct SegList {
+    __host__ __device__ static constexpr int sw(int j) { return (SWPACK >> (4 * j)) & 15; }
+    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && sw(k) != 0) ++k; return k; }
+    __host__ __device__ static constexpr int bits_upto(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += sw(i); return b; }
+    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
+};
+
+// One K-group of warpgroup WG with a compile-time width list: its segments j = WG, WG+2 (at most two
+// when the list has at most four), both halves, straight-line code.  fac[q], cfac[q]: per-item factors
+// so that multiplier(position 0) = s1 * fac and the tile constant = s1 * cfac (segment 0: lo * 2^-S).
+template <int GS, int SWPACK, int WG, typename WaitEmpty, typename Publish>
+__device__ __forceinline__ void dequant_group_fixed(uint32_t wb, int rr, int kmax, float s1, float lo_scaled,
+                                                    const float (&fac)[2], const float (&cfac)[2], uint32_t a_slots,
+                                                    WaitEmpty&& wait_empty, Publish&& publish) {
+    using SL = SegList<SWPACK>;
+    constexpr int HALVES = GS / 64;
+    __half2 mult[2][8];
+    __half2 addend[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        constexpr int dummy = 0; (void)dummy;
+        const int j = WG + 2 * q;
+        if (j < SL::count()) {
+            const __half2 m0 = __float2half2_rn(s1 * fac[q]);
+            if (SL::sw(j < 8 ? j : 0) == 1) make_multipliers<1>(m0, mult[q]);
+            else if (SL::sw(j < 8 ? j : 0) == 2) make_multipliers<2>(m0, mult[q]);
+            else if (SL::sw(j < 8 ? j : 0) == 4) make_multipliers<4>(m0, mult[q]);
+            else make_multipliers<8>(m0, mult[q]);
+            addend[q] = __float2half2_rn(j == 0 ? lo_scaled : s1 * cfac[q]);
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < HALVES; ++h) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            constexpr int K = SL::count();
+            const int j = WG + 2 * q;
+            if (j < K) {
+                if (j <= kmax) {
+                    wait_empty(q);
+                    const uint32_t seg = wb + (uint32_t)SL::seg_off(GS, j < 8 ? j : 0);
+                    const uint32_t taddr = a_slots + q * 32;
+                    if (SL::sw(j < 8 ? j : 0) == 1) dequant_half_tile<GS, 1>(seg, rr, h, mult[q], addend[q], taddr);
+                    else if (SL::sw(j < 8 ? j : 0) == 2) dequant_half_tile<GS, 2>(seg, rr, h, mult[q], addend[q], taddr);
+                    else if (SL::sw(j < 8 ? j : 0) == 4) dequant_half_tile<GS, 4>(seg, rr, h, mult[q], addend[q], taddr);
+                    else dequant_half_tile<GS, 8>(seg, rr, h, mult[q], addend[q], taddr);
+                    publish(q);
+                }
+            }
+        }
+    }
+}
+
+template <int GS, int SWPACK>
 __global__ void __launch_bounds__(DEC_THREADS, 2)
 ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaMaps maps) {
     constexpr int HALVES = GS / 64;
@@ -181,7 +241,7 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < DEC_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 128); }
+        for (int i = 0; i < DEC_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 256); }
         for (int i = 0; i < DEC_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 2); }
         for (int wg = 0; wg < 2; ++wg)
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
@@ -262,68 +322,86 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
             STAT_FLUSH(true);
         }
     } else if (warp >= DEC_WARP_MMA) {
-        // Two MMA issuers: issuer m takes the segments j with j % 2 == m (disjoint accumulators D_j), from
-        // operand slot m of either warpgroup.  One thread issues at most one tcgen05.mma per ~45 cycles
-        // whatever its size, so the issue work is split and kept to a few instructions per MMA.
-        if (lane == 0) {
+        // Two MMA issuers, one per dequant warpgroup: issuer w multiplies the tiles warpgroup w writes
+        // (segments w, w+2, ...: accumulators disjoint from the other issuer's) from that warpgroup's two
+        // operand slots, which alternate, so a slot is refilled while the other one is being multiplied.
+        // One thread issues at most one tcgen05.mma per ~45 cycles whatever its size, so the issue work
+        // is split over two warps.  The whole warp runs the loop and one elected lane issues, so that
+        // addresses and descriptors stay in the uniform datapath (fewer instructions per MMA, which
+        // matters because the issuer competes with the dequant warps for issue slots).
+        {
             STAT_DECL();
 #ifdef D2MOE_WAIT_STATS
             const long long _tt = clock64();
 #endif
-            const int m = warp - DEC_WARP_MMA;
+            const int w = warp - DEC_WARP_MMA;
             uint32_t it = 0, ic = 0;
-            uint32_t use0 = 0, use1 = 0;                     // uses of slot m of warpgroup 0 / 1
+            uint32_t use0 = 0, use1 = 0;                     // uses of slot 0 / 1 of warpgroup w
             const uint32_t n_cap_bytes = (uint32_t)p.n_cap * 128u;
+            const uint32_t a_slot0 = a_tmem + (w * 2) * 32, a_slot1 = a_slot0 + 32;
             for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
                 const DecItem ii = dec_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
                 const int kmax = u->kmax;
-                const int n_mine = kmax >= m ? (kmax - m) / 2 + 1 : 0;       // segments m, m+2, ...
+                const int n_mine = kmax >= w ? (kmax - w) / 2 + 1 : 0;       // segments w, w+2, ...
                 uint32_t idesc[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) idesc[q] = instr_desc_f16(u->cnt[(2 * q + m) & 7]);
+                for (int q = 0; q < 4; ++q) idesc[q] = instr_desc_f16(u->cnt[(2 * q + w) & 7]);
                 { STAT_T0(); mbar_wait(D_EMPTY, (ic & 1) ^ 1, abort_flag, p.status); STAT_ADD(2); }
                 tc_fence_after();
                 for (int G = ii.g0; G < ii.g1; ++G, ++it) {
                     const int s = it % DEC_NSB;
-                    const int wg = it & 1;
                     { STAT_T0(); mbar_wait(B_FULL(s), (it / DEC_NSB) & 1, abort_flag, p.status); STAT_ADD(3); }
                     const uint64_t bdesc = smem_desc_sw128(bbuf + s * b_slot_bytes);
-                    const uint32_t a_addr = a_tmem + (wg * 2 + m) * 32;
-                    const uint32_t full_bar = A_FULL(wg, m), empty_bar = A_EMPTY(wg, m);
-                    uint32_t use = wg ? use1 : use0;
                     const uint32_t first = (G != ii.g0) ? 1u : 0u;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (q < n_mine) {
-                            const uint32_t d_addr = d_tmem + (2 * q + m) * p.n_cap;
+                    for (int qp = 0; qp < 2; ++qp) {                  // pairs of my segments: slots 0 and 1
 #pragma unroll
-                            for (int h = 0; h < HALVES; ++h) {
-                                { STAT_T0(); mbar_wait(full_bar, use & 1, abort_flag, p.status); STAT_ADD(4); }
-                                tc_fence_after();
-                                const uint64_t bh = bdesc + (uint64_t)((h * n_cap_bytes) >> 4);
-                                tc_mma_ts(d_addr, a_addr + 0, bh + 0, idesc[q], h == 0 ? first : 1u);
-                                tc_mma_ts(d_addr, a_addr + 8, bh + 2, idesc[q], 1u);
-                                tc_mma_ts(d_addr, a_addr + 16, bh + 4, idesc[q], 1u);
-                                tc_mma_ts(d_addr, a_addr + 24, bh + 6, idesc[q], 1u);
-                                tc_commit(empty_bar);
-                                ++use;
+                        for (int h = 0; h < HALVES; ++h) {
+#pragma unroll
+                            for (int sl = 0; sl < 2; ++sl) {
+                                const int q = 2 * qp + sl;
+                                if (q < n_mine) {
+                                    const uint32_t d_addr = d_tmem + (2 * q + w) * p.n_cap;
+                                    const uint32_t a_addr = sl ? a_slot1 : a_slot0;
+                                    const uint32_t use = sl ? use1 : use0;
+                                    { STAT_T0(); mbar_wait(A_FULL(w, sl), use & 1, abort_flag, p.status); STAT_ADD(4); }
+                                    tc_fence_after();
+                                    const uint64_t bh = bdesc + (uint64_t)((h * n_cap_bytes) >> 4);
+                                    {
+                                        STAT_T0();
+                                        if (elect_one()) {
+                                            tc_mma_ts(d_addr, a_addr + 0, bh + 0, idesc[q], h == 0 ? first : 1u);
+                                            tc_mma_ts(d_addr, a_addr + 8, bh + 2, idesc[q], 1u);
+                                            tc_mma_ts(d_addr, a_addr + 16, bh + 4, idesc[q], 1u);
+                                            tc_mma_ts(d_addr, a_addr + 24, bh + 6, idesc[q], 1u);
+                                            tc_commit(A_EMPTY(w, sl));
+                                        }
+                                        __syncwarp();
+                                        STAT_ADD(12);
+#ifdef D2MOE_WAIT_STATS
+                                        stat[13] += 1;
+#endif
+                                    }
+                                    if (sl) ++use1; else ++use0;
+                                }
                             }
                         }
                     }
-                    if (wg) use1 = use; else use0 = use;
-                    tc_commit(B_EMPTY(s));
+                    if (elect_one()) tc_commit(B_EMPTY(s));
+                    __syncwarp();
                 }
-                tc_commit(D_FULL);
+                if (elect_one()) tc_commit(D_FULL);
+                __syncwarp();
             }
             if (ic > 0) mbar_wait(D_FULL, (ic - 1) & 1, abort_flag, p.status, true);
 #ifdef D2MOE_WAIT_STATS
             stat[5] = clock64() - _tt;
 #endif
-            STAT_FLUSH(m == 0);
+            STAT_FLUSH(w == 0 && lane == 0);
         }
     } else {
-        // ---------------- two dequant warpgroups (alternate K-groups) + epilogue ----------------
+        // -------- two dequant warpgroups (warpgroup w: segments w, w+2, ... of every K-group) + epilogue --------
         const int wg = warp >> 2;
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
         const int blk = r >> 6, rr = r & 63;
@@ -342,8 +420,24 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
             const int S = matrix_exponent(mat);
             const float two_mS = exp2f((float)-S);
 
+            // per-item factors of my segments (compile-time width list only)
+            float fac[2] = {0.0f, 0.0f}, cfac[2] = {0.0f, 0.0f};
+            if constexpr (SWPACK != 0) {
+                using SL = SegList<SWPACK>;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int j = wg + 2 * q;
+                    if (j < SL::count()) {
+                        const int delta = (wg == 0 ? SL::bits_upto(2 * q < 8 ? 2 * q : 0) : SL::bits_upto(2 * q + 1 < 8 ? 2 * q + 1 : 0)) - SL::sw(0);
+                        const int wj = wg == 0 ? SL::sw(2 * q < 8 ? 2 * q : 0) : SL::sw(2 * q + 1 < 8 ? 2 * q + 1 : 0);
+                        const float Mfac = exp2f((float)(-delta - S));                 // M_j 2^-S = s1 * Mfac
+                        fac[q] = Mfac * 16777216.0f;
+                        cfac[q] = -0.5f * (float)((1 << wj) - 1) * Mfac;
+                    }
+                }
+            }
+
             for (int G = ii.g0; G < ii.g1; ++G, ++it) {
-                if ((int)(it & 1) != wg) continue;
                 const int s = it % nsw;
                 { STAT_T0(); mbar_wait(W_FULL(s), (it / nsw) & 1, abort_flag, p.status); STAT_ADD(6); }
                 const uint32_t wb = wbuf + s * w_slot_bytes + blk * p.L.block_bytes;
@@ -351,36 +445,61 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
                 const __half2 mh = as_h2(meta);
                 const float s1 = __low2float(mh) * two_mS, lo = __high2float(mh) * two_mS;
-                // segments in pairs (2jp, 2jp+1): segment j fills operand slot j % 2, read by issuer j % 2
+                if constexpr (SWPACK != 0) {
+                    auto wait_empty = [&](int sl) {
+                        const uint32_t use = sl ? use1 : use0;
+                        STAT_T0(); mbar_wait(A_EMPTY(wg, sl), (use & 1) ^ 1, abort_flag, p.status); STAT_ADD(7);
+                        tc_fence_after();
+                    };
+                    auto publish = [&](int sl) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(A_FULL(wg, sl));
+                        if (sl) ++use1; else ++use0;
+                    };
+                    const float s1raw = __low2float(mh);
+                    if (wg == 0) dequant_group_fixed<GS, SWPACK, 0>(wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + lane_addr, wait_empty, publish);
+                    else dequant_group_fixed<GS, SWPACK, 1>(wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + 64 + lane_addr, wait_empty, publish);
+                } else {
+                // my segments j = wg + 2q, in pairs: q = 2qp + sl fills operand slot sl
+                    const int n_mine = kmax >= wg ? (kmax - wg) / 2 + 1 : 0;
 #pragma unroll 1
-                for (int jp = 0; 2 * jp <= kmax; ++jp) {
-                    __half2 m0[2], addend[2];
-                    uint32_t seg[2];
-                    int sw[2];
+                    for (int qp = 0; 2 * qp < n_mine; ++qp) {
+                        __half2 m0[2], addend[2];
+                        uint32_t seg[2];
+                        int sw[2];
 #pragma unroll
-                    for (int m = 0; m < 2; ++m) {
-                        const int j = min(2 * jp + m, kmax);
-                        sw[m] = p.L.seg_sw[j];
-                        // M_j 2^-S, the position-0 multiplier M_j 2^(24-S), and the tile's constant
-                        const float Mj = s1 * exp2f((float)(-(p.D.bits[j] - p.D.bits[0])));
-                        m0[m] = h2dup(Mj * 16777216.0f);
-                        addend[m] = h2dup(j == 0 ? lo : -0.5f * (float)((1 << p.L.seg_w[j]) - 1) * Mj);
-                        seg[m] = wb + (uint32_t)p.L.seg_off[j];
-                    }
+                        for (int sl = 0; sl < 2; ++sl) {
+                            const int j = min(wg + 2 * (2 * qp + sl), kmax);
+                            sw[sl] = p.L.seg_sw[j];
+                            // M_j 2^-S, the position-0 multiplier M_j 2^(24-S), and the tile's constant
+                            const float Mj = s1 * exp2f((float)(-(p.D.bits[j] - p.D.bits[0])));
+                            m0[sl] = h2dup(Mj * 16777216.0f);
+                            addend[sl] = h2dup(j == 0 ? lo : -0.5f * (float)((1 << p.L.seg_w[j]) - 1) * Mj);
+                            seg[sl] = wb + (uint32_t)p.L.seg_off[j];
+                        }
 #pragma unroll
-                    for (int h = 0; h < HALVES; ++h) {
+                        for (int h = 0; h < HALVES; ++h) {
 #pragma unroll
-                        for (int m = 0; m < 2; ++m) {
-                            if (2 * jp + m <= kmax) {
-                                const uint32_t use = m ? use1 : use0;
-                                { STAT_T0(); mbar_wait(A_EMPTY(wg, m), (use & 1) ^ 1, abort_flag, p.status); STAT_ADD(7); }
-                                tc_fence_after();
-                                dequant_half_dispatch<GS>(sw[m], seg[m], rr, h, m0[m], addend[m],
-                                                          a_tmem + (wg * 2 + m) * 32 + lane_addr);
-                                { STAT_T0(); tc_wait_st(); STAT_ADD(8); }
-                                tc_fence_before();
-                                mbar_arrive(A_FULL(wg, m));
-                                if (m) ++use1; else ++use0;
+                            for (int sl = 0; sl < 2; ++sl) {
+                                if (2 * qp + sl < n_mine) {
+                                    const uint32_t use = sl ? use1 : use0;
+                                    { STAT_T0(); mbar_wait(A_EMPTY(wg, sl), (use & 1) ^ 1, abort_flag, p.status); STAT_ADD(7); }
+                                    tc_fence_after();
+                                    {
+                                        STAT_T0();
+                                        dequant_half_dispatch<GS>(sw[sl], seg[sl], rr, h, m0[sl], addend[sl],
+                                                                  a_tmem + (wg * 2 + sl) * 32 + lane_addr);
+                                        STAT_ADD(14);
+#ifdef D2MOE_WAIT_STATS
+                                        stat[15] += 1;
+#endif
+                                    }
+                                    { STAT_T0(); tc_wait_st(); STAT_ADD(8); }
+                                    tc_fence_before();
+                                    mbar_arrive(A_FULL(wg, sl));
+                                    if (sl) ++use1; else ++use0;
+                                }
                             }
                         }
                     }
@@ -599,16 +718,27 @@ cudaError_t launch_ffn_decode(const d2moe_config* c, const MoeDims& D, const Pac
         p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         mark(mode == 0 ? 1 : 2);
-        cudaError_t e;
-        if (D.g == 128) {
-            e = cudaFuncSetAttribute(ffn_dec_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            if (e != cudaSuccess) return e;
-            ffn_dec_kernel<128><<<2 * sms, DEC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
-        } else {
-            e = cudaFuncSetAttribute(ffn_dec_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            if (e != cudaSuccess) return e;
-            ffn_dec_kernel<64><<<2 * sms, DEC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+        // width lists whose segments are stored exactly get a kernel specialised on the list
+        int swpack = 0;
+        bool exact = p.L.n_seg <= 4;
+        for (int j = 0; j < p.L.n_seg && exact; ++j) {
+            exact = p.L.seg_w[j] == p.L.seg_sw[j];
+            swpack |= p.L.seg_sw[j] << (4 * j);
         }
+        if (!exact) swpack = 0;
+        auto launch = [&](auto kern) -> cudaError_t {
+            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (err != cudaSuccess) return err;
+            kern<<<2 * sms, DEC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            return cudaSuccess;
+        };
+        cudaError_t e;
+        if (D.g == 128 && swpack == 0x4112) e = launch(ffn_dec_kernel<128, 0x4112>);
+        else if (D.g == 128 && swpack == 0x422) e = launch(ffn_dec_kernel<128, 0x422>);
+        else if (D.g == 64 && swpack == 0x422) e = launch(ffn_dec_kernel<64, 0x422>);
+        else if (D.g == 128) e = launch(ffn_dec_kernel<128, 0>);
+        else e = launch(ffn_dec_kernel<64, 0>);
+        if (e != cudaSuccess) return e;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

@@ -27,6 +27,21 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// try_wait with a suspend-time hint: the warp sleeps in hardware (issuing nothing) until the phase
+// completes or about `ns` nanoseconds pass, instead of spinning through the issue slots and the
+// integer pipe that the working warps need.
+__device__ __forceinline__ bool mbar_try_sleep(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -40,8 +55,8 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return;
     unsigned long long t0 = 0;
     for (unsigned spin = 0;; ++spin) {
-        if (mbar_try(bar, parity)) return;
-        if ((spin & 255u) == 255u) {
+        if (mbar_try_sleep(bar, parity, 4000u)) return;
+        if ((spin & 15u) == 15u) {
             if (*abort_flag && !drain) return;      // a drain wait keeps its own one-second limit
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
