@@ -112,37 +112,32 @@ __device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, c
     constexpr int NPOS = 8 / SW;                             // distinct bit positions per byte lane
     constexpr uint32_t FIELD = ((1u << SW) - 1u) * 0x00010001u;
 
-    uint32_t out[32];
+    uint32_t w[NLD * WPL];
 #pragma unroll
     for (int l = 0; l < NLD; ++l) {
         const int off = h * HALF_BYTES + l * LD;             // byte offset inside the row's bytes
         const int c = off / CS, within = off % CS;           // (h is a loop constant after unrolling)
         const uint32_t addr = seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS + within);
-        uint32_t w[WPL];
         if constexpr (WPL == 4) {
-            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[l * 4 + 0]), "=r"(w[l * 4 + 1]), "=r"(w[l * 4 + 2]), "=r"(w[l * 4 + 3]) : "r"(addr));
         } else if constexpr (WPL == 2) {
-            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr));
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[l * 2 + 0]), "=r"(w[l * 2 + 1]) : "r"(addr));
         } else {
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[0]) : "r"(addr));
-        }
-#pragma unroll
-        for (int q = 0; q < WPL; ++q) {
-            const uint32_t lo8 = w[q];
-            const uint32_t hi8 = __umulhi(w[q], 1u << 24);   // w >> 8 on the multiply pipe
-#pragma unroll
-            for (int e = 0; e < PER; ++e) {
-                const uint32_t src = e < NPOS ? lo8 : hi8;
-                const __half2 code = as_h2(src & (FIELD << ((e % NPOS) * SW)));
-                out[(l * WPL + q) * PER + e] = as_u32(__hfma2(code, mult[e % NPOS], addend));
-            }
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[l]) : "r"(addr));
         }
     }
-    uint32_t v0[16], v1[16];
+    // two batches of 16 registers, each stored to TMEM as soon as it is complete
 #pragma unroll
-    for (int j = 0; j < 16; ++j) { v0[j] = out[j]; v1[j] = out[16 + j]; }
-    tc_st16(taddr, v0);
-    tc_st16(taddr + 16, v1);
+    for (int b = 0; b < 2; ++b) {
+        uint32_t v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int idx = b * 16 + i, q = idx / PER, e = idx % PER;
+            const uint32_t src = e < NPOS ? w[q] : (w[q] >> 8);
+            v[i] = as_u32(__hfma2(as_h2(src & (FIELD << ((e % NPOS) * SW))), mult[e % NPOS], addend));
+        }
+        tc_st16(taddr + b * 16, v);
+    }
 }
 
 template <int GS>
