@@ -129,6 +129,33 @@ d2moe_status d2moe_route(const d2moe_config* cfg, int64_t T,
                          int32_t* device_status, void* workspace, size_t workspace_bytes,
                          void* stream);
 
+/*
+ * d2moe_route without a workspace argument (the paper has no counterpart: this is an integration
+ * aid).  Some callers may not allocate device memory at the point where they route a batch: a
+ * serving loop whose memory pool is frozen after start-up, a plug-in that runs inside another
+ * framework's step and must not touch its allocator, a component working under a fixed memory
+ * budget.  For them the scratch that routing needs (sort keys and the (expert, width) histogram) is
+ * a fixed array inside the library: (D2MOE_STATIC_MAX_ASSIGNMENTS + D2MOE_STATIC_MAX_KEYS) * 4
+ * bytes = 72 KiB of device memory that every GPU loading the library holds until the process exits.  The call itself allocates nothing (no
+ * cudaMalloc, no cudaFree, no allocating library routine).
+ *   - Limits: T * top_k <= D2MOE_STATIC_MAX_ASSIGNMENTS and n_experts * n_bits <=
+ *     D2MOE_STATIC_MAX_KEYS; anything larger is refused with D2MOE_ERR_WORKSPACE before any launch.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Calls that may overlap on the GPU (different
+ *     streams, or graphs replayed concurrently) race on it and give wrong routing; serialise them.
+ *     Nothing needs clearing between calls: every scratch word is written before it is read.
+ * Inputs, outputs, rounding and error reporting are those of d2moe_route.
+ */
+#define D2MOE_STATIC_MAX_ASSIGNMENTS 16384
+#define D2MOE_STATIC_MAX_KEYS 2048
+d2moe_status d2moe_route_static_scratch(const d2moe_config* cfg, int64_t T,
+                                        const void* x_bf16, const void* gate_w_bf16, const float* logits,
+                                        const void* bit_w_bf16, const int8_t* forced_bit_idx,
+                                        int32_t* topk_idx, float* topk_w, int8_t* bit_idx,
+                                        int32_t* perm, int32_t* inv_perm, int32_t* group_off,
+                                        int32_t* device_status, void* stream);
+
 typedef struct {
     const void* gate_w_bf16;        /* device bf16 [E, d_model] or NULL */
     const float* logits;            /* device fp32 [T, E] or NULL       */

@@ -49,7 +49,8 @@ _lib = None
 
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
-           "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count"]
+           "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count",
+           "d2moe_route_static_scratch"]
 
 
 def lib() -> ctypes.CDLL:
@@ -71,6 +72,7 @@ def lib() -> ctypes.CDLL:
     L.d2moe_workspace_bytes.restype = sz
     L.d2moe_workspace_bytes.argtypes = [cfgp, i64]
     L.d2moe_route.argtypes = [cfgp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.d2moe_route_static_scratch.argtypes = [cfgp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.d2moe_moe_forward.argtypes = [cfgp, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(_RouteIn),
                                     ctypes.POINTER(_RouteOut), vp, vp, vp, sz, vp]
     L.d2moe_moe_forward_events.argtypes = [cfgp, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(_RouteIn),
@@ -208,6 +210,33 @@ def route(cfg: Config, x: torch.Tensor, *, gate_w=None, logits=None, bit_w=None,
                              _ptr(forced_bit_idx), _ptr(r.topk_idx), _ptr(r.topk_w), _ptr(r.bit_idx),
                              _ptr(r.perm), _ptr(r.inv_perm), _ptr(r.group_off), _ptr(r.device_status),
                              _ptr(workspace), workspace.numel(), _stream(stream)), "d2moe_route")
+    return r
+
+
+STATIC_MAX_ASSIGNMENTS, STATIC_MAX_KEYS = 16384, 2048
+
+
+def route_static_scratch(cfg: Config, x: torch.Tensor, *, gate_w=None, logits=None, bit_w=None,
+                         forced_bit_idx=None, out: Optional[RouteResult] = None, stream=None) -> RouteResult:
+    """d2moe_route for callers that cannot provide a workspace: the library's built-in scratch array is
+    used instead (see the limits in include/d2moe.h).  Pass ``out`` (a RouteResult whose tensors were
+    allocated earlier) to make the call itself allocation-free on the Python side too."""
+    T = x.shape[0]
+    dev = x.device
+    A = T * cfg.top_k
+    r = out
+    if r is None:
+        r = RouteResult(torch.empty((T, cfg.top_k), dtype=torch.int32, device=dev),
+                        torch.empty((T, cfg.top_k), dtype=torch.float32, device=dev),
+                        torch.empty((T, cfg.top_k), dtype=torch.int8, device=dev),
+                        torch.empty(A, dtype=torch.int32, device=dev),
+                        torch.empty(A, dtype=torch.int32, device=dev),
+                        torch.empty(cfg.n_experts * len(cfg.bits) + 1, dtype=torch.int32, device=dev),
+                        torch.zeros(1, dtype=torch.int32, device=dev))
+    _check(lib().d2moe_route_static_scratch(ctypes.byref(cfg.c()), T, _ptr(x), _ptr(gate_w), _ptr(logits),
+                                            _ptr(bit_w), _ptr(forced_bit_idx), _ptr(r.topk_idx), _ptr(r.topk_w),
+                                            _ptr(r.bit_idx), _ptr(r.perm), _ptr(r.inv_perm), _ptr(r.group_off),
+                                            _ptr(r.device_status), _stream(stream)), "d2moe_route_static_scratch")
     return r
 
 

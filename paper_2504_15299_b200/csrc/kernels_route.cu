@@ -195,3 +195,77 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     scatter_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
     return cudaGetLastError();
 }
+
+// ------------------------------------------------------------------------------------------------
+// d2moe_route_static_scratch: the routing call for callers that cannot hand over a workspace.
+//
+// Its scratch (the per-assignment sort keys and the (expert, width) histogram that d2moe_route keeps
+// in the caller's workspace) lives in one file-scope device array, so the call needs no allocation
+// of any kind.  The array is part of the library image: every GPU that loads the library holds these
+// bytes until the process exits.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+#define D2MOE_STATIC_SCRATCH_BYTES ((D2MOE_STATIC_MAX_ASSIGNMENTS + D2MOE_STATIC_MAX_KEYS) * 4)
+
+static __device__ __align__(256) unsigned char g_route_scratch[D2MOE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};   // device address of g_route_scratch, per device ordinal
+}  // namespace
+
+extern "C" d2moe_status d2moe_route_static_scratch(const d2moe_config* c, int64_t T, const void* x,
+                                                   const void* gate_w, const float* logits, const void* bit_w,
+                                                   const int8_t* forced, int32_t* topk_idx, float* topk_w,
+                                                   int8_t* bit_idx, int32_t* perm, int32_t* inv_perm,
+                                                   int32_t* group_off, int32_t* device_status, void* stream) {
+    d2moe_status s = d2moe_check_config(c);
+    if (s != D2MOE_OK) return s;
+    if (T < 0) return D2MOE_ERR_SHAPE;
+    // the fixed scratch bounds the problem: say so instead of overrunning it
+    if (T * c->top_k > D2MOE_STATIC_MAX_ASSIGNMENTS || c->n_experts * c->n_bits > D2MOE_STATIC_MAX_KEYS)
+        return D2MOE_ERR_WORKSPACE;
+    if (!topk_idx || !topk_w || !bit_idx || !perm || !inv_perm || !group_off) return D2MOE_ERR_NULL;
+    if (T > 0 && !x) return D2MOE_ERR_NULL;
+    if ((gate_w == nullptr) == (logits == nullptr)) return D2MOE_ERR_NULL;
+    if ((bit_w == nullptr) == (forced == nullptr)) return D2MOE_ERR_NULL;
+
+    // In host code `g_route_scratch` is only a handle for the symbol, not an address a kernel can
+    // use.  The device address is looked up once per device, with that device current, and kept.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return D2MOE_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {
+            void* addr = nullptr;
+            if (cudaGetSymbolAddress(&addr, g_route_scratch) != cudaSuccess || !addr) return D2MOE_ERR_CUDA;
+            g_scratch_addr[dev] = addr;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n_keys = c->n_experts * c->n_bits;
+    if (T == 0) {
+        cudaError_t e = cudaMemsetAsync(group_off, 0, (size_t)(n_keys + 1) * 4, st);
+        return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+    }
+    MoeDims D;
+    D.T = (int)T; D.d = c->d_model; D.F = c->d_ffn; D.E = c->n_experts; D.k = c->top_k;
+    D.n_shared = c->n_shared; D.g = c->group_size; D.K = c->n_bits;
+    for (int i = 0; i < 8; ++i) D.bits[i] = i < c->n_bits ? c->bits[i] : 0;
+    D.A = (int)(T * c->top_k);
+    D.A_tot = D.A + (int)(T * c->n_shared);
+    D.renormalize = c->renormalize;
+    // Nothing in the scratch has to start at zero: the key of every assignment and the count of every
+    // (expert, width) pair are written before they are read, so the previous call's contents are inert.
+    int32_t* keys = reinterpret_cast<int32_t*>(scratch);
+    int32_t* hist = keys + D2MOE_STATIC_MAX_ASSIGNMENTS;
+    RouteBufs R{topk_idx, topk_w, bit_idx, perm, inv_perm, group_off};
+    cudaError_t e = launch_route(D, (const __nv_bfloat16*)x, (const __nv_bfloat16*)gate_w, logits,
+                                 (const __nv_bfloat16*)bit_w, forced, R, nullptr, keys, hist, device_status, st);
+    return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+}
