@@ -180,6 +180,152 @@ __global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ ke
     }
 }
 
+// Same dot product with both vectors already in shared memory.
+__device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const __nv_bfloat16* b, int d, int lane) {
+    float acc = 0.0f;
+#pragma unroll 8
+    for (int i = lane; i < d; i += 32)
+        acc = fmaf(__bfloat162float(a[i]), __bfloat162float(b[i]), acc);
+    for (int off = 16; off; off >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, off);
+    return acc;
+}
+
+__device__ __forceinline__ void stage_row(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int d) {
+    const uint4* s = reinterpret_cast<const uint4*>(src);
+    uint4* t = reinterpret_cast<uint4*>(dst);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
+}
+
+// One block (8 warps) per token: the same results as route_kernel, with the token row and batches of
+// EB weight rows staged in shared memory by 16-byte loads (the pinned summation order makes a lane
+// walk a row with stride 32, which is slow straight from global memory); warp w takes row w of a batch.
+__global__ void __launch_bounds__(256)
+route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gate_w,
+                   const float* __restrict__ logits_in, const __nv_bfloat16* __restrict__ bit_w,
+                   const int8_t* __restrict__ forced, RouteBufs R, int32_t* __restrict__ keys,
+                   int32_t* __restrict__ device_status, int EB) {
+    extern __shared__ __align__(16) uint8_t rsm[];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(rsm);
+    __nv_bfloat16* ws = xs + D.d;
+    float* lg_s = reinterpret_cast<float*>(ws + (size_t)EB * D.d);     // [E]
+    float* u_s = lg_s + D.E;                                             // [k * K]
+    int* sel_s = reinterpret_cast<int*>(u_s + MAX_TOPK * 8);             // [k]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x;
+    const int E = D.E;
+
+    if (!(logits_in && forced)) stage_row(xs, x + (size_t)t * D.d, D.d);
+    if (logits_in) {
+        for (int e = threadIdx.x; e < E; e += blockDim.x) lg_s[e] = logits_in[(size_t)t * E + e];
+        __syncthreads();
+    } else {
+        for (int eb = 0; eb < E; eb += EB) {
+            const int n = min(EB, E - eb);
+            for (int r = 0; r < n; ++r) stage_row(ws + (size_t)r * D.d, gate_w + (size_t)(eb + r) * D.d, D.d);
+            __syncthreads();
+            for (int r = warp; r < n; r += 8) {
+                const float v = dot_pinned_smem(xs, ws + (size_t)r * D.d, D.d, lane);
+                if (lane == 0) lg_s[eb + r] = v;
+            }
+            __syncthreads();
+        }
+    }
+
+    float w[MAX_TOPK];
+    float wsum = 0.0f;
+    int sel[MAX_TOPK];
+    if (warp == 0) {
+        float lg[MAX_E_PER_LANE];
+        bool bad = false;
+#pragma unroll
+        for (int m = 0; m < MAX_E_PER_LANE; ++m) {
+            const int e = lane + 32 * m;
+            lg[m] = e < E ? lg_s[e] : -INFINITY;
+            if (e < E && !isfinite(lg[m])) bad = true;
+        }
+        if (__any_sync(0xffffffffu, bad) && lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_NONFINITE);
+        unsigned taken = 0;
+        float selv[MAX_TOPK];
+#pragma unroll
+        for (int s = 0; s < MAX_TOPK; ++s) {
+            sel[s] = 0; selv[s] = 0.0f;
+            if (s < D.k) {
+                float bv = -INFINITY; int bi = 0x7fffffff;
+#pragma unroll
+                for (int m = 0; m < MAX_E_PER_LANE; ++m) {
+                    const int e = lane + 32 * m;
+                    if (e < E && !((taken >> m) & 1u)) {
+                        if (bi == 0x7fffffff || lg[m] > bv) { bv = lg[m]; bi = e; }
+                    }
+                }
+                for (int off = 16; off; off >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                    const bool take = (oi != 0x7fffffff) && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
+                    if (take) { bv = ov; bi = oi; }
+                }
+                sel[s] = bi; selv[s] = bv;
+                if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+                if (lane == 0) sel_s[s] = bi;
+            }
+        }
+        const float mx = selv[0];
+        float part = 0.0f;
+#pragma unroll
+        for (int m = 0; m < MAX_E_PER_LANE; ++m)
+            if (lane + 32 * m < E) part += expf(lg[m] - mx);
+        for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+#pragma unroll
+        for (int s = 0; s < MAX_TOPK; ++s) {
+            w[s] = 0.0f;
+            if (s < D.k) { w[s] = expf(selv[s] - mx) / part; wsum += w[s]; }
+        }
+    }
+    __syncthreads();
+
+    if (!forced) {              // bit-width router logits of the selected experts: rows (slot s, width c)
+        const int n_rows = D.k * D.K;
+        for (int rb = 0; rb < n_rows; rb += EB) {
+            const int n = min(EB, n_rows - rb);
+            for (int r = 0; r < n; ++r) {
+                const int s = (rb + r) / D.K, c = (rb + r) - s * D.K;
+                stage_row(ws + (size_t)r * D.d, bit_w + ((size_t)sel_s[s] * D.K + c) * D.d, D.d);
+            }
+            __syncthreads();
+            for (int r = warp; r < n; r += 8) {
+                const float v = dot_pinned_smem(xs, ws + (size_t)r * D.d, D.d, lane);
+                if (lane == 0) u_s[rb + r] = v;
+            }
+            __syncthreads();
+        }
+    }
+
+    if (warp == 0 && lane == 0) {
+#pragma unroll
+        for (int s = 0; s < MAX_TOPK; ++s) {
+            if (s < D.k) {
+                const int a = t * D.k + s;
+                int kk = 0;
+                if (forced) {
+                    kk = forced[a];
+                    if (kk < 0 || kk >= D.K) {
+                        if (device_status) atomicOr(device_status, D2MOE_DEV_BAD_INDEX);
+                        kk = kk < 0 ? 0 : D.K - 1;
+                    }
+                } else {
+                    float best = u_s[s * D.K];
+                    for (int c = 1; c < D.K; ++c)
+                        if (u_s[s * D.K + c] > best) { best = u_s[s * D.K + c]; kk = c; }
+                }
+                R.topk_idx[a] = sel[s];
+                R.topk_w[a] = D.renormalize ? w[s] / wsum : w[s];
+                R.bit_idx[a] = (int8_t)kk;
+                keys[a] = sel[s] * D.K + kk;
+            }
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
@@ -188,6 +334,18 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
                          int32_t* device_status, cudaStream_t st) {
     const int warps_per_block = 4;
     const int n_keys = D.E * D.K;
+    // block-per-token kernel when the token row plus at least one weight row fit in shared memory
+    const size_t row_bytes = (size_t)D.d * 2;
+    const size_t tail_bytes = (size_t)(D.E + MAX_TOPK * 8 + MAX_TOPK) * 4 + 64;
+    const size_t budget = 200 * 1024;
+    int EB = row_bytes + tail_bytes < budget ? (int)((budget - row_bytes - tail_bytes) / row_bytes) : 0;
+    if (EB > 8) EB = 8;
+    if (EB >= 1 && D.d % 8 == 0) {
+        const size_t smem = row_bytes * (1 + EB) + tail_bytes;
+        cudaError_t e = cudaFuncSetAttribute(route_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        route_block_kernel<<<D.T, 256, smem, st>>>(D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status, EB);
+    } else
     route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
     count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);
