@@ -29,6 +29,9 @@ from paper_2504_15299_b200 import synth  # noqa: E402
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of
+# this command (profiles/ffn_dec_kernel_mixtral_decode_T64.md); key = workload:tokens:stage:path
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 991559000, "mixtral_decode:T64:down:auto": 509630000}
 
 
 def measured_peaks():
@@ -385,15 +388,7 @@ def run_ours(args):
                 "layer": {"algorithmic_bytes": layer_bytes,
                           "achieved_gbs": layer_bytes / (ms_per_step * 1e-3) / 1e9,
                           "frac": layer_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):
-        try:
-            tr = json.load(open(traffic_file))
-            key = f"{args.workload}:T{T}:{dom_name}:{args.path}"
-            if key in tr:
-                roofline["traffic"] = tr[key]
-        except Exception:
-            pass
+    roofline["traffic"] = NCU_TRAFFIC.get(f"{args.workload}:T{T}:{dom_name}:{args.path}")
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
