@@ -13,9 +13,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
-import tempfile
 import time
 
 import torch
@@ -81,54 +79,68 @@ def algorithmic_bytes(wl, T, group_off):
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Polls NVML (read-only queries) from a background thread every ~2 ms while the timed region runs:
+    SM clock, max SM clock and the active clock-event (throttle) reasons."""
+
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+               "sw_thermal_slowdown": 0x20, "hw_power_brake_slowdown": 0x80}
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
-        self.proc = None
-        self.path = None
+        self.samples = []
+        self.reason_bits = 0
+        self.max_mhz = None
+        self._stop = None
+        self._thread = None
+        self._nvml = None
 
     def start(self):
         try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            import threading
+
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            # CUDA_VISIBLE_DEVICES may renumber devices: match by PCI bus id
+            bus = torch.cuda.get_device_properties(self.gpu).pci_bus_id if hasattr(
+                torch.cuda.get_device_properties(self.gpu), "pci_bus_id") else None
+            handle = None
+            if bus is not None:
+                for i in range(pynvml.nvmlDeviceGetCount()):
+                    h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                    if pynvml.nvmlDeviceGetPciInfo(h).bus == bus:
+                        handle = h
+                        break
+            if handle is None:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self._stop = threading.Event()
+
+            def poll():
+                while not self._stop.is_set():
+                    try:
+                        self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)))
+                        self.reason_bits |= int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(handle))
+                    except Exception:
+                        pass
+                    time.sleep(0.002)
+
+            self._thread = threading.Thread(target=poll, daemon=True)
+            self._thread.start()
         except Exception:
-            self.proc = None
+            self._thread = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.proc is None:
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        if self._thread is None:
             return out
-        try:
-            self.proc.terminate()
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        try:
-            sm, mx, reasons = [], [], set()
-            for line in open(self.path):
-                f = [s.strip() for s in line.split(",")]
-                if len(f) < 9:
-                    continue
-                try:
-                    sm.append(float(f[1])); mx.append(float(f[2]))
-                except ValueError:
-                    continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
-            if sm:
-                sm.sort()
-                out = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                       "samples": len(sm)}
-            os.unlink(self.path)
-        except Exception:
-            pass
+        self._stop.set()
+        self._thread.join(timeout=2)
+        if self.samples:
+            sm = sorted(self.samples)
+            out["sm_mhz"] = sm[len(sm) // 2]
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(n for n, bit in self.REASONS.items() if self.reason_bits & bit)
         return out
 
 
@@ -227,6 +239,20 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's device time."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling: fixed tokens per rank)."""
+    return tokens_per_rank * world / (ms_per_step * 1e-3)
+
+
 def workload_config(wl, T, path):
     return {"workload": f"{wl.name} T={T}: d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} top{wl.top_k} "
                         f"g={wl.group_size} bits={list(wl.bits)} p={list(wl.bit_probs)}",
@@ -323,12 +349,7 @@ def run_ours(args):
     e1.record(stream)
     sync_all()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = e0.elapsed_time(e1)
-    if dist:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
-    ms_per_step = ms_total / args.steps
+    ms_per_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
     stage_ms = [sum(stage_ev[i][s].elapsed_time(stage_ev[i][s + 1]) for i in range(args.steps)) / args.steps
@@ -361,12 +382,7 @@ def run_ours(args):
         e2e_step(i)
     f1.record(stream)
     sync_all()
-    e2e_ms = f0.elapsed_time(f1)
-    if dist:
-        tt = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_ms /= args.steps
+    e2e_ms = max_over_ranks(f0.elapsed_time(f1), dist, dev) / args.steps
 
     if rank != 0:
         if dist:
@@ -392,18 +408,18 @@ def run_ours(args):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        v, per, hid = oracle_tokens_per_s(wl, T, 1, 2, 2, 0, device_for_inputs=dev)
+        v, per, hid = oracle_tokens_per_s(wl, T, 1, 32, 2, 0, device_for_inputs=dev)
         cpu = {"value": v, "unit": UNIT, "cores": used_threads(), "kind": "oracle",
                "sample": f"first token of the batch, all its experts at the routed widths, hidden units "
                          f"0..{hid - 1} of {wl.d_ffn} per expert, time scaled by {wl.d_ffn}/{hid} "
                          f"(extrapolated); 2 passes"}
 
-    line = {"metric": METRIC, "value": T * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+    line = {"metric": METRIC, "value": job_tokens_per_s(T, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic", "config": workload_config(wl, T, args.path),
             "clocks": clocks,
-            "e2e": {"value": T * world / (e2e_ms * 1e-3), "unit": UNIT,
+            "e2e": {"value": job_tokens_per_s(T, world, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": hx[0].numel() * 2 + hfb[0].numel(),
                     "d2h_bytes_per_step": hy.numel() * 2},
             "gpu_launches": B.forward_launch_count(cfg, T) * args.steps,
@@ -416,7 +432,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mixtral_decode", choices=sorted(synth.WORKLOADS))

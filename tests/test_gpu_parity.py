@@ -294,3 +294,58 @@ def test_stack_layer_tiny(B):
     assert np.array_equal(np_f32(xn), moe.round_to_bf16(moe.rmsnorm(x0)))
     for t in range(16):
         assert max_norm_rel_err(np_f32(x)[t], ref[t]) < TOL
+
+
+# ------------------------------------------------------------------ prefill (grouped dequant-GEMM) and the stack
+def test_mixtral_prefill_tensor_path_matches_cuda_core_path(B, mixtral_blobs):
+    """T = 2048 with Zipf-skewed expert loads: the grouped dequant-GEMM (one tile per width, units of up to
+    128 tokens, heavy experts split over many units) against the CUDA-core path on every token."""
+    wl = synth.WORKLOADS["mixtral_prefill"]
+    err, _ = cross_check_paths(B, wl, 2048, mixtral_blobs)
+    assert err < TOL, err
+
+
+def test_mixtral_prefill_sampled_token_against_oracle(B, mixtral_blobs):
+    wl = synth.WORKLOADS["mixtral_prefill"]
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 2048, tokens=[1234], kernel_path=0, blobs=mixtral_blobs)
+    assert max(errs.values()) < TOL, errs
+
+
+def test_stack_two_full_size_layers_teacher_forced(B):
+    """Two layers of the Mixtral-shaped stack (T = 16, learned bit widths): each layer is fed the oracle's
+    input (teacher forcing) and one sampled token of its output is recomputed by the oracle."""
+    _, routing, moe = oracle_mods()
+    wl = synth.WORKLOADS["mixtral_stack"]
+    cfg = B.Config.from_workload(wl)
+    T, tok = 16, 5
+    x_or = np_f32(synth.tokens_bf16(wl, T, "cpu", step=1)).astype(np.float64)
+    for layer in range(2):
+        blobs = gpu_layer(B, cfg, wl, layer=layer)
+        gw = synth.gate_weight_bf16(wl, "cuda", layer=layer)
+        bw = synth.bit_router_weight_bf16(wl, "cuda", layer=layer)
+        x_gpu = torch.from_numpy(x_or.astype(np.float32)).to("cuda", torch.bfloat16)
+        xn = torch.empty_like(x_gpu)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.stack_layer(cfg, x_gpu, xn, blobs, gate_w=gw, bit_w=bw, device_status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        # oracle: same layer, sampled token
+        xn_or = moe.round_to_bf16(moe.rmsnorm(x_or)).astype(np.float64)
+        assert np.array_equal(np_f32(xn), xn_or.astype(np.float32))
+        rt = routing.route(xn_or.astype(np.float32), E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
+                           renormalize=True, gate_w=np_f32(gw), bit_w=np_f32(bw))
+        r_gpu = B.route(cfg, xn, gate_w=gw, bit_w=bw)
+        torch.cuda.synchronize()
+        assert np.array_equal(r_gpu.topk_idx.cpu().numpy(), rt.topk_idx)
+        assert np.array_equal(r_gpu.bit_idx.cpu().numpy(), rt.bit_idx)
+        ol = OracleLayer(wl, layer=layer)
+        y_tok = moe.moe_layer(xn_or, rt, ol, wl.bits, wl.n_experts, tokens=[tok])[tok]
+        ref_row = moe.round_to_bf16(x_or[tok] + y_tok).astype(np.float64)
+        assert max_norm_rel_err(np_f32(x_gpu)[tok], ref_row) < TOL
+        # teacher forcing: the next layer starts from the GPU output only where the oracle has no value;
+        # the sampled row comes from the oracle, the rest is what the GPU produced (already checked above
+        # to route identically)
+        x_next = np_f32(x_gpu).astype(np.float64)
+        x_next[tok] = ref_row
+        x_or = x_next
+        del blobs
