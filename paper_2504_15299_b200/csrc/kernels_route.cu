@@ -196,6 +196,27 @@ __device__ __forceinline__ void stage_row(__nv_bfloat16* dst, const __nv_bfloat1
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
 }
 
+// Gate logits for many experts: a block stages TB token rows and EB weight rows once and forms the
+// TB x EB dot products (pinned order), so a weight row is read once per TB tokens instead of per token.
+__global__ void __launch_bounds__(256)
+gate_logits_kernel(int T, int E, int d, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gate_w,
+                   float* __restrict__ logits, int TB, int EB) {
+    extern __shared__ __align__(16) uint8_t rsm[];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(rsm);
+    __nv_bfloat16* ws = xs + (size_t)TB * d;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t0 = blockIdx.x * TB, e0 = blockIdx.y * EB;
+    const int nt = min(TB, T - t0), ne = min(EB, E - e0);
+    for (int r = 0; r < nt; ++r) stage_row(xs + (size_t)r * d, x + (size_t)(t0 + r) * d, d);
+    for (int r = 0; r < ne; ++r) stage_row(ws + (size_t)r * d, gate_w + (size_t)(e0 + r) * d, d);
+    __syncthreads();
+    for (int pr = warp; pr < nt * ne; pr += 8) {
+        const int tt = pr / ne, ee = pr - tt * ne;
+        const float v = dot_pinned_smem(xs + (size_t)tt * d, ws + (size_t)ee * d, d, lane);
+        if (lane == 0) logits[(size_t)(t0 + tt) * E + e0 + ee] = v;
+    }
+}
+
 // One block (8 warps) per token: the same results as route_kernel, with the token row and batches of
 // EB weight rows staged in shared memory by 16-byte loads (the pinned summation order makes a lane
 // walk a row with stride 32, which is slow straight from global memory); warp w takes row w of a batch.
@@ -330,7 +351,7 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
 
 cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
                          const float* logits_in, const __nv_bfloat16* bit_w, const int8_t* forced,
-                         const RouteBufs& R, float* /*logits_ws*/, int32_t* keys_ws, int32_t* hist_ws,
+                         const RouteBufs& R, float* logits_ws, int32_t* keys_ws, int32_t* hist_ws,
                          int32_t* device_status, cudaStream_t st) {
     const int warps_per_block = 4;
     const int n_keys = D.E * D.K;
@@ -341,6 +362,17 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     int EB = row_bytes + tail_bytes < budget ? (int)((budget - row_bytes - tail_bytes) / row_bytes) : 0;
     if (EB > 8) EB = 8;
     if (EB >= 1 && D.d % 8 == 0) {
+        // many experts: gate logits by the tiled kernel first, then route from those logits
+        if (!logits_in && D.E > 16 && logits_ws && 16 * row_bytes <= budget) {
+            const int TB = 8, EBL = 8;
+            const size_t lsm = (size_t)(TB + EBL) * row_bytes;
+            cudaError_t e = cudaFuncSetAttribute(gate_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsm);
+            if (e != cudaSuccess) return e;
+            dim3 grid((D.T + TB - 1) / TB, (D.E + EBL - 1) / EBL);
+            gate_logits_kernel<<<grid, 256, lsm, st>>>(D.T, D.E, D.d, x, gate_w, logits_ws, TB, EBL);
+            logits_in = logits_ws;
+            gate_w = nullptr;
+        }
         const size_t smem = row_bytes * (1 + EB) + tail_bytes;
         cudaError_t e = cudaFuncSetAttribute(route_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
