@@ -57,6 +57,7 @@ struct DecParams {
     long long R_alloc;
     int32_t* status;
     int smem_w_off, smem_epi_off, smem_bar_off;
+    int dbg;                  // debug builds only: bit 0 skips the MMAs, bit 1 skips the dequant math
 };
 
 struct DecItem { int unit, tile, split, g0, g1; };
@@ -165,7 +166,7 @@ struct SegList {
 // when the list has at most four), both halves, straight-line code.  fac[q], cfac[q]: per-item factors
 // so that multiplier(position 0) = s1 * fac and the tile constant = s1 * cfac (segment 0: lo * 2^-S).
 template <int GS, int SWPACK, int WG, typename WaitEmpty, typename Publish>
-__device__ __forceinline__ void dequant_group_fixed(uint32_t wb, int rr, int kmax, float s1, float lo_scaled,
+__device__ __forceinline__ void dequant_group_fixed(int dbg, uint32_t wb, int rr, int kmax, float s1, float lo_scaled,
                                                     const float (&fac)[2], const float (&cfac)[2], uint32_t a_slots,
                                                     WaitEmpty&& wait_empty, Publish&& publish) {
     using SL = SegList<SWPACK>;
@@ -185,7 +186,7 @@ __device__ __forceinline__ void dequant_group_fixed(uint32_t wb, int rr, int kma
             addend[q] = __float2half2_rn(j == 0 ? lo_scaled : s1 * cfac[q]);
         }
     }
-#pragma unroll
+#pragma unroll 1
     for (int h = 0; h < HALVES; ++h) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -196,6 +197,9 @@ __device__ __forceinline__ void dequant_group_fixed(uint32_t wb, int rr, int kma
                     wait_empty(q);
                     const uint32_t seg = wb + (uint32_t)SL::seg_off(GS, j < 8 ? j : 0);
                     const uint32_t taddr = a_slots + q * 32;
+#ifdef D2MOE_WAIT_STATS
+                    if (dbg & 2) { publish(q); continue; }
+#endif
                     if (SL::sw(j < 8 ? j : 0) == 1) dequant_half_tile<GS, 1>(seg, rr, h, mult[q], addend[q], taddr);
                     else if (SL::sw(j < 8 ? j : 0) == 2) dequant_half_tile<GS, 2>(seg, rr, h, mult[q], addend[q], taddr);
                     else if (SL::sw(j < 8 ? j : 0) == 4) dequant_half_tile<GS, 4>(seg, rr, h, mult[q], addend[q], taddr);
@@ -349,14 +353,15 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
                     { STAT_T0(); mbar_wait(B_FULL(s), (it / DEC_NSB) & 1, abort_flag, p.status); STAT_ADD(3); }
                     const uint64_t bdesc = smem_desc_sw128(bbuf + s * b_slot_bytes);
                     const uint32_t first = (G != ii.g0) ? 1u : 0u;
-#pragma unroll
+#pragma unroll 1
                     for (int qp = 0; qp < 2; ++qp) {                  // pairs of my segments: slots 0 and 1
-#pragma unroll
+#pragma unroll 1
                         for (int h = 0; h < HALVES; ++h) {
 #pragma unroll
                             for (int sl = 0; sl < 2; ++sl) {
                                 const int q = 2 * qp + sl;
                                 if (q < n_mine) {
+                                    const uint32_t idq = q == 0 ? idesc[0] : q == 1 ? idesc[1] : q == 2 ? idesc[2] : idesc[3];
                                     const uint32_t d_addr = d_tmem + (2 * q + w) * p.n_cap;
                                     const uint32_t a_addr = sl ? a_slot1 : a_slot0;
                                     const uint32_t use = sl ? use1 : use0;
@@ -366,10 +371,15 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
                                     {
                                         STAT_T0();
                                         if (elect_one()) {
-                                            tc_mma_ts(d_addr, a_addr + 0, bh + 0, idesc[q], h == 0 ? first : 1u);
-                                            tc_mma_ts(d_addr, a_addr + 8, bh + 2, idesc[q], 1u);
-                                            tc_mma_ts(d_addr, a_addr + 16, bh + 4, idesc[q], 1u);
-                                            tc_mma_ts(d_addr, a_addr + 24, bh + 6, idesc[q], 1u);
+#ifdef D2MOE_WAIT_STATS
+                                            if (!(p.dbg & 1))
+#endif
+                                            {
+                                                tc_mma_ts(d_addr, a_addr + 0, bh + 0, idq, h == 0 ? first : 1u);
+                                                tc_mma_ts(d_addr, a_addr + 8, bh + 2, idq, 1u);
+                                                tc_mma_ts(d_addr, a_addr + 16, bh + 4, idq, 1u);
+                                                tc_mma_ts(d_addr, a_addr + 24, bh + 6, idq, 1u);
+                                            }
                                             tc_commit(A_EMPTY(w, sl));
                                         }
                                         __syncwarp();
@@ -453,8 +463,8 @@ ffn_dec_kernel(const __grid_constant__ DecParams p, const __grid_constant__ TmaM
                         if (sl) ++use1; else ++use0;
                     };
                     const float s1raw = __low2float(mh);
-                    if (wg == 0) dequant_group_fixed<GS, SWPACK, 0>(wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + lane_addr, wait_empty, publish);
-                    else dequant_group_fixed<GS, SWPACK, 1>(wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + 64 + lane_addr, wait_empty, publish);
+                    if (wg == 0) dequant_group_fixed<GS, SWPACK, 0>(p.dbg, wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + lane_addr, wait_empty, publish);
+                    else dequant_group_fixed<GS, SWPACK, 1>(p.dbg, wb, rr, kmax, s1raw, lo, fac, cfac, a_tmem + 64 + lane_addr, wait_empty, publish);
                 } else {
                 // my segments j = wg + 2q, in pairs: q = 2qp + sl fills operand slot sl
                     const int n_mine = kmax >= wg ? (kmax - wg) / 2 + 1 : 0;
@@ -666,7 +676,9 @@ dec_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __r
 
 }  // namespace
 
+static int g_host_dbg_mode = 0;
 #ifdef D2MOE_WAIT_STATS
+extern "C" int d2moe_debug_set_mode(int mode) { g_host_dbg_mode = mode; return 0; }
 extern "C" int d2moe_debug_wait_stats(unsigned long long* host16, int reset) {
     cudaDeviceSynchronize();
     if (cudaMemcpyFromSymbol(host16, g_wait_stats, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
@@ -699,6 +711,7 @@ cudaError_t launch_ffn_decode(const d2moe_config* c, const MoeDims& D, const Pac
         p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
         p.units = B.units; p.n_units = B.n_units;
         p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
+        p.dbg = g_host_dbg_mode;
         const int b_bytes = DEC_NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
         const int epi_bytes = 2 * 64 * DEC_EPI_STRIDE * 4;

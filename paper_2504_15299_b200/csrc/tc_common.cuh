@@ -49,10 +49,10 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 }
 
 // Bounded wait.  `abort_flag` (shared) is set by the first wait that runs out (about one second);
-// once it is set no wait blocks any more, so the CTA drains and exits instead of hanging.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          bool drain = false) {
-    if (mbar_try(bar, parity)) return;
+// once it is set no wait blocks any more, so the CTA drains and exits instead of hanging.  The loop
+// lives in a function of its own: the waits are inlined dozens of times and the hot loops of the
+// expert kernels are bound by instruction fetch, so only the first try is inline.
+static __device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, bool drain) {
     unsigned long long t0 = 0;
     for (unsigned spin = 0;; ++spin) {
         if (mbar_try_sleep(bar, parity, 4000u)) return;
@@ -67,6 +67,11 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          bool drain = false) {
+    if (mbar_try(bar, parity)) return;
+    mbar_wait_slow(bar, parity, abort_flag, status, drain);
 }
 
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
