@@ -510,7 +510,7 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     pl->decode = avg <= 24 ? 1 : 0;
     if (pl->decode) {
         int cap = (128 / c->n_bits) & ~15;
-        pl->n_cap = cap > 64 ? 64 : cap;
+        pl->n_cap = cap > 32 ? 32 : cap;     // 32 tokens x g columns of activations per ring slot
     } else {
         pl->n_cap = 128;
     }

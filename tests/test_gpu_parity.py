@@ -349,3 +349,87 @@ def test_stack_two_full_size_layers_teacher_forced(B):
         x_next[tok] = ref_row
         x_or = x_next
         del blobs
+
+
+# ------------------------------------------------------------------ other width lists, group sizes, loads
+def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=21, one_expert=False):
+    """Random small layer through the tensor-core path, the CUDA-core path and the oracle."""
+    _, routing, moe = oracle_mods()
+    from oracle import mwq
+    K = len(bits)
+    cfg_tc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=0)
+    cfg_cc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=1)
+    raw = {}
+    blobs = []
+    for e in range(E + n_shared):
+        mats = []
+        for m in range(3):
+            shape = (F, d) if m < 2 else (d, F)
+            W = synth.normal(seed, 100 + 3 * e + m, shape, 0.02, "cuda")
+            mats.append(np_f32(W))
+            blobs.append(B.pack_mwq(cfg_tc, W))
+        raw[e] = mats
+    x = synth.bf16_exact(synth.normal(seed, 1, (T, d), 1.0, "cuda"))
+    logits = synth.normal(seed, 5, (T, E), 1.0, "cuda")
+    if one_expert:
+        logits[:, 0] += 100.0          # every token picks expert 0 first: units beyond n_cap
+    fb = synth.categorical(seed, 4, (T, k), probs or [1.0 / K] * K, "cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_tc = B.moe_forward(cfg_tc, x, blobs, logits=logits, forced_bit_idx=fb, device_status=st)
+    y_cc = B.moe_forward(cfg_cc, x, blobs, logits=logits, forced_bit_idx=fb, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    a, b = y_cc.float(), y_tc.float()
+    cross = float(((a - b).abs().amax(dim=1) / a.abs().amax(dim=1)).max().item())
+    rt = routing.route(np_f32(x), E=E, K=K, top_k=k, renormalize=True, logits=np_f32(logits),
+                       forced_bit_idx=fb.cpu().numpy())
+    packed = {}
+
+    def get(e):
+        if e not in packed:
+            packed[e] = tuple(mwq.quantize(W, bits, g) for W in raw[e])
+        return packed[e]
+
+    toks = sorted(set([0, T // 2, T - 1]))
+    ref = moe.moe_layer(np_f32(x), rt, get, bits, E, n_shared, tokens=toks)
+    err = max(max_norm_rel_err(np_f32(y_tc)[t], ref[t]) for t in toks)
+    return cross, err
+
+
+@pytest.mark.parametrize("bits,g", [((2, 3, 4), 128), ((4, 8), 128), ((8,), 64), ((1, 2, 3, 4, 5, 6, 7, 8), 128),
+                                    ((3, 5), 64), ((2, 8), 128), ((5, 6, 7, 8), 64)])
+def test_other_width_lists_on_the_tensor_core_paths(B, bits, g):
+    cross, err = small_layer_case(B, d=256, F=384, E=4, k=2, g=g, bits=bits, T=24)
+    assert cross < TOL and err < TOL, (cross, err)
+
+
+def test_all_tokens_on_one_expert_and_shared_experts(B):
+    # 80 tokens all choose expert 0 (units beyond the per-unit token cap), one shared expert on top
+    cross, err = small_layer_case(B, d=256, F=256, E=4, k=2, g=128, bits=(2, 3, 4, 8), T=80, n_shared=1,
+                                  one_expert=True)
+    assert cross < TOL and err < TOL, (cross, err)
+
+
+def test_prefill_sized_load_small_shape(B):
+    # 400 tokens on 2 experts: the grouped dequant-GEMM path (more than 24 tokens per expert)
+    cross, err = small_layer_case(B, d=256, F=256, E=2, k=1, g=128, bits=(2, 3, 4, 8), T=400,
+                                  probs=[0.1, 0.2, 0.4, 0.3])
+    assert cross < TOL and err < TOL, (cross, err)
+
+
+def test_single_token_and_single_width(B):
+    cross, err = small_layer_case(B, d=128, F=128, E=2, k=1, g=64, bits=(2, 4, 8), T=1, probs=[0, 0, 1.0])
+    assert cross < TOL and err < TOL, (cross, err)
+
+
+@pytest.mark.parametrize("d,F,g", [(192, 256, 64), (256, 160, 32), (512, 512, 256)])
+def test_shapes_outside_the_tensor_core_path_use_the_cuda_core_path(B, d, F, g):
+    # d % 128 != 0, F % 64 != 0 or g not in {64, 128}: kernel_path AUTO must still be right
+    cross, err = small_layer_case(B, d=d, F=F, E=3, k=2, g=g, bits=(2, 4, 8), T=9)
+    assert cross < TOL and err < TOL, (cross, err)
+    cfg = B.Config(d, F, 3, 2, g, (2, 4, 8), kernel_path=2)
+    x = torch.zeros((1, d), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.D2MoEError) as e:
+        B.moe_forward(cfg, x, [x] * 9, logits=torch.zeros((1, 3), device="cuda"),
+                      forced_bit_idx=torch.zeros((1, 2), dtype=torch.int8, device="cuda"))
+    assert e.value.code == 4
