@@ -21,23 +21,27 @@
 // All tiles carry a common power-of-two factor 2^-S (S per matrix, from the largest scale seen at
 // pack time) so that the multipliers stay inside fp16 range; the epilogue multiplies by 2^S.
 //
-// Warp roles (224 threads, 2 CTAs per SM): 0-3 dequant + epilogue, 4 weight producer (bulk async
-// copies of packed blocks, HBM -> shared), 5 activation producer (TMA tensor loads, 128B swizzle),
-// 6 MMA issuer.  Every wait is bounded: on expiry the CTA raises D2MOE_DEV_TIMEOUT, stops
-// waiting, drains and exits.
+// Warp roles (352 threads, 1 CTA per SM, all 512 TMEM columns): warps 0-3 and 4-7 are two dequant
+// warpgroups, each owning one K-half of every tile (thread = weight row = TMEM lane) and taking
+// alternate 16-column chunks of the epilogue; warp 8 streams packed blocks (cp.async.bulk), warp 9
+// streams activation tiles (TMA, 128B swizzle, boxes of up to 256 rows), warp 10 issues the MMAs (the
+// whole warp runs the loop, one elected lane issues).  A unit holds up to 320 tokens, so that one
+// dequantization of a weight tile is amortised over enough tensor work to leave the kernel bound by
+// the tensor cores; an MMA covers at most 256 of a piece's columns.  Every wait is bounded: on expiry
+// the CTA raises D2MOE_DEV_TIMEOUT, stops waiting, drains and exits.
 #include "d2moe_common.cuh"
 #include "kernels_ffn_tc.cuh"
 #include "tc_common.cuh"
 
 namespace {
 
-constexpr int TC_THREADS = 224;
-constexpr int WARP_WPROD = 4, WARP_BPROD = 5, WARP_MMA = 6;
-constexpr int TMEM_COLS = 256;
-constexpr int D_COLS = 128;            // accumulator columns (n_cap <= 128)
-constexpr int A_SLOTS = 2;
+constexpr int TC_THREADS = 352;        // 8 dequant warps (2 warpgroups) + weight producer + activation producer + MMA issuer
+constexpr int WARP_WPROD = 8, WARP_BPROD = 9, WARP_MMA = 10;
+constexpr int TMEM_COLS = 512;
+constexpr int D_COLS = 384;            // accumulator columns (n_cap <= 320)
+constexpr int A_SLOTS = 2;             // operand tiles of GS/2 columns at TMEM columns 384 and 448
 constexpr int NSB = 2;                 // activation ring depth
-constexpr int MAX_NSW = 8;             // weight ring depth (upper bound)
+constexpr int MAX_NSW = 4;             // weight ring depth (upper bound)
 constexpr int EPI_STRIDE = 17;
 
 struct TcParams {
@@ -56,19 +60,22 @@ struct TcParams {
 };
 
 // ------------------------------------------------------------------------------------------------
-// Dequantization of one segment of one row into the running tile.
+// Dequantization of one K-half of one segment of one row into the running tile.
 //   seg     shared-memory address of the segment inside the block (this row's chunks are at
 //           (c*64 + rr)*cs)
-//   acc     running tile U (GS/2 half2 registers: register i = elements 2i, 2i+1 of the group)
+//   half    which half of the group's g elements this warpgroup owns (0 or 1)
+//   acc     running tile U (GS/4 half2 registers: register i = elements 2i, 2i+1 of the half)
 //   m0      multiplier for a code at bit position 0: M_j * 2^(24 - S); position p uses m0 * 2^-p
 //   FIRST   segment 0: the addend is u0 = (lo - s1/2) * 2^-S instead of acc
 // ------------------------------------------------------------------------------------------------
 template <int GS, int SW, bool FIRST>
-__device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, __half2 (&acc)[GS / 2], __half2 m0, __half2 u0) {
+__device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], __half2 m0, __half2 u0) {
     constexpr int ROW_BYTES = GS * SW / 8;
     constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
-    constexpr int NCHUNK = ROW_BYTES / CS;
-    constexpr int WPC = CS / 4;                 // words per chunk
+    constexpr int HB = ROW_BYTES / 2;            // bytes of this half
+    constexpr int LD = HB < 16 ? HB : 16;
+    constexpr int NLD = HB / LD;
+    constexpr int WPL = LD / 4;                 // words per load
     constexpr int PER = 16 / SW;                // registers per word
     constexpr int NPOS = 8 / SW;                // distinct bit positions per byte lane
     constexpr uint32_t FIELD = ((1u << SW) - 1u) * 0x00010001u;
@@ -78,26 +85,26 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, __half2 (&
 #pragma unroll
     for (int q = 1; q < NPOS; ++q) mult[q] = __hmul2(mult[q - 1], step);
 #pragma unroll
-    for (int c = 0; c < NCHUNK; ++c) {
-        uint32_t w[WPC];
-        const uint32_t addr = seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS);
-        if constexpr (WPC == 4) {
+    for (int l = 0; l < NLD; ++l) {
+        uint32_t w[WPL];
+        const int off = half * HB + l * LD;
+        const int c = off / CS, within = off % CS;
+        const uint32_t addr = seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS + within);
+        if constexpr (WPL == 4) {
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
-        } else if constexpr (WPC == 2) {
+        } else if constexpr (WPL == 2) {
             asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr));
         } else {
             asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[0]) : "r"(addr));
         }
 #pragma unroll
-        for (int q = 0; q < WPC; ++q) {
-            const int m = c * WPC + q;
+        for (int q = 0; q < WPL; ++q) {
             const uint32_t lo8 = w[q], hi8 = w[q] >> 8;
 #pragma unroll
             for (int e = 0; e < PER; ++e) {
-                const int pos = (e % NPOS) * SW;
                 const uint32_t src = e < NPOS ? lo8 : hi8;
-                const __half2 code = as_h2(src & (FIELD << pos));
-                const int i = m * PER + e;
+                const __half2 code = as_h2(src & (FIELD << ((e % NPOS) * SW)));
+                const int i = (l * WPL + q) * PER + e;
                 acc[i] = __hfma2(code, mult[e % NPOS], FIRST ? u0 : acc[i]);
             }
         }
@@ -105,12 +112,12 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, __half2 (&
 }
 
 template <int GS, bool FIRST>
-__device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, __half2 (&acc)[GS / 2], __half2 m0, __half2 u0) {
+__device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], __half2 m0, __half2 u0) {
     switch (sw) {
-        case 1: dequant_segment<GS, 1, FIRST>(seg, rr, acc, m0, u0); break;
-        case 2: dequant_segment<GS, 2, FIRST>(seg, rr, acc, m0, u0); break;
-        case 4: dequant_segment<GS, 4, FIRST>(seg, rr, acc, m0, u0); break;
-        default: dequant_segment<GS, 8, FIRST>(seg, rr, acc, m0, u0); break;
+        case 1: dequant_segment<GS, 1, FIRST>(seg, rr, half, acc, m0, u0); break;
+        case 2: dequant_segment<GS, 2, FIRST>(seg, rr, half, acc, m0, u0); break;
+        case 4: dequant_segment<GS, 4, FIRST>(seg, rr, half, acc, m0, u0); break;
+        default: dequant_segment<GS, 8, FIRST>(seg, rr, half, acc, m0, u0); break;
     }
 }
 
@@ -134,20 +141,20 @@ __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
 // The kernel
 // ------------------------------------------------------------------------------------------------
 template <int GS>
-__global__ void __launch_bounds__(TC_THREADS, 2)
+__global__ void __launch_bounds__(TC_THREADS, 1)
 ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMaps maps) {
+    constexpr int HALVES = GS / 64;              // 64-element K slabs of the activation tile
+    constexpr int TILE_COLS = GS / 2;            // TMEM columns of one operand tile
     extern __shared__ uint8_t smem_raw[];
     // shared layout (from a 1024-byte boundary, which the 128B-swizzled operand tiles need):
-    // [activation ring: NSB x n_cap*GS*2] [weight ring: nsw x 2 blocks] [epilogue] [barriers]
+    // [activation ring: NSB x n_cap*GS*2] [weight ring: nsw x 2 blocks] [epilogue x2] [barriers]
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t b_slot_bytes = (uint32_t)p.n_cap * GS * 2;
     const uint32_t w_slot_bytes = 2u * (uint32_t)p.L.block_bytes;
     const uint32_t bbuf = smem_base;
     const uint32_t wbuf = smem_base + p.smem_w_off;
-    float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.smem_bar_off);
-    // barrier indices
     const uint32_t bar0 = smem_u32(bars);
     auto W_FULL = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     auto W_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(MAX_NSW + i); };
@@ -163,11 +170,11 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 128); }
+        for (int i = 0; i < MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 256); }
         for (int i = 0; i < NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 1); }
-        for (int i = 0; i < A_SLOTS; ++i) { mbar_init(A_FULL(i), 128); mbar_init(A_EMPTY(i), 1); }
+        for (int i = 0; i < A_SLOTS; ++i) { mbar_init(A_FULL(i), 256); mbar_init(A_EMPTY(i), 1); }
         mbar_init(D_FULL, 1);
-        mbar_init(D_EMPTY, 128);
+        mbar_init(D_EMPTY, 256);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -181,8 +188,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t d_tmem = tmem_base;                       // columns [0, 128)
-    const uint32_t a_tmem = tmem_base + D_COLS;              // A_SLOTS tiles of GS/2 columns
+    const uint32_t d_tmem = tmem_base;                       // columns [0, n_cap)
+    const uint32_t a_tmem = tmem_base + D_COLS;              // A_SLOTS tiles, 64 columns apart
 
     const int n_units = *p.n_units;
     const int total_items = n_units * p.n_row_tiles * p.n_split;
@@ -212,7 +219,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             }
             // drain: every copy issued must have landed before the CTA may exit
             for (int s = 0; s < nsw && s < (int)it; ++s) {
-                const uint32_t last = it - 1 - ((it - 1 - s) % nsw + nsw) % nsw;   // last iteration that used slot s
+                const uint32_t last = it - 1 - (it - 1 - s) % nsw;   // last iteration that used slot s
                 mbar_wait(W_FULL(s), (last / nsw) & 1, abort_flag, p.status, true);
             }
         }
@@ -223,71 +230,86 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
                 const ItemInfo ii = decode_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
-                const int ncols = u->ncols;
-                int mi = 0, box = 16;
-                while (box < ncols) { box <<= 1; ++mi; }
-                const uint32_t bytes = (uint32_t)box * 128u * (GS / 64);
+                const int ncols = u->ncols;                       // multiple of 16, <= n_cap
+                const uint32_t bytes = (uint32_t)ncols * 128u * HALVES;
                 for (int G = ii.g0; G < ii.g1; ++G, ++it) {
                     const int s = it % NSB;
                     mbar_wait(B_EMPTY(s), ((it / NSB) & 1) ^ 1, abort_flag, p.status);
                     mbar_expect_tx(B_FULL(s), bytes);
                     const uint32_t dst = bbuf + s * b_slot_bytes;
+                    // the rows of the unit as boxes of 256, 128, 64, 32, 16 rows (largest first)
+                    int r = 0;
+                    for (int mi = 4; mi >= 0; --mi) {
+                        const int box = 16 << mi;
+                        while (ncols - r >= box) {
 #pragma unroll
-                    for (int h = 0; h < GS / 64; ++h)
-                        tma_load_2d(dst + h * (uint32_t)p.n_cap * 128u, &maps.m[mi], G * GS + h * 64, u->row0, B_FULL(s));
+                            for (int h = 0; h < HALVES; ++h)
+                                tma_load_2d(dst + h * (uint32_t)p.n_cap * 128u + (uint32_t)r * 128u, &maps.m[mi],
+                                            G * GS + h * 64, u->row0 + r, B_FULL(s));
+                            r += box;
+                        }
+                    }
                 }
             }
             for (int s = 0; s < NSB && s < (int)it; ++s) {
-                const uint32_t last = it - 1 - ((it - 1 - s) % NSB + NSB) % NSB;
+                const uint32_t last = it - 1 - (it - 1 - s) % NSB;
                 mbar_wait(B_FULL(s), (last / NSB) & 1, abort_flag, p.status, true);
             }
         }
     } else if (warp == WARP_MMA) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            uint32_t it = 0, at = 0, ic = 0;
-            for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
-                const ItemInfo ii = decode_item(p, item);
-                const TcUnit* u = p.units + ii.unit;
-                const int kmax = u->kmax;
-                mbar_wait(D_EMPTY, (ic & 1) ^ 1, abort_flag, p.status);
-                tc_fence_after();
-                for (int G = ii.g0; G < ii.g1; ++G, ++it) {
-                    const int s = it % NSB;
-                    mbar_wait(B_FULL(s), (it / NSB) & 1, abort_flag, p.status);
-                    const uint32_t bsl = bbuf + s * b_slot_bytes;
-                    for (int kk = 0; kk <= kmax; ++kk) {
-                        const int cnt = u->cnt[kk];
-                        if (cnt == 0) continue;
-                        const int slot = at % A_SLOTS;
-                        mbar_wait(A_FULL(slot), (at / A_SLOTS) & 1, abort_flag, p.status);
-                        tc_fence_after();
-                        const uint32_t idesc = instr_desc_f16(cnt);
-                        const int col0 = u->col0[kk];
+        // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
+        uint32_t it = 0, at = 0, ic = 0;
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
+            const ItemInfo ii = decode_item(p, item);
+            const TcUnit* u = p.units + ii.unit;
+            const int kmax = u->kmax;
+            mbar_wait(D_EMPTY, (ic & 1) ^ 1, abort_flag, p.status);
+            tc_fence_after();
+            for (int G = ii.g0; G < ii.g1; ++G, ++it) {
+                const int s = it % NSB;
+                mbar_wait(B_FULL(s), (it / NSB) & 1, abort_flag, p.status);
+                const uint32_t bsl = bbuf + s * b_slot_bytes;
+                for (int kk = 0; kk <= kmax; ++kk) {
+                    const int cnt = u->cnt[kk];
+                    if (cnt == 0) continue;
+                    const int slot = at % A_SLOTS;
+                    mbar_wait(A_FULL(slot), (at / A_SLOTS) & 1, abort_flag, p.status);
+                    tc_fence_after();
+                    const int col0 = u->col0[kk];
+                    if (elect_one()) {
+                        for (int c = 0; c < cnt; c += 256) {          // an MMA covers at most 256 columns
+                            const int n = min(256, cnt - c);
+                            const uint32_t idesc = instr_desc_f16(n);
+                            const uint64_t bd = smem_desc_sw128(bsl + (uint32_t)(col0 + c) * 128u);
 #pragma unroll
-                        for (int j = 0; j < GS / 16; ++j) {
-                            const uint32_t a_addr = a_tmem + slot * (GS / 2) + j * 8;
-                            const uint32_t b_addr = bsl + (j >> 2) * (uint32_t)p.n_cap * 128u + (uint32_t)col0 * 128u + (j & 3) * 32u;
-                            tc_mma_ts(d_tmem + col0, a_addr, smem_desc_sw128(b_addr), idesc,
-                                      (G != ii.g0 || j != 0) ? 1u : 0u);
+                            for (int j = 0; j < GS / 16; ++j) {
+                                const uint32_t a_addr = a_tmem + slot * 64 + j * 8;
+                                const uint64_t bj = bd + (uint64_t)(((j >> 2) * (uint32_t)p.n_cap * 128u + (j & 3) * 32u) >> 4);
+                                tc_mma_ts(d_tmem + col0 + c, a_addr, bj, idesc, (G != ii.g0 || j != 0) ? 1u : 0u);
+                            }
                         }
                         tc_commit(A_EMPTY(slot));
-                        ++at;
                     }
-                    tc_commit(B_EMPTY(s));
+                    __syncwarp();
+                    ++at;
                 }
-                tc_commit(D_FULL);
+                if (elect_one()) tc_commit(B_EMPTY(s));
+                __syncwarp();
             }
-            // all MMAs must be complete before TMEM is freed
-            if (ic > 0) mbar_wait(D_FULL, (ic - 1) & 1, abort_flag, p.status, true);
+            if (elect_one()) tc_commit(D_FULL);
+            __syncwarp();
         }
+        // all MMAs must be complete before TMEM is freed
+        if (ic > 0) mbar_wait(D_FULL, (ic - 1) & 1, abort_flag, p.status, true);
     } else {
-        // ---------------- dequant + epilogue warps ----------------
-        const int r = threadIdx.x;               // row of the tile = TMEM lane
+        // ---------------- dequant + epilogue warps: warpgroup wg owns K-half wg of every tile ----------------
+        const int wg = warp >> 2;
+        const int r = threadIdx.x & 127;         // row of the tile = TMEM lane
         const int blk = r >> 6, rr = r & 63;
-        const uint32_t lane_addr = ((uint32_t)(warp * 32)) << 16;
+        const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
+        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * EPI_STRIDE);
         uint32_t it = 0, at = 0, ic = 0;
-        __half2 acc[GS / 2];
+        __half2 acc[GS / 4];
         for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
             const ItemInfo ii = decode_item(p, item);
             const TcUnit* u = p.units + ii.unit;
@@ -298,6 +320,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             unsigned present = 0;
             for (int kk = 0; kk <= kmax; ++kk) present |= (u->cnt[kk] > 0 ? 1u : 0u) << kk;
 
+#pragma unroll 1
             for (int G = ii.g0; G < ii.g1; ++G, ++it) {
                 const int s = it % nsw;
                 mbar_wait(W_FULL(s), (it / nsw) & 1, abort_flag, p.status);
@@ -314,16 +337,16 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     const float Mk = s1 * exp2f((float)(-(p.D.bits[kk] - p.D.bits[0]))) * two_mS;
                     const __half2 m0 = h2dup(Mk * 16777216.0f);
                     const uint32_t seg = wb + (uint32_t)p.L.seg_off[kk];
-                    if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, acc, m0, u0);
-                    else dequant_dispatch<GS, false>(sw, seg, rr, acc, m0, u0);
+                    if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
+                    else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
                     if ((present >> kk) & 1u) {
                         const int slot = at % A_SLOTS;
                         mbar_wait(A_EMPTY(slot), ((at / A_SLOTS) & 1) ^ 1, abort_flag, p.status);
                         tc_fence_after();
                         const __half2 half_m = h2dup(0.5f * Mk);
-                        const uint32_t dst = a_tmem + slot * (GS / 2) + lane_addr;
+                        const uint32_t dst = a_tmem + slot * 64 + wg * (TILE_COLS / 2) + lane_addr;
 #pragma unroll
-                        for (int c = 0; c < GS / 32; ++c) {
+                        for (int c = 0; c < GS / 64; ++c) {
                             uint32_t v[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = as_u32(__hadd2(acc[c * 16 + j], half_m));
@@ -338,18 +361,18 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 mbar_arrive(W_EMPTY(s));
             }
 
-            // ---- epilogue: D (128 rows x ncols) -> global ----
+            // ---- epilogue: D (128 rows x ncols) -> global; the two warpgroups take alternate 16-column chunks ----
             mbar_wait(D_FULL, ic & 1, abort_flag, p.status);
             tc_fence_after();
             const float two_S = exp2f((float)S);
             const int ncols = u->ncols;
-            for (int c0 = 0; c0 < ncols; c0 += 16) {
+            for (int c0 = wg * 16; c0 < ncols; c0 += 32) {
                 int nreal = 0;
                 for (int kk = 0; kk <= kmax; ++kk) {
                     const int rel = c0 - u->col0[kk];
                     if (u->cnt[kk] > 0 && rel >= 0 && rel < u->cnt[kk]) nreal = min(16, max(0, u->real[kk] - rel));
                 }
-                if (nreal == 0) continue;            // padding columns only (uniform across the CTA)
+                if (nreal == 0) continue;            // padding columns only (uniform across the warpgroup)
                 uint32_t v[16];
                 tc_ld16(d_tmem + lane_addr + c0, v);
                 tc_wait_ld();
@@ -359,7 +382,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 #pragma unroll
                         for (int j = 0; j < 16; ++j) epi[rr * EPI_STRIDE + j] = __uint_as_float(v[j]) * two_S;
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
                     if (blk == 0) {
                         __half* dst = p.hbuf + grow * p.D.F + (long long)ii.tile * 64 + rr;
 #pragma unroll
@@ -371,7 +394,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                             }
                         }
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
                 } else {
                     float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + r;
 #pragma unroll
@@ -512,7 +535,7 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
         int cap = (128 / c->n_bits) & ~15;
         pl->n_cap = cap > 32 ? 32 : cap;     // 32 tokens x g columns of activations per ring slot
     } else {
-        pl->n_cap = 128;
+        pl->n_cap = 320;
     }
     const long long n_pieces = pl->decode ? (long long)c->n_experts + c->n_shared
                                           : (long long)c->n_experts * c->n_bits + c->n_shared;
@@ -558,9 +581,9 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
         const int b_bytes = NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
-        const int epi_bytes = 64 * EPI_STRIDE * 4;
+        const int epi_bytes = 2 * 64 * EPI_STRIDE * 4;
         const int bar_bytes = 512;
-        const int budget = 112 * 1024;
+        const int budget = 224 * 1024;
         int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
         if (nsw > MAX_NSW) nsw = MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
@@ -574,11 +597,11 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         if (D.g == 128) {
             e = cudaFuncSetAttribute(ffn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
             if (e != cudaSuccess) return e;
-            ffn_tc_kernel<128><<<2 * sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            ffn_tc_kernel<128><<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
         } else {
             e = cudaFuncSetAttribute(ffn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
             if (e != cudaSuccess) return e;
-            ffn_tc_kernel<64><<<2 * sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            ffn_tc_kernel<64><<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
