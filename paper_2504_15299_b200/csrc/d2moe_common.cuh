@@ -13,7 +13,7 @@
 #define D2MOE_TILE_ROWS 64          // rows per packed block
 #define D2MOE_HEADER_BYTES 256
 #define D2MOE_MAGIC 0x4D32444Du     // "MD2M"
-#define D2MOE_LAYOUT_VERSION 1u
+#define D2MOE_LAYOUT_VERSION 2u
 #define D2MOE_MAX_EXPERTS 320       // routed + shared
 
 // ------------------------------------------------------------------------------------------------
@@ -26,9 +26,12 @@
 //   [shift_j + w_j - 1 : shift_j] of the top-width code) stored sw_j in {1,2,4,8} bits each, i.e.
 //   g*sw_j/8 bytes per row, cut in chunks of cs_j = min(16, g*sw_j/8) bytes; chunk c of row r lies
 //   at byte (c*64 + r)*cs_j of the segment, so 32 consecutive rows read 32 consecutive chunks.
-//   Inside a row's bytes, 32-bit word m holds 32/sw codes: with per = 16/sw, the code of element
-//   k = 2*(m*per + e) + h (h = 0,1) sits at bit 16*h + sw*e.  (One AND with a mask that has the
-//   same field in both 16-bit halves therefore yields the pair (k, k+1) as two 16-bit lanes.)
+//   Inside a row's bytes, 32-bit word m holds per = 32/sw codes: the code of element
+//   k = m*per + 4*u + i (u < 8/sw, i < 4) sits in byte B(i) = {0, 2, 1, 3}[i] at bit sw*u of that
+//   byte.  One AND with a mask that repeats the field at bit sw*u in all four bytes therefore yields
+//   the four codes of elements 4u..4u+3 as four 8-bit lanes (byte order k, k+2, k+1, k+3: the operand
+//   cell of the 8-bit MMA), and the same AND read as two 16-bit lanes yields the pair (k, k+1) from
+//   bytes 0 and 2, and the pair (k+2, k+3) from bytes 1 and 3 after a shift by 8.
 //
 // A call at width bits[kk] needs meta and segments 0..kk of a block: one contiguous prefix.
 // ------------------------------------------------------------------------------------------------
@@ -83,10 +86,11 @@ __host__ __device__ inline void d2moe_make_layout(PackLayout& L, const int* bits
 // Byte offset (inside a block) of the 32-bit word that holds element k of row r in segment j, and
 // the bit position of the element inside that word.
 __host__ __device__ inline int d2moe_elem_word(const PackLayout& L, int j, int r, int k, int* bitpos) {
-    int sw = L.seg_sw[j], per = 16 / sw;
-    int i = k >> 1, h = k & 1;
-    int m = i / per, e = i - m * per;
-    *bitpos = 16 * h + sw * e;
+    int sw = L.seg_sw[j], per = 32 / sw;
+    int m = k / per, ko = k - m * per;
+    int u = ko >> 2, i = ko & 3;
+    int byte = ((i & 1) << 1) | (i >> 1);       // element order inside a cell: bytes 0, 2, 1, 3
+    *bitpos = 8 * byte + sw * u;
     int ob = 4 * m, cs = L.seg_cs[j];
     int c = ob / cs, within = ob - c * cs;
     return L.seg_off[j] + (c * D2MOE_TILE_ROWS + r) * cs + within;

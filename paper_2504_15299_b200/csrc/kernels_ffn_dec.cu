@@ -134,8 +134,8 @@ __device__ __forceinline__ void dequant_half_tile(uint32_t seg, int rr, int h, c
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             const int idx = b * 16 + i, q = idx / PER, e = idx % PER;
-            const uint32_t src = e < NPOS ? w[q] : (w[q] >> 8);
-            v[i] = as_u32(__hfma2(as_h2(src & (FIELD << ((e % NPOS) * SW))), mult[e % NPOS], addend));
+            const uint32_t src = (e & 1) ? (w[q] >> 8) : w[q];   // pair e of the word: bytes (0,2) or (1,3), bit SW*(e/2)
+            v[i] = as_u32(__hfma2(as_h2(src & (FIELD << ((e >> 1) * SW))), mult[e >> 1], addend));
         }
         tc_st16(taddr + b * 16, v);
     }

@@ -102,10 +102,10 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, 
             const uint32_t lo8 = w[q], hi8 = w[q] >> 8;
 #pragma unroll
             for (int e = 0; e < PER; ++e) {
-                const uint32_t src = e < NPOS ? lo8 : hi8;
-                const __half2 code = as_h2(src & (FIELD << ((e % NPOS) * SW)));
+                const uint32_t src = (e & 1) ? hi8 : lo8;       // pair e of the word: bytes (0,2) or (1,3), bit SW*(e/2)
+                const __half2 code = as_h2(src & (FIELD << ((e >> 1) * SW)));
                 const int i = (l * WPL + q) * PER + e;
-                acc[i] = __hfma2(code, mult[e % NPOS], FIRST ? u0 : acc[i]);
+                acc[i] = __hfma2(code, mult[e >> 1], FIRST ? u0 : acc[i]);
             }
         }
     }

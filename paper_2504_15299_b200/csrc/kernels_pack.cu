@@ -81,7 +81,7 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
     __syncthreads();
 
     for (int j = 0; j < L.n_seg; ++j) {
-        const int sw = L.seg_sw[j], per = 16 / sw, cs = L.seg_cs[j];
+        const int sw = L.seg_sw[j], per = 32 / sw, cs = L.seg_cs[j];
         const int row_bytes = g * sw / 8;
         const int n_words = D2MOE_TILE_ROWS * row_bytes / 4;
         const unsigned mask = (1u << L.seg_w[j]) - 1u;
@@ -93,12 +93,12 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
             const int r = rem / cs, within = rem - r * cs;
             const int m = (c * cs + within) >> 2;
             uint32_t word = 0;
-            for (int e = 0; e < per; ++e)
-                for (int h = 0; h < 2; ++h) {
-                    const int k = 2 * (m * per + e) + h;
-                    const uint32_t v = (codes[r * g + k] >> L.seg_shift[j]) & mask;
-                    word |= v << (16 * h + sw * e);
-                }
+            for (int ko = 0; ko < per; ++ko) {         // element m*per + 4u + i: byte {0,2,1,3}[i], bit sw*u
+                const int u = ko >> 2, i = ko & 3;
+                const int byte = ((i & 1) << 1) | (i >> 1);
+                const uint32_t v = (codes[r * g + m * per + ko] >> L.seg_shift[j]) & mask;
+                word |= v << (8 * byte + sw * u);
+            }
             dst[wi] = word;
         }
     }
