@@ -28,8 +28,8 @@ METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of
-# this command (profiles/ffn_dec_kernel_mixtral_decode_T64.md); key = workload:tokens:stage:path
-NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 991534592, "mixtral_decode:T64:down:auto": 510644992}
+# this command (profiles/ffn_i8_kernel_mixtral_decode_T64.md); key = workload:tokens:stage:path
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1044381184, "mixtral_decode:T64:down:auto": 535324416}
 
 
 def measured_peaks():
@@ -419,7 +419,11 @@ def run_ours(args):
     # prefill-sized expert loads (the grouped dequant-GEMM) are bound by the tensor cores: report
     # the dominant kernel against the measured dense 16-bit matmul rate instead (fp16 operands have the
     # same nominal rate as the bf16 the peak was measured with; sustained figure: kernel inside a step)
-    if T * wl.top_k / wl.n_experts > 24:
+    # arithmetic type of the expert kernels: the decode kernel multiplies unsigned 8-bit codes with signed
+    # 8-bit activation halves (int32 accumulation, fp32 scaling), the grouped GEMM runs on fp16 tiles
+    dtype = "f32" if args.path == "cuda_core" else "i8"
+    if -(-T * wl.top_k // wl.n_experts) > 24 and args.path != "cuda_core":
+        dtype = "f16"
         A_tot = T * (wl.top_k + wl.n_shared)
         flops = {"gate_up": A_tot * 2 * 2 * wl.d_model * wl.d_ffn, "down": A_tot * 2 * wl.d_model * wl.d_ffn}
         tpeak, tkind = measured_tensor_peak()
@@ -441,7 +445,7 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": job_tokens_per_s(T, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype,
             "data": "synthetic", "config": workload_config(wl, T, args.path),
             "clocks": clocks,
             "e2e": {"value": job_tokens_per_s(T, world, e2e_ms), "unit": UNIT,

@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checks, workspace carving, launches.
 #include "d2moe_common.cuh"
+#include <cstdlib>
 #include "kernels_ffn_tc.cuh"
 
 #include <string.h>
@@ -135,8 +136,16 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
         ws->off_xp16 = take((size_t)pl.R_alloc * c->d_model * 2);
         ws->off_h = take((size_t)pl.R_alloc * c->d_ffn * 2);
         ws->off_o = take((size_t)pl.n_split * pl.R_alloc * c->d_model * 4);
+        ws->off_h32 = ws->off_xk_x = ws->off_xk_h = ws->off_slot_f = 0;
+        if (pl.decode) {
+            ws->off_h32 = take((size_t)pl.R_alloc * c->d_ffn * 4);
+            ws->off_xk_x = take((size_t)(c->d_model / c->group_size) * pl.R_alloc * 8);
+            ws->off_xk_h = take((size_t)(c->d_ffn / c->group_size) * pl.R_alloc * 8);
+            ws->off_slot_f = take((size_t)3 * pl.R_alloc * 4);
+        }
     } else {
         ws->off_units = ws->off_n_units = ws->off_pad_off = ws->off_row_map = ws->off_src_token = ws->off_xp16 = 0;
+        ws->off_h32 = ws->off_xk_x = ws->off_xk_h = ws->off_slot_f = 0;
         ws->off_h = take(A_tot * (size_t)c->d_ffn * 4);
         ws->off_o = take(A_tot * (size_t)c->d_model * 4);
     }
@@ -262,7 +271,9 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
         B.pad_off = (int32_t*)(w + ws.off_pad_off); B.row_map = (int32_t*)(w + ws.off_row_map);
         B.src_token = (int32_t*)(w + ws.off_src_token);
         B.xp16 = (__half*)(w + ws.off_xp16); B.h16 = (__half*)(w + ws.off_h); B.o32 = (float*)(w + ws.off_o);
-        e = pl.decode ? launch_ffn_decode(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev)
+        B.h32 = (float*)(w + ws.off_h32); B.xk_x = (float*)(w + ws.off_xk_x); B.xk_h = (float*)(w + ws.off_xk_h);
+        B.slot_f = (float*)(w + ws.off_slot_f);
+        e = pl.decode ? launch_ffn_i8(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev)
                       : launch_ffn_tensor(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev);
         if (e != cudaSuccess) return D2MOE_ERR_CUDA;
         mark(3);
@@ -309,7 +320,12 @@ extern "C" d2moe_status d2moe_moe_forward_events(const d2moe_config* c, int64_t 
 extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int routing_precomputed) {
     if (d2moe_check_config(c) != D2MOE_OK || T <= 0) return 0;
     const int route = routing_precomputed ? 0 : 4;     // route, count, scan, scatter
-    if (use_tensor_path(c)) return route + 5;           // unit build, gather, gate/up, down, combine
+    if (use_tensor_path(c)) {
+        TcPlan pl;
+        tc_plan(c, T, &pl);
+        // unit build, gather (decode: quantise x), gate/up, (decode: quantise h), down, combine
+        return route + (pl.decode ? 6 : 5);
+    }
     return route + 3;                                   // gate/up, down, combine
 }
 

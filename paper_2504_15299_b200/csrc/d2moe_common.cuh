@@ -127,6 +127,7 @@ struct Workspace {
     size_t off_topk_idx, off_topk_w, off_bit_idx, off_perm, off_inv_perm, off_group_off;
     size_t off_h, off_o, off_status;
     size_t off_units, off_n_units, off_pad_off, off_row_map, off_src_token, off_xp16;   // tensor-core path
+    size_t off_h32, off_xk_x, off_xk_h, off_slot_f;                                     // 8-bit decode kernel
 };
 
 void d2moe_carve_workspace(const d2moe_config* cfg, long long max_tokens, Workspace* ws);

@@ -1,0 +1,892 @@
+// Memory-bound expert kernel for decode-sized loads: 8-bit tensor-core products on the packed codes
+// themselves, scales applied to the accumulators (tcgen05 kind::i8 + TMEM).
+//
+// The reconstruction rule of Section 3.3.1 in closed form, for a token routed at width b (index kk),
+//     W_hat_b[r, k] = lo + s1 * ( Q_b[r, k] * 2^-(top - b1) + 2^-(b - b1 + 1) - 1/2 ),
+// where Q_b is the nested top-width code with the bits below width b cleared (the sum of the
+// segments 0..kk, each at its position inside the top-width code), (s1, lo) belong to (row, group)
+// and b1 / top are the narrowest / widest width.  With the activations of a token written as
+// x[k] = sigma * xq[k] (xq a 15-bit integer, sigma per token), one output element is
+//     y[r] = sigma * sum_G { s1' * ( sum_{k in G} Q_b[r, k] xq[k]  +  kappa_b X_G )  +  lo * X_G },
+//     s1' = s1 * 2^-(top - b1),  kappa_b = 2^(top - b - 1) - 2^(top - b1 - 1),  X_G = sum_{k in G} xq[k].
+// The inner sum is an exact integer contraction: the tensor cores run it on unsigned 8-bit codes
+// and signed 8-bit activation halves (xq = 128 hi + lo8), so the CUDA cores never expand a code to
+// a floating-point weight.  What is left for them per packed word is one shift and one AND per four
+// codes (the packed layout keeps the four codes of an operand cell in the four bytes of a word), and
+// per (row, group, token) five instructions that fold the accumulator into the running output.
+//
+//   * The tokens of a unit are laid out by width, widest first, each width class padded to 8 slots:
+//     the slots that include segment j are the first npad[j] of the unit, and the product of
+//     segment j runs over exactly those (N = 2 npad[j]: a high and a low activation row per slot).
+//     All segments of a group accumulate into ONE accumulator, each at its position in the code.
+//   * Every segment plane is read from HBM once per (unit, row tile) whatever the mix of widths
+//     (the plane reuse of Section 3.4), through a ring of bulk async copies; a unit whose widest
+//     token is narrower than the top width reads only the prefix it needs.
+//   * The accumulator is double buffered per group: while the products of group G+1 run, the
+//     dequant threads fold group G into fp32 registers.
+//
+// CTA = 320 threads, 2 CTAs per SM (96 registers per thread).  Warps 0-3 and 4-7 are two warpgroups (thread = weight row =
+// TMEM lane): warpgroup w unpacks the segments w, w+2, ... of every group into two alternating
+// 32-column operand slots in TMEM and folds half of the unit's token blocks; warp 8 streams packed
+// blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and the per-group activation sums,
+// warp 9 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns + 4 x 32
+// operand columns.  Every wait is bounded; on expiry the CTA raises D2MOE_DEV_TIMEOUT, stops
+// waiting, drains its copies, frees its TMEM and exits.
+#include "d2moe_common.cuh"
+#include "kernels_ffn_tc.cuh"
+#include "tc_common.cuh"
+
+#include <type_traits>
+
+namespace {
+
+constexpr int I8_THREADS = 320;
+constexpr int I8_WARP_PROD = 8, I8_WARP_MMA = 9;
+constexpr int I8_TMEM_COLS = 256;
+constexpr int I8_D_COLS = 64;                 // one accumulator buffer: 32 slots x (high, low)
+constexpr int I8_SLOTS = 32;                  // token slots per unit
+constexpr int I8_NSB = 4;                     // activation ring depth
+constexpr int I8_MAX_NSW = 8;                 // weight ring depth (upper bound)
+constexpr int I8_B_TILE = 2 * I8_SLOTS * 128; // 64 rows x 128 bytes (128 input columns)
+constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa X) per slot, one group
+constexpr int I8_B_STAGE = I8_B_TILE + 2 * I8_XK_BYTES;
+constexpr int I8_EPI_STRIDE = 17;
+constexpr float I8_XMAX = 16191.0f;           // |xq| <= 126 * 128 + 63
+
+struct I8Params {
+    MoeDims D;
+    PackLayout L;
+    ExpertPtrs P;
+    int mode;                 // 0: gate/up + SwiGLU -> hbuf;  1: down -> obuf
+    int n_row_tiles, n_split, groups_per_split, nsw;
+    const I8Unit* units;
+    const int* n_units;
+    const float* xk;          // [n_groups][R_alloc][2]
+    const float* sigma;       // [R_alloc]
+    float* hbuf;              // [R_alloc, F]
+    float* obuf;              // [n_split][R_alloc, d]
+    long long R_alloc;
+    int32_t* status;
+    int smem_w_off, smem_epi_off, smem_bar_off;
+    int dbg;                  // debug builds only: bit 0 skips the MMAs, bit 1 the unpack math, bit 2 the fold math
+};
+
+struct I8Item { int unit, tile, split, g0, g1; };
+
+#if defined(D2MOE_WAIT_STATS) || defined(D2MOE_I8_DBG)
+#define I8_SKIP(bit) if (!(p.dbg & bit))      // debug builds only: leave out part of the work
+#define I8_STREAM_ONLY (p.dbg & 8)            // debug builds only: stream the rings, do nothing else
+#else
+#define I8_SKIP(bit)
+#define I8_STREAM_ONLY false
+#endif
+
+#ifdef D2MOE_WAIT_STATS
+// Debug build only: cycles per wait category, summed over all CTAs.  0 wprod.w_empty 1 bprod.b_empty
+// 2 mma.d_empty 3 mma.b_full 4 mma.a_full 5 mma.total 6 deq.w_full 7 deq.a_empty 8 deq.wait_st
+// 9 deq.d_full 10 deq.total 11 deq.fold 12 deq.unpack 13 groups 14 deq.output
+__device__ unsigned long long g_i8_stats[16];
+#define I8S_T0() const long long _t0 = clock64()
+#define I8S_ADD(slot) stat[slot] += clock64() - _t0
+#define I8S_DECL() long long stat[16] = {0}
+#define I8S_FLUSH(cond) do { if (cond) { for (int _i = 0; _i < 16; ++_i) if (stat[_i]) atomicAdd(&g_i8_stats[_i], (unsigned long long)stat[_i]); } } while (0)
+#else
+#define I8S_T0()
+#define I8S_ADD(slot)
+#define I8S_DECL()
+#define I8S_FLUSH(cond)
+#endif
+
+__device__ __forceinline__ I8Item i8_item(const I8Params& p, int item) {
+    I8Item it;
+    const int per_unit = p.n_row_tiles * p.n_split;
+    it.unit = item / per_unit;
+    const int rem = item - it.unit * per_unit;
+    it.tile = rem / p.n_split;
+    it.split = rem - it.tile * p.n_split;
+    it.g0 = it.split * p.groups_per_split;
+    it.g1 = min(p.L.n_groups, it.g0 + p.groups_per_split);
+    return it;
+}
+
+// unsigned 8-bit x signed 8-bit -> int32, A and B K-major, M = 128
+__device__ __forceinline__ uint32_t instr_desc_i8(int n) {
+    return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+}
+
+// The GS codes of one segment of one row -> GS/4 operand cells (four unsigned bytes each, the code
+// moved to bit P of its byte = its position inside the top-width code), written to TMEM columns
+// [taddr, taddr + GS/4).  SW: storage width, W: logical width (W <= SW).
+template <int GS, int SW>
+__device__ __forceinline__ void unpack_segment(uint32_t seg, int rr, int W, int P, uint32_t taddr) {
+    constexpr int ROW_BYTES = GS * SW / 8;
+    constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;      // chunk size of the packed layout
+    constexpr int NLD = ROW_BYTES / CS;
+    constexpr int WPL = CS / 4;                              // words per load
+    constexpr int CPW = 8 / SW;                              // cells per word
+    constexpr int NCELL = GS / 4;
+    const uint32_t mask = (((1u << W) - 1u) << P) * 0x01010101u;
+
+    constexpr int NB = NCELL / 16;                           // batches of 16 cells = one tcgen05.st
+    constexpr int WPB = 16 / CPW;                            // words per batch: 8, 4, 2 for SW = 4, 2, 1 (16 for 8)
+    constexpr int NW = NLD * WPL;
+    // words are loaded batch by batch when a batch spans whole loads, otherwise once for all batches
+    constexpr bool PER_BATCH = WPB >= WPL;
+    uint32_t w[PER_BATCH ? WPB : NW];
+    auto load = [&](int l, uint32_t* dst) {
+        const uint32_t addr = seg + (uint32_t)((l * D2MOE_TILE_ROWS + rr) * CS);
+        if constexpr (WPL == 4) {
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(dst[0]), "=r"(dst[1]), "=r"(dst[2]), "=r"(dst[3]) : "r"(addr));
+        } else if constexpr (WPL == 2) {
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(dst[0]), "=r"(dst[1]) : "r"(addr));
+        } else {
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(dst[0]) : "r"(addr));
+        }
+    };
+    if constexpr (!PER_BATCH) {
+#pragma unroll
+        for (int l = 0; l < NLD; ++l) load(l, w + l * WPL);
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        if constexpr (PER_BATCH) {
+#pragma unroll
+            for (int l = 0; l < WPB / WPL; ++l) load(b * (WPB / WPL) + l, w + l * WPL);
+        }
+        uint32_t v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int cell = b * 16 + i, q = PER_BATCH ? i / CPW : cell / CPW, u = cell % CPW;
+            const int sh = P - SW * u;                       // compile-time sign when P is a constant
+            const uint32_t moved = sh >= 0 ? (w[q] << (sh & 31)) : (w[q] >> ((-sh) & 31));
+            v[i] = moved & mask;
+        }
+        tc_st16(taddr + b * 16, v);
+    }
+}
+
+template <int GS>
+__device__ __forceinline__ void unpack_dispatch(int sw, uint32_t seg, int rr, int W, int P, uint32_t taddr) {
+    switch (sw) {
+        case 1: unpack_segment<GS, 1>(seg, rr, W, P, taddr); break;
+        case 2: unpack_segment<GS, 2>(seg, rr, W, P, taddr); break;
+        case 4: unpack_segment<GS, 4>(seg, rr, W, P, taddr); break;
+        default: unpack_segment<GS, 8>(seg, rr, W, P, taddr); break;
+    }
+}
+
+// Compile-time description of a width list whose segments are stored exactly (widths 1, 2, 4, 8):
+// nibble j of SWPACK is the width of segment j.  SWPACK == 0 selects the run-time path.
+template <int SWPACK>
+struct I8SegList {
+    __host__ __device__ static constexpr int sw(int j) { return (SWPACK >> (4 * j)) & 15; }
+    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && sw(k) != 0) ++k; return k; }
+    __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += sw(i); return b; }
+    __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += sw(i); return top() - b; }
+    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
+};
+
+// Output phase of one work item for one thread: scales the folded sums by the tokens' activation
+// scales, applies SwiGLU across the gate / up halves of the tile (mode 0) and writes the result.
+// blks: byte i = first slot / 4 of the thread's block i.
+static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, int wg, int r, int n_mine, uint32_t blks,
+                                                 float (&acc)[4][4], float* epi) {
+    const I8Item io = i8_item(p, item);
+    const int slot0 = p.units[io.unit].slot0;
+    const int blk = r >> 6, rr = r & 63;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (i < n_mine) {
+            const float4 sg = *reinterpret_cast<const float4*>(p.sigma + slot0 + 4 * ((blks >> (8 * i)) & 255u));
+            acc[i][0] *= sg.x; acc[i][1] *= sg.y; acc[i][2] *= sg.z; acc[i][3] *= sg.w;
+        }
+    }
+    if (p.mode == 0) {
+        if (blk == 1) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < n_mine)
+#pragma unroll
+                    for (int s = 0; s < 4; ++s) epi[rr * I8_EPI_STRIDE + 4 * i + s] = acc[i][s];
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+        if (blk == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (i < n_mine) {
+                    float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io.tile * 64 + rr;
+#pragma unroll
+                    for (int s = 0; s < 4; ++s) {
+                        const float g = acc[i][s];
+                        const float up = epi[rr * I8_EPI_STRIDE + 4 * i + s];
+                        dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
+                    }
+                }
+            }
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < n_mine) {
+                float* dst = p.obuf + (long long)io.split * p.R_alloc * p.D.d
+                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io.tile * 128 + r;
+#pragma unroll
+                for (int s = 0; s < 4; ++s) dst[(long long)s * p.D.d] = acc[i][s];
+            }
+        }
+    }
+}
+
+template <int GS, int SWPACK>
+__global__ void __launch_bounds__(I8_THREADS, 2)
+ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMaps maps) {
+    constexpr int GPS = 128 / GS;              // groups per ring stage (a stage spans 128 input columns)
+    constexpr int KSTEPS = GS / 32;            // MMAs (K = 32) per segment and group
+    extern __shared__ uint8_t smem_raw[];
+    // shared layout from a 1024-byte boundary:
+    // [activation tiles: I8_NSB x 8 KiB] [activation sums: I8_NSB x 512 B] [weight ring: nsw x GPS x 2 blocks] [epilogue x2] [barriers]
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t w_slot_bytes = (uint32_t)(GPS * 2) * (uint32_t)p.L.block_bytes;
+    const uint32_t bbuf = smem_base;
+    const uint32_t xkbuf = smem_base + I8_NSB * I8_B_TILE;   // per stage: 2 x (X, kappa X) of 32 slots
+    const uint32_t wbuf = smem_base + p.smem_w_off;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.smem_bar_off);
+    const uint32_t bar0 = smem_u32(bars);
+    auto W_FULL = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    auto W_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(I8_MAX_NSW + i); };
+    auto B_FULL = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + i); };
+    auto B_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + I8_NSB + i); };
+    auto A_FULL = [&](int wg, int sl) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + wg * 2 + sl); };
+    auto A_EMPTY = [&](int wg, int sl) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 4 + wg * 2 + sl); };
+    auto D_FULL = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 8 + b); };
+    auto D_EMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 10 + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * I8_MAX_NSW + 2 * I8_NSB + 12);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t abort_addr = smem_u32(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 256); }
+        // an activation stage is released by the MMA issuer (its products have read the tile) and by
+        // the eight folding warps (they have read the sums)
+        for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 9); }
+        for (int wg = 0; wg < 2; ++wg)
+            for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == I8_WARP_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(I8_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t d_tmem = tmem_base;                         // buffer b: columns [64 b, 64 b + 64)
+    const uint32_t a_tmem = tmem_base + 2 * I8_D_COLS;         // warpgroup wg, slot sl: + (wg*2 + sl)*32
+
+    const int n_units = *p.n_units;
+    const int total_items = n_units * p.n_row_tiles * p.n_split;
+    const int nsw = p.nsw;
+
+    if (warp == I8_WARP_PROD) {
+        // One producer thread feeds both rings, stage by stage (they are consumed at the same rate).
+        if (lane == 0) {
+            I8S_DECL();
+            uint32_t it = 0;
+            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+                const I8Item ii = i8_item(p, item);
+                const I8Unit* u = p.units + ii.unit;
+                const int e = u->e, kmax = u->kmax;
+                const uint32_t bytes = (uint32_t)p.L.seg_off[kmax + 1];
+                const uint8_t *m0, *m1;
+                int rt0, rt1;
+                if (p.mode == 0) { m0 = p.P.w[3 * e + 0]; m1 = p.P.w[3 * e + 1]; rt0 = rt1 = ii.tile; }
+                else { m0 = m1 = p.P.w[3 * e + 2]; rt0 = 2 * ii.tile; rt1 = 2 * ii.tile + 1; }
+                const int nslots = u->nslots, slot0 = u->slot0;
+                const int mi = nslots <= 8 ? 0 : (nslots <= 16 ? 1 : 2);        // boxes of 16, 32, 64 rows
+                const uint32_t tile_bytes = (16u << mi) * 128u;
+                const uint32_t xk_bytes = (uint32_t)nslots * 8u;
+                for (int G = ii.g0; G < ii.g1; G += GPS, ++it) {
+                    const int ng = min(GPS, ii.g1 - G);
+                    {
+                        const int s = it % nsw;
+                        { I8S_T0(); mbar_wait_ptx(W_EMPTY(s), ((it / nsw) & 1) ^ 1, abort_addr, p.status); I8S_ADD(0); }
+                        mbar_expect_tx(W_FULL(s), 2 * bytes * ng);
+                        const uint32_t dst = wbuf + s * w_slot_bytes;
+                        for (int sub = 0; sub < ng; ++sub) {
+                            bulk_g2s(dst + (2 * sub) * p.L.block_bytes, m0 + d2moe_block_offset(p.L, rt0, G + sub), bytes, W_FULL(s));
+                            bulk_g2s(dst + (2 * sub + 1) * p.L.block_bytes, m1 + d2moe_block_offset(p.L, rt1, G + sub), bytes, W_FULL(s));
+                        }
+                    }
+                    {
+                        const int s = it % I8_NSB;
+                        { I8S_T0(); mbar_wait_ptx(B_EMPTY(s), ((it / I8_NSB) & 1) ^ 1, abort_addr, p.status); I8S_ADD(1); }
+                        mbar_expect_tx(B_FULL(s), tile_bytes + ng * xk_bytes);
+                        tma_load_2d(bbuf + s * I8_B_TILE, &maps.m[mi], G * GS, 2 * slot0, B_FULL(s));
+                        for (int sub = 0; sub < ng; ++sub)
+                            bulk_g2s(xkbuf + (2 * s + sub) * I8_XK_BYTES,
+                                     p.xk + ((long long)(G + sub) * p.R_alloc + slot0) * 2, xk_bytes, B_FULL(s));
+                    }
+                }
+            }
+            for (int s = 0; s < nsw && s < (int)it; ++s) {      // drain: all copies issued have landed
+                const uint32_t last = it - 1 - (it - 1 - s) % nsw;
+                mbar_wait(W_FULL(s), (last / nsw) & 1, abort_flag, p.status, true);
+            }
+            for (int s = 0; s < I8_NSB && s < (int)it; ++s) {
+                const uint32_t last = it - 1 - (it - 1 - s) % I8_NSB;
+                mbar_wait(B_FULL(s), (last / I8_NSB) & 1, abort_flag, p.status, true);
+            }
+            I8S_FLUSH(true);
+        }
+    } else if (warp == I8_WARP_MMA) {
+        // One issuer: all segments of a group accumulate into the same columns, so their products
+        // must be issued in order.  The whole warp runs the loop and one elected lane issues, so that
+        // addresses and descriptors stay in the uniform datapath.  A warpgroup hands over up to two
+        // operand tiles at a time (its segments j and j + 2).
+        uint32_t gc = 0, bs = 0, bph = 0, hs[2] = {0, 0};
+        I8S_DECL();
+#ifdef D2MOE_WAIT_STATS
+        const long long _tt = clock64();
+#endif
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+            const I8Item ii = i8_item(p, item);
+            const I8Unit* u = p.units + ii.unit;
+            const int kmax = u->kmax;
+            uint32_t idesc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) idesc[j] = instr_desc_i8(2 * max(u->npad[j], 8));
+            for (int G = ii.g0; G < ii.g1; G += GPS) {
+                const int ng = min(GPS, ii.g1 - G);
+                { I8S_T0(); mbar_wait_ptx(B_FULL(bs), bph, abort_addr, p.status); I8S_ADD(3); }
+                const uint64_t bdesc = smem_desc_sw128(bbuf + bs * I8_B_TILE);
+#pragma unroll
+                for (int sub = 0; sub < GPS; ++sub) {
+                    if (sub < ng && !I8_STREAM_ONLY) {
+                        const int buf = gc & 1;
+                        { I8S_T0(); mbar_wait_ptx(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1, abort_addr, p.status); I8S_ADD(2); }
+                        tc_fence_after();
+                        const uint32_t d_addr = d_tmem + buf * I8_D_COLS;
+#pragma unroll
+                        for (int hp = 0; hp < (SWPACK != 0 ? 1 : 2); ++hp) {
+#pragma unroll
+                            for (int wg = 0; wg < 2; ++wg) {
+                                const int j0 = wg + 4 * hp, j1 = j0 + 2;
+                                if (j0 <= kmax) {
+                                    { I8S_T0(); mbar_wait_ptx(A_FULL(wg, 0), hs[wg] & 1, abort_addr, p.status); I8S_ADD(4); }
+                                    tc_fence_after();
+                                    const uint32_t a_addr = a_tmem + wg * 64;
+                                    if (elect_one()) {
+                                        I8_SKIP(1)
+                                        {
+#pragma unroll
+                                            for (int ks = 0; ks < KSTEPS; ++ks)
+                                                tc_mma_i8_ts(d_addr, a_addr + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
+                                                             idesc[j0], (j0 == 0 && ks == 0) ? 0u : 1u);
+                                            if (j1 <= kmax) {
+#pragma unroll
+                                                for (int ks = 0; ks < KSTEPS; ++ks)
+                                                    tc_mma_i8_ts(d_addr, a_addr + 32 + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
+                                                                 idesc[j1 & 7], 1u);
+                                            }
+                                        }
+                                        tc_commit(A_EMPTY(wg, 0));
+                                    }
+                                    __syncwarp();
+                                    ++hs[wg];
+                                }
+                            }
+                        }
+                        if (elect_one()) tc_commit(D_FULL(buf));
+                        __syncwarp();
+                        ++gc;
+                    }
+                }
+                if (elect_one()) tc_commit(B_EMPTY(bs));
+                __syncwarp();
+                if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
+            }
+        }
+        // all products have completed before TMEM is released
+        if (gc > 0) mbar_wait(D_FULL((gc - 1) & 1), ((gc - 1) >> 1) & 1, abort_flag, p.status, true);
+        if (gc > 1) mbar_wait(D_FULL((gc - 2) & 1), ((gc - 2) >> 1) & 1, abort_flag, p.status, true);
+#ifdef D2MOE_WAIT_STATS
+        stat[5] = clock64() - _tt;
+#endif
+        I8S_FLUSH(lane == 0);
+    } else if (warp < 8) {
+        // -------- two warpgroups: unpack (segments wg, wg+2, ... of every group), fold, write out --------
+        const int wg = warp >> 2;
+        const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
+        const int blk = r >> 6, rr = r & 63;
+        const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
+        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
+        const uint32_t a_base = a_tmem + wg * 64 + lane_addr;          // my two operand tiles: +0, +32
+        const uint32_t d_base = d_tmem + lane_addr;
+        const uint32_t AF = A_FULL(wg, 0), AE = A_EMPTY(wg, 0);
+        const uint32_t w_addr0 = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
+        uint32_t gc = 0, hs = 0;                   // groups folded / operand hand-offs so far
+        uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
+        uint32_t w_addr = w_addr0;
+        I8S_DECL();
+#ifdef D2MOE_WAIT_STATS
+        const long long _tt = clock64();
+#endif
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+            const I8Item ii = i8_item(p, item);
+            const I8Unit* u = p.units + ii.unit;
+            const int kmax = u->kmax, nblk = u->nblk;
+            const int h0 = (nblk + 1) >> 1;
+            const int n_mine = wg == 0 ? h0 : nblk - h0;        // my token blocks (at most 4)
+            uint32_t myblks = 0;                                 // byte i: first slot / 4 of my block i
+#pragma unroll
+            for (int i = 0; i < 4; ++i) myblks |= (uint32_t)u->blk[min((wg == 0 ? 0 : h0) + i, 7)] << (8 * i);
+#define MYBLK(i) ((myblks >> (8 * (i))) & 255u)
+            float acc[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int s = 0; s < 4; ++s) acc[i][s] = 0.0f;
+
+            // fold the group whose accumulator is buffer `buf` into acc; pb: ring position of its sums
+            // (bits 0-1), phase (bit 2), last group of its stage (bit 3), group inside the stage (bit 4)
+            auto fold = [&](uint32_t g, uint32_t pb, uint32_t meta) {
+                const int buf = g & 1;
+                { I8S_T0(); mbar_wait_ptx(D_FULL(buf), (g >> 1) & 1, abort_addr, p.status); I8S_ADD(9); }
+                tc_fence_after();
+                I8S_T0();
+                const __half2 mh = as_h2(meta);
+                const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
+                const float lo = __high2float(mh);
+                mbar_wait_ptx(B_FULL(pb & 3), (pb >> 2) & 1, abort_addr, p.status);
+                const uint32_t xk_addr = xkbuf + ((pb & 3) * 2 + (pb >> 4)) * I8_XK_BYTES;
+                // two rounds of two blocks: 16 accumulator registers in flight instead of 32
+#pragma unroll
+                for (int rd = 0; rd < 2; ++rd) {
+                    uint32_t v[2][8];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+                        if (2 * rd + i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(2 * rd + i), v[i]);
+                    tc_wait_ld();
+                    if (rd == 1) { tc_fence_before(); mbar_arrive(D_EMPTY(buf)); }
+                    I8_SKIP(4)
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        if (2 * rd + i < n_mine) {
+                            float xk[8];
+                            const uint32_t a = xk_addr + 32u * MYBLK(2 * rd + i);
+                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
+                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
+#pragma unroll
+                            for (int s = 0; s < 4; ++s) {
+                                const int di = (int)v[i][2 * s] * 128 + (int)v[i][2 * s + 1];
+                                const float t = (float)di + xk[2 * s + 1];
+                                acc[2 * rd + i][s] = fmaf(s1p, t, acc[2 * rd + i][s]);
+                                acc[2 * rd + i][s] = fmaf(lo, xk[2 * s], acc[2 * rd + i][s]);
+                            }
+                        }
+                    }
+                }
+                if (pb & 8) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(B_EMPTY(pb & 3));
+                }
+                I8S_ADD(11);
+            };
+
+            bool pend = false;
+            uint32_t pend_pb = 0, pend_meta = 0;
+            for (int G = ii.g0; G < ii.g1; G += GPS) {
+                const int ng = min(GPS, ii.g1 - G);
+                { I8S_T0(); mbar_wait_ptx(W_FULL(ws), wph, abort_addr, p.status); I8S_ADD(6); }
+                if (I8_STREAM_ONLY) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(B_EMPTY(bs));
+                }
+#pragma unroll
+                for (int sub = 0; sub < GPS; ++sub) {
+                    if (sub < ng && !I8_STREAM_ONLY) {
+                        const uint32_t wb = w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes;
+                        uint32_t meta;
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
+                        auto handoff_begin = [&]() {
+                            { I8S_T0(); mbar_wait_ptx(AE, (hs & 1) ^ 1, abort_addr, p.status); I8S_ADD(7); }
+                            tc_fence_after();
+                        };
+                        auto handoff_end = [&]() {
+                            { I8S_T0(); tc_wait_st(); I8S_ADD(8); }
+                            tc_fence_before();
+                            mbar_arrive(AF);
+                            ++hs;
+                        };
+                        if constexpr (SWPACK != 0) {
+                            using SL = I8SegList<SWPACK>;
+                            auto do_seg = [&](auto jc) {
+                                constexpr int J = decltype(jc)::value;
+                                if constexpr (J < SL::count()) {
+                                    if ((J & 1) == wg && J <= kmax) {
+                                        I8_SKIP(2)
+                                        unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::sw(J), SL::pos(J),
+                                                                      a_base + (J >> 1) * 32);
+                                    }
+                                }
+                            };
+                            if (wg <= kmax) {
+                                handoff_begin();
+                                I8S_T0();
+                                do_seg(std::integral_constant<int, 0>{});
+                                do_seg(std::integral_constant<int, 1>{});
+                                do_seg(std::integral_constant<int, 2>{});
+                                do_seg(std::integral_constant<int, 3>{});
+                                I8S_ADD(12);
+                                handoff_end();
+                            }
+                        } else {
+#pragma unroll 1
+                            for (int j = wg; j <= kmax; j += 4) {
+                                handoff_begin();
+                                unpack_dispatch<GS>(p.L.seg_sw[j], wb + (uint32_t)p.L.seg_off[j], rr, p.L.seg_w[j], p.L.seg_shift[j], a_base);
+                                if (j + 2 <= kmax)
+                                    unpack_dispatch<GS>(p.L.seg_sw[j + 2], wb + (uint32_t)p.L.seg_off[j + 2], rr, p.L.seg_w[j + 2],
+                                                        p.L.seg_shift[j + 2], a_base + 32);
+                                handoff_end();
+                            }
+                        }
+                        if (pend) fold(gc - 1, pend_pb, pend_meta);
+                        pend = true;
+                        pend_meta = meta;
+                        pend_pb = bs | (bph << 2) | (sub == ng - 1 ? 8u : 0u) | ((uint32_t)sub << 4);
+                        ++gc;
+#ifdef D2MOE_WAIT_STATS
+                        stat[13] += 1;
+#endif
+                    }
+                }
+                mbar_arrive(W_EMPTY(ws));
+                w_addr += w_slot_bytes;
+                if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = w_addr0; }
+                if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
+            }
+            if (pend) fold(gc - 1, pend_pb, pend_meta);
+
+            // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
+            I8S_T0();
+            float out[4][4];                   // a copy: acc itself must stay in registers
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) out[i][q] = acc[i][q];
+            i8_write_out(p, item, wg, r, n_mine, myblks, out, epi);
+            I8S_ADD(14);
+        }
+#ifdef D2MOE_WAIT_STATS
+        stat[10] = clock64() - _tt;
+#endif
+        I8S_FLUSH((threadIdx.x & 127) == 0);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == I8_WARP_MMA) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(I8_TMEM_COLS) : "memory");
+    }
+}
+
+__device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
+
+// One block.  Lays every expert's tokens out by width, widest first, each width class padded to a
+// multiple of 8 slots; cuts every expert into units of 32 slots; records per unit and segment how many
+// of its slots include the segment, and which blocks of 4 slots hold real tokens.
+__global__ void __launch_bounds__(256)
+i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
+               int32_t* src_token, float* kappa, int max_units, int top, int b1) {
+    __shared__ int s_total;
+    const int n_exp = D.E + D.n_shared;
+    if (threadIdx.x < 32) {                       // padded expert offsets (one warp scans)
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int base = 0; base < n_exp; base += 32) {
+            const int e = base + lane;
+            int v = 0;
+            if (e < D.E) {
+                for (int j = 0; j < D.K; ++j) v += round8(R.group_off[e * D.K + j + 1] - R.group_off[e * D.K + j]);
+            } else if (e < n_exp) {
+                v = round8(D.T);
+            }
+            int incl = v;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (e < n_exp) pad_off[e] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) { pad_off[n_exp] = carry; s_total = carry; }
+    }
+    __syncthreads();
+    const int total = s_total;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) { src_token[i] = -1; kappa[i] = 0.0f; }
+    __syncthreads();
+    for (int a = threadIdx.x; a < D.A; a += blockDim.x) {
+        const int pos = R.inv_perm[a];
+        const int e = R.topk_idx[a], kk = R.bit_idx[a];
+        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) { row_map[a] = 0; continue; }
+        int start = 0;                            // classes of a larger width index come first
+        for (int i = kk + 1; i < D.K; ++i) start += round8(R.group_off[e * D.K + i + 1] - R.group_off[e * D.K + i]);
+        const int slot = pad_off[e] + start + (pos - R.group_off[e * D.K + kk]);
+        row_map[a] = slot;
+        if (slot >= 0 && slot < total) {
+            src_token[slot] = a / D.k;
+            kappa[slot] = exp2f((float)(top - D.bits[kk] - 1)) - exp2f((float)(top - b1 - 1));
+        }
+    }
+    for (int i = threadIdx.x; i < D.n_shared * D.T; i += blockDim.x) {
+        const int s = i / D.T, t = i - s * D.T;
+        const int slot = pad_off[D.E + s] + t;
+        row_map[D.A + i] = slot;
+        src_token[slot] = t;
+        kappa[slot] = 0.5f - exp2f((float)(top - b1 - 1));
+    }
+    if (threadIdx.x == 0) {
+        int nu = 0;
+        for (int e = 0; e < n_exp; ++e) {
+            const int p0 = pad_off[e], len_e = pad_off[e + 1] - p0;
+            int cnt[8], cpad[9];                  // cpad[j]: padded slots of the classes with index >= j
+            cpad[D.K] = 0;
+            for (int j = D.K - 1; j >= 0; --j) {
+                cnt[j] = e < D.E ? R.group_off[e * D.K + j + 1] - R.group_off[e * D.K + j] : (j == D.K - 1 ? D.T : 0);
+                cpad[j] = cpad[j + 1] + round8(cnt[j]);
+            }
+            for (int start = 0; start < len_e && nu < max_units; start += I8_SLOTS) {
+                const int len = min(len_e - start, I8_SLOTS);
+                I8Unit u;
+                u.e = e; u.slot0 = p0 + start; u.nslots = len; u.kmax = 0; u.nblk = 0;
+                for (int j = 0; j < 8; ++j) {
+                    u.blk[j] = 0;
+                    u.npad[j] = j < D.K ? max(0, min(len, cpad[j] - start)) : 0;
+                    if (u.npad[j] > 0) u.kmax = j;
+                }
+                for (int j = D.K - 1; j >= 0; --j) {          // real slots of class j: [cpad[j+1], cpad[j+1] + cnt[j])
+                    const int a0 = max(cpad[j + 1], start), a1 = min(cpad[j + 1] + cnt[j], start + len);
+                    for (int b = a0 / 4; 4 * b < a1; ++b)
+                        if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
+                }
+                if (u.nblk > 0) units[nu++] = u;
+            }
+        }
+        *n_units = nu;
+    }
+}
+
+// Quantises one activation row per slot to 15-bit integers xq = rint(x / sigma), sigma = max|x| / 16191,
+// stored as two signed bytes per element (xq = 128 hi + lo8, lo8 in [-64, 63]) in rows 2 slot and
+// 2 slot + 1 of q, in the byte order of the operand cells (elements k, k+2, k+1, k+3), and writes
+// per group the integer sum X of the row's xq and kappa * X.  GATHER: the row of slot s is
+// x[src_token[s]] (bf16); otherwise it is row s of an fp32 buffer.  Padding slots become zeros.
+template <bool GATHER>
+__global__ void __launch_bounds__(256)
+i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, const int32_t* __restrict__ src_token,
+                const int32_t* __restrict__ pad_off, int n_off, const float* __restrict__ kappa,
+                int8_t* __restrict__ q, float* __restrict__ xk, float* __restrict__ sigma) {
+    __shared__ float s_red[8];
+    const int total = pad_off[n_off];
+    const int n_cells = n / 4, cpg = g / 4;                 // cells per group: 16 or 32
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int slot = blockIdx.x; slot < total; slot += gridDim.x) {
+        const int t = src_token[slot];
+        uint32_t* qh = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot) * n);
+        uint32_t* ql = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot + 1) * n);
+        auto load4 = [&](int c, float (&v)[4]) {
+            if (GATHER) {
+                const uint2 raw = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(src) + (size_t)t * n)[c];
+                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+            } else {
+                const float4 f = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + (size_t)slot * n)[c];
+                v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+            }
+        };
+        float amax = 0.0f;
+        if (t >= 0) {
+            for (int c = threadIdx.x; c < n_cells; c += 256) {
+                float v[4];
+                load4(c, v);
+                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[0]), fabsf(v[1]))), fmaxf(fabsf(v[2]), fabsf(v[3])));
+            }
+        }
+        for (int off = 16; off; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+        __syncthreads();
+        if (lane == 0) s_red[warp] = amax;
+        __syncthreads();
+        amax = s_red[0];
+        for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_red[i]);
+        const bool live = t >= 0 && amax > 0.0f && amax < 3.0e38f;
+        const float scale = live ? I8_XMAX / amax : 0.0f;
+        const float kap = kappa[slot];
+        if (threadIdx.x == 0) sigma[slot] = live ? amax / I8_XMAX : 0.0f;
+        const int n_iter = (n_cells + 255) / 256;
+        for (int itr = 0; itr < n_iter; ++itr) {
+            const int c = itr * 256 + threadIdx.x;
+            int sum = 0;
+            if (c < n_cells) {
+                uint32_t wh = 0, wl = 0;
+                if (live) {
+                    float v[4];
+                    load4(c, v);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        int xq = __float2int_rn(v[i] * scale);
+                        xq = max(-16191, min(16191, xq));
+                        const int lo8 = ((xq + 64) & 127) - 64;
+                        const int hi = (xq - lo8) >> 7;
+                        const int byte = ((i & 1) << 1) | (i >> 1);
+                        wh |= (uint32_t)(hi & 255) << (8 * byte);
+                        wl |= (uint32_t)(lo8 & 255) << (8 * byte);
+                        sum += xq;
+                    }
+                }
+                qh[c] = wh; ql[c] = wl;
+            }
+            for (int off = cpg >> 1; off; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            if (c < n_cells && (c % cpg) == 0) {
+                const int G = c / cpg;
+                float2 o;
+                o.x = (float)sum; o.y = kap * (float)sum;
+                reinterpret_cast<float2*>(xk)[(size_t)G * R_alloc + slot] = o;
+            }
+        }
+    }
+}
+
+// tensor maps over a row-major byte matrix [rows, cols], 128-byte swizzle, boxes of 128 columns x 16/32/64 rows
+static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long long cols) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    for (int i = 0; i < 3; ++i) {
+        cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)cols};
+        cuuint32_t box[2] = {128, (cuuint32_t)(16 << i)};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&maps->m[i], CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    maps->m[3] = maps->m[2]; maps->m[4] = maps->m[2];
+    return true;
+}
+
+}  // namespace
+
+static int g_i8_dbg_mode = 0;
+#if defined(D2MOE_WAIT_STATS) || defined(D2MOE_I8_DBG)
+extern "C" int d2moe_debug_i8_set_mode(int mode) { g_i8_dbg_mode = mode; return 0; }
+#endif
+#ifdef D2MOE_WAIT_STATS
+extern "C" int d2moe_debug_i8_stats(unsigned long long* host16, int reset) {
+    cudaDeviceSynchronize();
+    if (cudaMemcpyFromSymbol(host16, g_i8_stats, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_i8_stats, z, sizeof(z)); }
+    return 0;
+}
+#endif
+
+cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                          const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
+                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
+    auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
+    const int n_exp = D.E + D.n_shared;
+    I8Unit* units = reinterpret_cast<I8Unit*>(B.units);
+    float* kappa = B.slot_f;
+    float* sigma_x = B.slot_f + pl.R_alloc;
+    float* sigma_h = B.slot_f + 2 * pl.R_alloc;
+    int8_t* qx = reinterpret_cast<int8_t*>(B.xp16);
+    int8_t* qh = reinterpret_cast<int8_t*>(B.h16);
+    const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
+
+    i8_prep_kernel<<<1, 256, 0, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
+                                      pl.max_units, Lgu.top, Lgu.b1);
+    i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
+                                                    qx, B.xk_x, sigma_x);
+
+    TmaMaps maps_x, maps_h;
+    if (!make_maps_u8(&maps_x, qx, 2 * pl.R_alloc, D.d) || !make_maps_u8(&maps_h, qh, 2 * pl.R_alloc, D.F))
+        return cudaErrorNotSupported;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+
+    for (int mode = 0; mode < 2; ++mode) {
+        I8Params p;
+        p.D = D; p.L = mode == 0 ? Lgu : Ld; p.P = P; p.mode = mode;
+        p.n_row_tiles = mode == 0 ? D.F / 64 : D.d / 128;
+        p.n_split = mode == 0 ? 1 : pl.n_split;
+        p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
+        p.units = units; p.n_units = B.n_units;
+        p.xk = mode == 0 ? B.xk_x : B.xk_h;
+        p.sigma = mode == 0 ? sigma_x : sigma_h;
+        p.hbuf = B.h32; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
+        p.dbg = g_i8_dbg_mode;
+        const int gps = 128 / D.g;
+        const int b_bytes = I8_NSB * I8_B_STAGE;
+        const int w_slot = gps * 2 * p.L.block_bytes;
+        const int epi_bytes = 2 * 64 * I8_EPI_STRIDE * 4;
+        const int bar_bytes = 512;
+        const int budget = 112 * 1024;
+        int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
+        if (nsw > I8_MAX_NSW) nsw = I8_MAX_NSW;
+        if (nsw < 2) return cudaErrorInvalidConfiguration;
+        p.nsw = nsw;
+        p.smem_w_off = b_bytes;
+        p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
+        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
+        if (mode == 1)
+            i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,
+                                                             kappa, qh, B.xk_h, sigma_h);
+        mark(mode == 0 ? 1 : 2);
+        // width lists whose segments are stored exactly get a kernel specialised on the list
+        int swpack = 0;
+        bool exact = p.L.n_seg <= 4;
+        for (int j = 0; j < p.L.n_seg && exact; ++j) {
+            exact = p.L.seg_w[j] == p.L.seg_sw[j];
+            swpack |= p.L.seg_sw[j] << (4 * j);
+        }
+        if (!exact) swpack = 0;
+        auto launch = [&](auto kern) -> cudaError_t {
+            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (err != cudaSuccess) return err;
+            kern<<<2 * sms, I8_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            return cudaSuccess;
+        };
+        cudaError_t e;
+        if (D.g == 128 && swpack == 0x4112) e = launch(ffn_i8_kernel<128, 0x4112>);
+        else if (D.g == 128 && swpack == 0x422) e = launch(ffn_i8_kernel<128, 0x422>);
+        else if (D.g == 128) e = launch(ffn_i8_kernel<128, 0>);
+        else e = launch(ffn_i8_kernel<64, 0>);
+        if (e != cudaSuccess) return e;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}

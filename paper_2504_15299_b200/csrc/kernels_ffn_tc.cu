@@ -532,14 +532,16 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     // decode-sized loads (few tokens per expert): the memory-bound kernel, K accumulators of n_cap columns
     pl->decode = avg <= 24 ? 1 : 0;
     if (pl->decode) {
-        int cap = (128 / c->n_bits) & ~15;
-        pl->n_cap = cap > 32 ? 32 : cap;     // 32 tokens x g columns of activations per ring slot
+        pl->n_cap = 32;                      // token slots per unit
     } else {
         pl->n_cap = 320;
     }
     const long long n_pieces = pl->decode ? (long long)c->n_experts + c->n_shared
                                           : (long long)c->n_experts * c->n_bits + c->n_shared;
-    long long pad_rows = A_tot + 15 * (n_pieces < A_tot ? n_pieces : A_tot);
+    // decode: every (expert, width) class is padded to 8 slots; otherwise pieces are padded to 16 rows
+    const long long n_classes = (long long)c->n_experts * c->n_bits + c->n_shared;
+    long long pad_rows = pl->decode ? A_tot + 7 * (n_classes < A_tot ? n_classes : A_tot)
+                                    : A_tot + 15 * (n_pieces < A_tot ? n_pieces : A_tot);
     pl->R_alloc = ((pad_rows + 255) / 256) * 256 + 256;
     pl->max_units = (int)(c->n_experts + c->n_shared + pl->R_alloc / pl->n_cap + 1);
     // split-K of the down projection: aim for >= 4 work items per resident CTA (2 per SM, 148 SMs)
@@ -551,6 +553,7 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     if (want > 8) want = 8;
     if (want > n_groups / 4) want = n_groups / 4 > 0 ? n_groups / 4 : 1;
     pl->groups_per_split = (int)((n_groups + want - 1) / want);
+    if (c->group_size == 64 && (pl->groups_per_split & 1)) ++pl->groups_per_split;   // whole 128-column ring stages
     pl->n_split = (n_groups + pl->groups_per_split - 1) / pl->groups_per_split;
 }
 

@@ -13,9 +13,22 @@ struct TcUnit {
     int real[8];   // its real (non-padding) columns inside the unit
 };
 
+// Unit of the 8-bit decode kernel: up to 32 consecutive token slots of one expert.  The slots of an
+// expert are laid out by width, widest first, every width class padded to a multiple of 8 slots, so
+// the slots that include segment j are the first npad[j] slots of the unit.
+struct I8Unit {
+    int e;         // expert (routed, then shared)
+    int slot0;     // first slot (multiple of 8); the quantised activations of slot s are rows 2s, 2s+1
+    int nslots;    // slots in this unit (multiple of 8, <= 32)
+    int kmax;      // highest width index present
+    int nblk;      // blocks of 4 slots that hold at least one real token
+    int npad[8];   // slots covered by the product of segment j (multiple of 8, 0 = absent)
+    int blk[8];    // the real blocks: first slot / 4, relative to slot0
+};
+
 struct TcPlan {
-    int decode;             // 1: memory-bound decode kernel (tokens sorted widest first, one tile per
-                            //    segment); 0: grouped dequant-GEMM (one tile per width, any load)
+    int decode;             // 1: memory-bound 8-bit decode kernel (tokens laid out widest first, scales applied
+                            //    to the accumulators); 0: grouped fp16 dequant-GEMM (one tile per width, any load)
     int n_cap;              // columns per unit
     long long R_alloc;      // rows of the padded activation buffers
     int max_units;
@@ -27,6 +40,11 @@ struct TcBuffers {
     __half* xp16;           // [R_alloc, d]   gathered tokens, fp16
     __half* h16;            // [R_alloc, F]   SwiGLU outputs, fp16
     float* o32;             // [n_split][R_alloc, d] partial expert outputs
+    // 8-bit decode kernel: xp16 / h16 are reused as the quantised activations [2 R_alloc, d] / [2 R_alloc, F]
+    float* h32;             // [R_alloc, F]   SwiGLU outputs, fp32
+    float* xk_x;            // [d / g][R_alloc][2]   per group and slot: sum of the quantised x, kappa * sum
+    float* xk_h;            // [F / g][R_alloc][2]
+    float* slot_f;          // [3][R_alloc]   kappa, scale of x, scale of h per slot
 };
 
 bool tc_path_supported(const d2moe_config* c);
@@ -34,6 +52,6 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl);
 cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                               const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
                               const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
-cudaError_t launch_ffn_decode(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
-                              const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
-                              const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
+cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
+                          const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
+                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);

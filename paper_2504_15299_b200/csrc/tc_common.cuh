@@ -74,6 +74,35 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     mbar_wait_slow(bar, parity, abort_flag, status, drain);
 }
 
+// The same bounded wait written entirely in PTX: the common case (phase already complete) costs the
+// try_wait and one predicated branch, with no integer instructions to turn the predicate into a
+// value and back.  abort_addr: shared-memory address of the CTA's abort flag; status must not be null.
+__device__ __forceinline__ void mbar_wait_ptx(uint32_t bar, uint32_t parity, uint32_t abort_addr, int32_t* status) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u32 ab;\n\t"
+        ".reg .u64 t0, t1;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%0], %1;\n\t"
+        "@p bra WAIT_DONE;\n\t"
+        "mov.u64 t0, %%globaltimer;\n"
+        "WAIT_RETRY:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%0], %1, 4000;\n\t"
+        "@p bra WAIT_DONE;\n\t"
+        "ld.volatile.shared.u32 ab, [%2];\n\t"
+        "setp.ne.u32 q, ab, 0;\n\t"
+        "@q bra WAIT_DONE;\n\t"
+        "mov.u64 t1, %%globaltimer;\n\t"
+        "sub.u64 t1, t1, t0;\n\t"
+        "setp.lt.u64 q, t1, 1000000000;\n\t"
+        "@q bra WAIT_RETRY;\n\t"
+        "st.volatile.shared.u32 [%2], 1;\n\t"
+        "red.global.or.b32 [%3], 2;\n"    // D2MOE_DEV_TIMEOUT
+        "WAIT_DONE:\n\t"
+        "}"
+        ::"r"(bar), "r"(parity), "r"(abort_addr), "l"(status) : "memory");
+}
+
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
