@@ -227,7 +227,7 @@ def run_reference(args):
     if rank != 0:
         return
     wl = synth.WORKLOADS[args.workload]
-    T = args.tokens
+    T = args.tokens or synth.WORKLOADS[args.workload].tokens[-1]
     total_steps = args.steps + args.warmup
     # size the sample so the whole run stays within ~2.5 minutes: calibrate on one hidden group
     t0 = time.perf_counter()
@@ -294,7 +294,7 @@ def run_ours(args):
     B.lib()
 
     wl = synth.WORKLOADS[args.workload]
-    T = args.tokens
+    T = args.tokens or synth.WORKLOADS[args.workload].tokens[-1]
     path = {"auto": B.PATH_AUTO, "cuda_core": B.PATH_CUDA_CORE, "tensor": B.PATH_TENSOR}[args.path]
     cfg = B.Config.from_workload(wl, kernel_path=path)
 
@@ -465,7 +465,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mixtral_decode", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--tokens", type=int, default=64)
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="tokens per step (default: the largest batch size of the workload, 64 for mixtral_decode)")
     ap.add_argument("--path", default="auto", choices=["auto", "cuda_core", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -185,14 +185,15 @@ __device__ __forceinline__ void unpack_dispatch(int sw, uint32_t seg, int rr, in
     }
 }
 
-// Compile-time description of a width list whose segments are stored exactly (widths 1, 2, 4, 8):
-// nibble j of SWPACK is the width of segment j.  SWPACK == 0 selects the run-time path.
-template <int SWPACK>
+// Compile-time description of a width list of at most four segments: nibble j of WPACK is the logical
+// width of segment j (stored 1, 2, 4 or 8 bits wide).  WPACK == 0 selects the run-time path.
+template <int WPACK>
 struct I8SegList {
-    __host__ __device__ static constexpr int sw(int j) { return (SWPACK >> (4 * j)) & 15; }
-    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && sw(k) != 0) ++k; return k; }
-    __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += sw(i); return b; }
-    __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += sw(i); return top() - b; }
+    __host__ __device__ static constexpr int w(int j) { return (WPACK >> (4 * j)) & 15; }
+    __host__ __device__ static constexpr int sw(int j) { return w(j) <= 1 ? 1 : (w(j) <= 2 ? 2 : (w(j) <= 4 ? 4 : 8)); }
+    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && w(k) != 0) ++k; return k; }
+    __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += w(i); return b; }
+    __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += w(i); return top() - b; }
     __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
 };
 
@@ -544,7 +545,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 if constexpr (J < SL::count()) {
                                     if ((J & 1) == wg && J <= kmax) {
                                         I8_SKIP(2)
-                                        unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::sw(J), SL::pos(J),
+                                        unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J),
                                                                       a_base + (J >> 1) * 32);
                                     }
                                 }
@@ -865,14 +866,10 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
             i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,
                                                              kappa, qh, B.xk_h, sigma_h);
         mark(mode == 0 ? 1 : 2);
-        // width lists whose segments are stored exactly get a kernel specialised on the list
-        int swpack = 0;
-        bool exact = p.L.n_seg <= 4;
-        for (int j = 0; j < p.L.n_seg && exact; ++j) {
-            exact = p.L.seg_w[j] == p.L.seg_sw[j];
-            swpack |= p.L.seg_sw[j] << (4 * j);
-        }
-        if (!exact) swpack = 0;
+        // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
+        int wpack = 0;
+        if (p.L.n_seg <= 4)
+            for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
         auto launch = [&](auto kern) -> cudaError_t {
             cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
             if (err != cudaSuccess) return err;
@@ -880,8 +877,9 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
             return cudaSuccess;
         };
         cudaError_t e;
-        if (D.g == 128 && swpack == 0x4112) e = launch(ffn_i8_kernel<128, 0x4112>);
-        else if (D.g == 128 && swpack == 0x422) e = launch(ffn_i8_kernel<128, 0x422>);
+        if (D.g == 128 && wpack == 0x4112) e = launch(ffn_i8_kernel<128, 0x4112>);        // {2,3,4,8}
+        else if (D.g == 128 && wpack == 0x422) e = launch(ffn_i8_kernel<128, 0x422>);     // {2,4,8}
+        else if (D.g == 128 && wpack == 0x1115) e = launch(ffn_i8_kernel<128, 0x1115>);   // {5,6,7,8}
         else if (D.g == 128) e = launch(ffn_i8_kernel<128, 0>);
         else e = launch(ffn_i8_kernel<64, 0>);
         if (e != cudaSuccess) return e;

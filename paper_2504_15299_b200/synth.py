@@ -196,6 +196,12 @@ WORKLOADS = {
     "mixtral_stack": Workload("mixtral_stack", 4096, 14336, 8, 2, 128, (2, 3, 4, 8),
                               (0.25, 0.25, 0.25, 0.25), seed=4, tokens=(16,), learned_bits=True,
                               n_layers=32),
+    # the same layer shape with the width list {5,6,7,8}, and a dense gated FFN (one expert, top-1) of
+    # LLaMA2-13B's FFN shape: both are plain configurations of the same path
+    "mixtral_v2": Workload("mixtral_v2", 4096, 14336, 8, 2, 128, (5, 6, 7, 8),
+                           (0.25, 0.25, 0.25, 0.25), seed=5, tokens=(64,)),
+    "dense_ffn": Workload("dense_ffn", 5120, 13824, 1, 1, 128, (2, 3, 4, 8),
+                          (0.1, 0.2, 0.4, 0.3), seed=6, tokens=(16,)),
 }
 
 

@@ -352,7 +352,8 @@ def test_stack_two_full_size_layers_teacher_forced(B):
 
 
 # ------------------------------------------------------------------ other width lists, group sizes, loads
-def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=21, one_expert=False):
+def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=21, one_expert=False,
+                     token_scales=None, outlier=None):
     """Random small layer through the tensor-core path, the CUDA-core path and the oracle."""
     _, routing, moe = oracle_mods()
     from oracle import mwq
@@ -369,7 +370,12 @@ def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=
             mats.append(np_f32(W))
             blobs.append(B.pack_mwq(cfg_tc, W))
         raw[e] = mats
-    x = synth.bf16_exact(synth.normal(seed, 1, (T, d), 1.0, "cuda"))
+    x = synth.normal(seed, 1, (T, d), 1.0, "cuda")
+    if token_scales is not None:       # per-token magnitudes (0 = an all-zero token)
+        x = x * torch.tensor(token_scales, dtype=x.dtype, device="cuda")[:, None]
+    if outlier is not None:            # (token, element, value): one element far above the rest of its token
+        x[outlier[0], outlier[1]] = outlier[2]
+    x = synth.bf16_exact(x)
     logits = synth.normal(seed, 5, (T, E), 1.0, "cuda")
     if one_expert:
         logits[:, 0] += 100.0          # every token picks expert 0 first: units beyond n_cap
@@ -392,12 +398,21 @@ def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=
 
     toks = sorted(set([0, T // 2, T - 1]))
     ref = moe.moe_layer(np_f32(x), rt, get, bits, E, n_shared, tokens=toks)
-    err = max(max_norm_rel_err(np_f32(y_tc)[t], ref[t]) for t in toks)
+    if token_scales is not None:
+        toks = list(range(T))
+        ref = moe.moe_layer(np_f32(x), rt, get, bits, E, n_shared, tokens=toks)
+    err = 0.0
+    for t in toks:
+        if np.abs(ref[t]).max() == 0.0:            # an all-zero token must come out as exact zeros
+            assert np.abs(np_f32(y_tc)[t]).max() == 0.0
+        else:
+            err = max(err, max_norm_rel_err(np_f32(y_tc)[t], ref[t]))
     return cross, err
 
 
 @pytest.mark.parametrize("bits,g", [((2, 3, 4), 128), ((4, 8), 128), ((8,), 64), ((1, 2, 3, 4, 5, 6, 7, 8), 128),
-                                    ((3, 5), 64), ((2, 8), 128), ((5, 6, 7, 8), 64)])
+                                    ((3, 5), 64), ((2, 8), 128), ((5, 6, 7, 8), 64), ((5, 6, 7, 8), 128),
+                                    ((2, 4, 8), 128), ((2, 3, 4, 8), 64)])
 def test_other_width_lists_on_the_tensor_core_paths(B, bits, g):
     cross, err = small_layer_case(B, d=256, F=384, E=4, k=2, g=g, bits=bits, T=24)
     assert cross < TOL and err < TOL, (cross, err)
@@ -414,6 +429,21 @@ def test_prefill_sized_load_small_shape(B):
     # 400 tokens on 2 experts: the grouped dequant-GEMM path (more than 24 tokens per expert)
     cross, err = small_layer_case(B, d=256, F=256, E=2, k=1, g=128, bits=(2, 3, 4, 8), T=400,
                                   probs=[0.1, 0.2, 0.4, 0.3])
+    assert cross < TOL and err < TOL, (cross, err)
+
+
+def test_decode_kernel_per_token_activation_scaling(B):
+    # the decode kernel quantises every token against its own largest element: tokens of very different
+    # magnitude, an all-zero token and a token with one element 100 times above the rest in one batch
+    scales = [1.0, 1e-3, 1e3, 0.0, 1.0, 37.5, 2.0 ** -10, 1.0, 5.0]
+    cross, err = small_layer_case(B, d=256, F=384, E=2, k=2, g=128, bits=(2, 3, 4, 8), T=9, token_scales=scales,
+                                  outlier=(4, 17, 100.0))
+    assert err < TOL, err
+
+
+def test_dense_ffn_single_expert(B):
+    # E = 1, k = 1: a dense gated FFN read at a per-token width (the method applied to a dense model)
+    cross, err = small_layer_case(B, d=384, F=512, E=1, k=1, g=128, bits=(2, 3, 4, 8), T=20)
     assert cross < TOL and err < TOL, (cross, err)
 
 
