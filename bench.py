@@ -273,6 +273,127 @@ def workload_config(wl, T, path):
 
 
 # ------------------------------------------------------------------------------------------------
+# layer stack (the 32-layer decode configuration): one step = every layer once, replayed as a CUDA graph
+# ------------------------------------------------------------------------------------------------
+def run_stack(args):
+    from paper_2504_15299_b200 import binding as B, build
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    build.build_library()
+    B.lib()
+    wl = synth.WORKLOADS[args.workload]
+    T = args.tokens or wl.tokens[-1]
+    L = args.layers or wl.n_layers
+    cfg = B.Config.from_workload(wl)
+    layers = []
+    for l in range(L):
+        blobs = []
+        for e in range(wl.n_experts + wl.n_shared):
+            for m in range(3):
+                W = synth.expert_matrix(wl, e, m, device=dev, layer=l)
+                blobs.append(B.pack_mwq(cfg, W))
+                del W
+        layers.append((blobs, synth.gate_weight_bf16(wl, dev, layer=l), synth.bit_router_weight_bf16(wl, dev, layer=l)))
+    ws = torch.empty(B.workspace_bytes(cfg, T), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n_batches = 4
+    xs = [synth.tokens_bf16(wl, T, dev, step=1000 + i) for i in range(n_batches)]
+    x = torch.empty_like(xs[0])
+    xn = torch.empty_like(x)
+
+    def one_step():
+        for blobs, gw, bw in layers:
+            B.stack_layer(cfg, x, xn, blobs, gate_w=gw, bit_w=bw, workspace=ws, device_status=status)
+
+    # algorithmic bytes of a step from the realised routing of every layer (batch 0, eager pass)
+    x.copy_(xs[0])
+    step_bytes = 0
+    for blobs, gw, bw in layers:
+        B.stack_layer(cfg, x, xn, blobs, gate_w=gw, bit_w=bw, workspace=ws, device_status=status)
+        r = B.route(cfg, xn, gate_w=gw, bit_w=bw)
+        torch.cuda.synchronize()
+        step_bytes += algorithmic_bytes(wl, T, r.group_off.cpu().tolist())["layer"]
+
+    side = torch.cuda.Stream()
+    graph = None
+    if not args.no_graph:
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            one_step()                     # warm-up on the capture stream (function attributes, tensor maps)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+
+    def step(i):
+        x.copy_(xs[i % n_batches])
+        if graph is not None:
+            graph.replay()
+        else:
+            one_step()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_per_step = e0.elapsed_time(e1) / args.steps
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    # end to end: tokens from pinned host memory, the stack, result back to the host, every step
+    hx = [t.cpu().pin_memory() for t in xs]
+    hy = torch.empty_like(hx[0]).pin_memory()
+
+    def e2e_step(i):
+        x.copy_(hx[i % n_batches], non_blocking=True)
+        if graph is not None:
+            graph.replay()
+        else:
+            one_step()
+        hy.copy_(x, non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(args.steps):
+        e2e_step(i)
+    f1.record()
+    torch.cuda.synchronize()
+    e2e_ms = f0.elapsed_time(f1) / args.steps
+
+    peak, peak_kind = measured_peaks()
+    achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": T / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "i8", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: {L} layers of d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} "
+                                   f"top{wl.top_k} g={wl.group_size} bits={list(wl.bits)}, widths from the per-expert "
+                                   f"bit-width routers, RMSNorm + residual per layer",
+                       "tokens_per_step": T, "layers": L, "cuda_graph": graph is not None,
+                       "l2": f"inputs larger than L2: {L} layers of distinct packed experts "
+                             f"({step_bytes / 1e9:.1f} GB read per step)"},
+            "clocks": clocks,
+            "e2e": {"value": T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hx[0].numel() * 2,
+                    "d2h_bytes_per_step": hy.numel() * 2},
+            "gpu_launches": (B.forward_launch_count(cfg, T) + 1) * L * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "whole step", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "algorithmic_bytes_per_step": step_bytes},
+            "cpu_baseline": None}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -468,11 +589,16 @@ def main():
     ap.add_argument("--tokens", type=int, default=0,
                     help="tokens per step (default: the largest batch size of the workload, 64 for mixtral_decode)")
     ap.add_argument("--path", default="auto", choices=["auto", "cuda_core", "tensor"])
+    ap.add_argument("--layers", type=int, default=0,
+                    help="mixtral_stack only: layers per step (default: the workload's 32; 46 GB of packed experts)")
+    ap.add_argument("--no-graph", action="store_true", help="mixtral_stack only: launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif synth.WORKLOADS[args.workload].n_layers > 1 and int(os.environ.get("WORLD_SIZE", "1")) == 1:
+        run_stack(args)
     else:
         run_ours(args)
 

@@ -617,31 +617,43 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // One block.  Lays every expert's tokens out by width, widest first, each width class padded to a
 // multiple of 8 slots; cuts every expert into units of 32 slots; records per unit and segment how many
 // of its slots include the segment, and which blocks of 4 slots hold real tokens.
+// Shared memory: group_off (E K + 1 ints), then per expert its first unit (n_exp + 1 ints).
 __global__ void __launch_bounds__(256)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
                int32_t* src_token, float* kappa, int max_units, int top, int b1) {
+    extern __shared__ int32_t s_prep[];
     __shared__ int s_total;
-    const int n_exp = D.E + D.n_shared;
-    if (threadIdx.x < 32) {                       // padded expert offsets (one warp scans)
+    const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
+    int32_t* go = s_prep;                          // group_off
+    int32_t* unit_off = s_prep + n_keys + 1;
+    for (int i = threadIdx.x; i <= n_keys; i += blockDim.x) go[i] = R.group_off[i];
+    __syncthreads();
+    if (threadIdx.x < 32) {                       // padded slot offsets and first units (one warp scans)
         const int lane = threadIdx.x;
-        int carry = 0;
+        int carry = 0, ucarry = 0;
         for (int base = 0; base < n_exp; base += 32) {
             const int e = base + lane;
             int v = 0;
             if (e < D.E) {
-                for (int j = 0; j < D.K; ++j) v += round8(R.group_off[e * D.K + j + 1] - R.group_off[e * D.K + j]);
+                for (int j = 0; j < D.K; ++j) v += round8(go[e * D.K + j + 1] - go[e * D.K + j]);
             } else if (e < n_exp) {
                 v = round8(D.T);
             }
-            int incl = v;
+            const int nu = (v + I8_SLOTS - 1) / I8_SLOTS;
+            int incl = v, uincl = nu;
             for (int off = 1; off < 32; off <<= 1) {
                 const int o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += o;
+                const int uo = __shfl_up_sync(0xffffffffu, uincl, off);
+                if (lane >= off) { incl += o; uincl += uo; }
             }
-            if (e < n_exp) pad_off[e] = carry + incl - v;
+            if (e < n_exp) { pad_off[e] = carry + incl - v; unit_off[e] = ucarry + uincl - nu; }
             carry += __shfl_sync(0xffffffffu, incl, 31);
+            ucarry += __shfl_sync(0xffffffffu, uincl, 31);
         }
-        if (lane == 0) { pad_off[n_exp] = carry; s_total = carry; }
+        if (lane == 0) {
+            pad_off[n_exp] = carry; s_total = carry; unit_off[n_exp] = ucarry;
+            *n_units = min(ucarry, max_units);
+        }
     }
     __syncthreads();
     const int total = s_total;
@@ -652,8 +664,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         const int e = R.topk_idx[a], kk = R.bit_idx[a];
         if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) { row_map[a] = 0; continue; }
         int start = 0;                            // classes of a larger width index come first
-        for (int i = kk + 1; i < D.K; ++i) start += round8(R.group_off[e * D.K + i + 1] - R.group_off[e * D.K + i]);
-        const int slot = pad_off[e] + start + (pos - R.group_off[e * D.K + kk]);
+        for (int i = kk + 1; i < D.K; ++i) start += round8(go[e * D.K + i + 1] - go[e * D.K + i]);
+        const int slot = pad_off[e] + start + (pos - go[e * D.K + kk]);
         row_map[a] = slot;
         if (slot >= 0 && slot < total) {
             src_token[slot] = a / D.k;
@@ -667,34 +679,31 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         src_token[slot] = t;
         kappa[slot] = 0.5f - exp2f((float)(top - b1 - 1));
     }
-    if (threadIdx.x == 0) {
-        int nu = 0;
-        for (int e = 0; e < n_exp; ++e) {
-            const int p0 = pad_off[e], len_e = pad_off[e + 1] - p0;
-            int cnt[8], cpad[9];                  // cpad[j]: padded slots of the classes with index >= j
-            cpad[D.K] = 0;
-            for (int j = D.K - 1; j >= 0; --j) {
-                cnt[j] = e < D.E ? R.group_off[e * D.K + j + 1] - R.group_off[e * D.K + j] : (j == D.K - 1 ? D.T : 0);
-                cpad[j] = cpad[j + 1] + round8(cnt[j]);
-            }
-            for (int start = 0; start < len_e && nu < max_units; start += I8_SLOTS) {
-                const int len = min(len_e - start, I8_SLOTS);
-                I8Unit u;
-                u.e = e; u.slot0 = p0 + start; u.nslots = len; u.kmax = 0; u.nblk = 0;
-                for (int j = 0; j < 8; ++j) {
-                    u.blk[j] = 0;
-                    u.npad[j] = j < D.K ? max(0, min(len, cpad[j] - start)) : 0;
-                    if (u.npad[j] > 0) u.kmax = j;
-                }
-                for (int j = D.K - 1; j >= 0; --j) {          // real slots of class j: [cpad[j+1], cpad[j+1] + cnt[j])
-                    const int a0 = max(cpad[j + 1], start), a1 = min(cpad[j + 1] + cnt[j], start + len);
-                    for (int b = a0 / 4; 4 * b < a1; ++b)
-                        if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
-                }
-                if (u.nblk > 0) units[nu++] = u;
-            }
+    for (int e = threadIdx.x; e < n_exp; e += blockDim.x) {        // one thread per expert: its units
+        const int p0 = pad_off[e], len_e = pad_off[e + 1] - p0;
+        int cnt[8], cpad[9];                      // cpad[j]: padded slots of the classes with index >= j
+        cpad[D.K] = 0;
+        for (int j = D.K - 1; j >= 0; --j) {
+            cnt[j] = e < D.E ? go[e * D.K + j + 1] - go[e * D.K + j] : (j == D.K - 1 ? D.T : 0);
+            cpad[j] = cpad[j + 1] + round8(cnt[j]);
         }
-        *n_units = nu;
+        int nu = unit_off[e];
+        for (int start = 0; start < len_e && nu < max_units; start += I8_SLOTS, ++nu) {
+            const int len = min(len_e - start, I8_SLOTS);
+            I8Unit u;
+            u.e = e; u.slot0 = p0 + start; u.nslots = len; u.kmax = 0; u.nblk = 0;
+            for (int j = 0; j < 8; ++j) {
+                u.blk[j] = 0;
+                u.npad[j] = j < D.K ? max(0, min(len, cpad[j] - start)) : 0;
+                if (u.npad[j] > 0) u.kmax = j;
+            }
+            for (int j = D.K - 1; j >= 0; --j) {          // real slots of class j: [cpad[j+1], cpad[j+1] + cnt[j])
+                const int a0 = max(cpad[j + 1], start), a1 = min(cpad[j + 1] + cnt[j], start + len);
+                for (int b = a0 / 4; 4 * b < a1; ++b)
+                    if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
+            }
+            units[nu] = u;                        // every window starts with a real token: never empty
+        }
     }
 }
 
@@ -825,7 +834,8 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     int8_t* qh = reinterpret_cast<int8_t*>(B.h16);
     const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
 
-    i8_prep_kernel<<<1, 256, 0, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
+    const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1) * 4;
+    i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
                                       pl.max_units, Lgu.top, Lgu.b1);
     i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
                                                     qx, B.xk_x, sigma_x);

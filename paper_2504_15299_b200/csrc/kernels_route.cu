@@ -180,6 +180,59 @@ __global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ ke
     }
 }
 
+// Decode-sized loads: the three steps above in one block, keys staged in shared memory (same
+// warp-per-key ballot walks, so the result is the same stable order).  smem: A keys + n_keys + 1 ints.
+__global__ void __launch_bounds__(1024)
+group_small_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
+                   int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+    extern __shared__ int32_t s_grp[];
+    int32_t* s_keys = s_grp;
+    int32_t* s_off = s_grp + ((A + 31) & ~31);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int a = threadIdx.x; a < A; a += blockDim.x) s_keys[a] = keys[a];
+    __syncthreads();
+    for (int key = warp; key < n_keys; key += n_warps) {
+        int cnt = 0;
+        for (int base = 0; base < A; base += 32) {
+            const int a = base + lane;
+            cnt += __popc(__ballot_sync(0xffffffffu, a < A && s_keys[a] == key));
+        }
+        if (lane == 0) s_off[key] = cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int base = 0; base < n_keys; base += 32) {
+            const int i = base + lane;
+            const int v = i < n_keys ? s_off[i] : 0;
+            int incl = v;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (i < n_keys) { s_off[i] = carry + incl - v; group_off[i] = carry + incl - v; }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) { s_off[n_keys] = carry; group_off[n_keys] = carry; }
+    }
+    __syncthreads();
+    for (int key = warp; key < n_keys; key += n_warps) {
+        int pos = s_off[key];
+        if (pos == s_off[key + 1]) continue;
+        for (int base = 0; base < A; base += 32) {
+            const int a = base + lane;
+            const bool m = a < A && s_keys[a] == key;
+            const unsigned bal = __ballot_sync(0xffffffffu, m);
+            if (m) {
+                const int p = pos + __popc(bal & ((1u << lane) - 1u));
+                perm[p] = a;
+                inv_perm[a] = p;
+            }
+            pos += __popc(bal);
+        }
+    }
+}
+
 // Same dot product with both vectors already in shared memory.
 __device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const __nv_bfloat16* b, int d, int lane) {
     float acc = 0.0f;
@@ -380,6 +433,13 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     } else
     route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
+    // few assignments and keys: histogram, scan and scatter in one single-block launch
+    const long long walks = (long long)n_keys * ((D.A + 31) / 32);
+    if (D.A <= 8192 && n_keys <= 2048 && walks <= 16384) {
+        const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
+        group_small_kernel<<<1, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+        return cudaGetLastError();
+    }
     count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);
     scan_kernel<<<1, 32, 0, st>>>(n_keys, hist_ws, R.group_off);
     scatter_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
