@@ -716,7 +716,7 @@ template <bool GATHER>
 __global__ void __launch_bounds__(256)
 i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, const int32_t* __restrict__ src_token,
                 const int32_t* __restrict__ pad_off, int n_off, const float* __restrict__ kappa,
-                int8_t* __restrict__ q, float* __restrict__ xk, float* __restrict__ sigma) {
+                int8_t* __restrict__ q, float* __restrict__ xk, float* __restrict__ sigma, int32_t* status) {
     __shared__ float s_red[8];
     const int total = pad_off[n_off];
     const int n_cells = n / 4, cpg = g / 4;                 // cells per group: 16 or 32
@@ -737,20 +737,24 @@ i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, c
             }
         };
         float amax = 0.0f;
+        int bad = 0;                               // a NaN or an infinity in the row (fmaxf would drop a NaN)
         if (t >= 0) {
             for (int c = threadIdx.x; c < n_cells; c += 256) {
                 float v[4];
                 load4(c, v);
                 amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[0]), fabsf(v[1]))), fmaxf(fabsf(v[2]), fabsf(v[3])));
+                bad |= !(fabsf(v[0]) < 3.0e38f) | !(fabsf(v[1]) < 3.0e38f) | !(fabsf(v[2]) < 3.0e38f) | !(fabsf(v[3]) < 3.0e38f);
             }
         }
         for (int off = 16; off; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
-        __syncthreads();
+        bad = __syncthreads_or(bad);
         if (lane == 0) s_red[warp] = amax;
         __syncthreads();
         amax = s_red[0];
         for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_red[i]);
-        const bool live = t >= 0 && amax > 0.0f && amax < 3.0e38f;
+        const bool live = t >= 0 && amax > 0.0f && !bad;
+        // a row with a NaN or an infinity cannot be quantised: its outputs are zero and the call is flagged
+        if (bad && threadIdx.x == 0 && status) atomicOr(status, D2MOE_DEV_NONFINITE);
         const float scale = live ? I8_XMAX / amax : 0.0f;
         const float kap = kappa[slot];
         if (threadIdx.x == 0) sigma[slot] = live ? amax / I8_XMAX : 0.0f;
@@ -838,7 +842,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
                                       pl.max_units, Lgu.top, Lgu.b1);
     i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
-                                                    qx, B.xk_x, sigma_x);
+                                                    qx, B.xk_x, sigma_x, device_status);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps_u8(&maps_x, qx, 2 * pl.R_alloc, D.d) || !make_maps_u8(&maps_h, qh, 2 * pl.R_alloc, D.F))
@@ -874,7 +878,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         if (mode == 1)
             i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,
-                                                             kappa, qh, B.xk_h, sigma_h);
+                                                             kappa, qh, B.xk_h, sigma_h, device_status);
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         int wpack = 0;

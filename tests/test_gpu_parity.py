@@ -441,6 +441,30 @@ def test_decode_kernel_per_token_activation_scaling(B):
     assert err < TOL, err
 
 
+def test_decode_kernel_flags_nonfinite_activations(B):
+    # a NaN in one token: the call is flagged, that token comes out as zeros, the others are untouched
+    d, F, E, k, g, bits, T = 256, 256, 2, 1, 128, (2, 4, 8), 6
+    cfg = B.Config(d, F, E, k, g, bits)
+    blobs = [B.pack_mwq(cfg, synth.normal(31, 100 + i, (F, d) if i % 3 < 2 else (d, F), 0.02, "cuda"))
+             for i in range(3 * E)]
+    x = synth.bf16_exact(synth.normal(31, 1, (T, d), 1.0, "cuda"))
+    logits = synth.normal(31, 5, (T, E), 1.0, "cuda")
+    fb = synth.categorical(31, 4, (T, k), [0.3, 0.3, 0.4], "cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_clean = B.moe_forward(cfg, x, blobs, logits=logits, forced_bit_idx=fb, device_status=st).clone()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    x_bad = x.clone()
+    x_bad[2, 5] = float("nan")
+    x_bad[4, 7] = float("inf")
+    y_bad = B.moe_forward(cfg, x_bad, blobs, logits=logits, forced_bit_idx=fb, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & 1                      # D2MOE_DEV_NONFINITE
+    keep = [0, 1, 3, 5]
+    assert torch.equal(y_bad[keep], y_clean[keep])
+    assert float(y_bad[[2, 4]].float().abs().max().item()) == 0.0
+
+
 def test_dense_ffn_single_expert(B):
     # E = 1, k = 1: a dense gated FFN read at a per-token width (the method applied to a dense model)
     cross, err = small_layer_case(B, d=384, F=512, E=1, k=1, g=128, bits=(2, 3, 4, 8), T=20)
