@@ -39,7 +39,8 @@ typedef enum {
 } d2moe_status;
 
 /* bits set in *device_status */
-#define D2MOE_DEV_NONFINITE 0x1
+#define D2MOE_DEV_NONFINITE 0x1  /* a router logit, or (decode kernel) an activation row, held a NaN or an
+                                    infinity; the outputs of such a row are zero                 */
 #define D2MOE_DEV_TIMEOUT   0x2
 #define D2MOE_DEV_BAD_INDEX 0x4  /* a supplied routing index was out of range and was skipped */
 
