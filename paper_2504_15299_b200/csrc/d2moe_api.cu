@@ -135,7 +135,13 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
         ws->off_src_token = take((size_t)pl.R_alloc * 4);
         ws->off_xp16 = take((size_t)pl.R_alloc * c->d_model * 2);
         ws->off_h = take((size_t)pl.R_alloc * c->d_ffn * 2);
-        ws->off_o = take((size_t)pl.n_split * pl.R_alloc * c->d_model * 4);
+        // the split-K factor of the down projection falls as the batch grows: size the partial outputs for
+        // the smallest batch that takes the same kernel, so that the total never shrinks when T grows
+        TcPlan pl_lo;
+        const long long t_dec = 64LL * c->n_experts / c->top_k;
+        tc_plan(c, pl.decode ? 1 : (t_dec + 1 < T ? t_dec + 1 : T), &pl_lo);
+        const int n_split_alloc = pl_lo.n_split > pl.n_split ? pl_lo.n_split : pl.n_split;
+        ws->off_o = take((size_t)n_split_alloc * pl.R_alloc * c->d_model * 4);
         ws->off_h32 = ws->off_xk_x = ws->off_xk_h = ws->off_slot_f = 0;
         if (pl.decode) {
             ws->off_h32 = take((size_t)pl.R_alloc * c->d_ffn * 4);
@@ -154,9 +160,18 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
 
 extern "C" size_t d2moe_workspace_bytes(const d2moe_config* c, int64_t max_tokens) {
     if (d2moe_check_config(c) != D2MOE_OK || max_tokens < 0 || max_tokens > (1 << 20)) return 0;
+    const long long T = max_tokens > 0 ? max_tokens : 1;
     Workspace ws;
-    d2moe_carve_workspace(c, max_tokens > 0 ? max_tokens : 1, &ws);
-    return ws.total;
+    d2moe_carve_workspace(c, T, &ws);
+    size_t total = ws.total;
+    // a call with fewer tokens may take the other expert kernel, whose buffers are laid out differently:
+    // cover the largest batch of that kind as well, so that every T <= max_tokens fits
+    const long long t_dec = 64LL * c->n_experts / c->top_k;      // largest batch the decode kernel takes
+    if (t_dec >= 1 && t_dec < T) {
+        d2moe_carve_workspace(c, t_dec, &ws);
+        if (ws.total > total) total = ws.total;
+    }
+    return total;
 }
 
 static d2moe_status check_route_inputs(const void* gate_w, const float* logits, const void* bit_w,

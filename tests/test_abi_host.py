@@ -88,6 +88,10 @@ def test_null_and_short_buffers_are_rejected_before_launch(lib):
     assert L.d2moe_unpack_codes(ctypes.byref(c), 4096, 64, 64, 1, 4096, None, None, None) == 3
     # workspace query
     assert binding.workspace_bytes(good(), 16) > 0
+    # a workspace sized for max_tokens serves every smaller batch, whichever expert kernel it takes
+    big = binding.Config(4096, 14336, 8, 2, 128, (2, 3, 4, 8))
+    sizes = [binding.workspace_bytes(big, t) for t in (1, 8, 64, 256, 257, 512, 2048)]
+    assert all(a <= b for a, b in zip(sizes, sizes[1:])), sizes
     bad = good(); bad.top_k = 9
     assert L.d2moe_workspace_bytes(ctypes.byref(bad.c()), 16) == 0
     # route: both / neither of gate_w and logits
