@@ -465,6 +465,22 @@ def test_decode_kernel_flags_nonfinite_activations(B):
     assert float(y_bad[[2, 4]].float().abs().max().item()) == 0.0
 
 
+def test_workspace_sized_for_a_larger_batch_serves_smaller_ones(B):
+    # one workspace sized for 300 tokens (grouped-GEMM kernel) also serves 1 and 16 tokens (decode kernel)
+    wl = synth.WORKLOADS["tiny"]
+    cfg = B.Config.from_workload(wl)
+    blobs = gpu_layer(B, cfg, wl)
+    gw = synth.gate_weight_bf16(wl, "cuda")
+    ws = torch.empty(B.workspace_bytes(cfg, 300), dtype=torch.uint8, device="cuda")
+    for T in (300, 16, 1):
+        x = synth.tokens_bf16(wl, T, "cuda")
+        fb = synth.forced_bit_idx(wl, T, "cuda")
+        y_shared = B.moe_forward(cfg, x, blobs, gate_w=gw, forced_bit_idx=fb, workspace=ws).clone()
+        y_own = B.moe_forward(cfg, x, blobs, gate_w=gw, forced_bit_idx=fb)
+        torch.cuda.synchronize()
+        assert torch.equal(y_shared, y_own)
+
+
 def test_dense_ffn_single_expert(B):
     # E = 1, k = 1: a dense gated FFN read at a per-token width (the method applied to a dense model)
     cross, err = small_layer_case(B, d=384, F=512, E=1, k=1, g=128, bits=(2, 3, 4, 8), T=20)
