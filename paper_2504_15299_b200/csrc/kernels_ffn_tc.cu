@@ -258,35 +258,52 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         }
     } else if (warp == WARP_MMA) {
         // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
+        // The issuer is a serial resource (one hand-off per tile), so everything an MMA needs is a register
+        // add away: per item the pieces' instruction descriptors, D columns and row offsets (an MMA covers at
+        // most 256 columns: a piece is at most two chunks); per stage the low word of the shared-memory
+        // descriptor (its high word is a constant).
+        constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
         uint32_t it = 0, at = 0, ic = 0;
+        const uint32_t slab_step = (uint32_t)p.n_cap * 8u;        // second 64-column slab of a stage, in 16-byte units
         for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
             const ItemInfo ii = decode_item(p, item);
             const TcUnit* u = p.units + ii.unit;
             const int kmax = u->kmax;
+            uint32_t id0[8], id1[8], dc[8], bo[8];                // chunk 0 / chunk 1 descriptors, D column, B rows / 16 B
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const int cnt = kk <= kmax ? u->cnt[kk] : 0;
+                const int col0 = u->col0[kk];
+                id0[kk] = cnt ? instr_desc_f16(min(cnt, 256)) : 0u;
+                id1[kk] = cnt > 256 ? instr_desc_f16(cnt - 256) : 0u;
+                dc[kk] = d_tmem + col0;
+                bo[kk] = (uint32_t)col0 * 8u;
+            }
             mbar_wait(D_EMPTY, (ic & 1) ^ 1, abort_flag, p.status);
             tc_fence_after();
             for (int G = ii.g0; G < ii.g1; ++G, ++it) {
                 const int s = it % NSB;
                 mbar_wait(B_FULL(s), (it / NSB) & 1, abort_flag, p.status);
-                const uint32_t bsl = bbuf + s * b_slot_bytes;
-                for (int kk = 0; kk <= kmax; ++kk) {
-                    const int cnt = u->cnt[kk];
-                    if (cnt == 0) continue;
-                    const int slot = at % A_SLOTS;
-                    mbar_wait(A_FULL(slot), (at / A_SLOTS) & 1, abort_flag, p.status);
-                    tc_fence_after();
-                    const int col0 = u->col0[kk];
-                    if (elect_one()) {
-                        for (int c = 0; c < cnt; c += 256) {          // an MMA covers at most 256 columns
-                            const int n = min(256, cnt - c);
-                            const uint32_t idesc = instr_desc_f16(n);
-                            const uint64_t bd = smem_desc_sw128(bsl + (uint32_t)(col0 + c) * 128u);
+                const uint32_t blo = (((bbuf + s * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
+                const uint32_t accum = (G != ii.g0) ? 1u : 0u;
 #pragma unroll
-                            for (int j = 0; j < GS / 16; ++j) {
-                                const uint32_t a_addr = a_tmem + slot * 64 + j * 8;
-                                const uint64_t bj = bd + (uint64_t)(((j >> 2) * (uint32_t)p.n_cap * 128u + (j & 3) * 32u) >> 4);
-                                tc_mma_ts(d_tmem + col0 + c, a_addr, bj, idesc, (G != ii.g0 || j != 0) ? 1u : 0u);
-                            }
+                for (int kk = 0; kk < 8; ++kk) {
+                    if (id0[kk] == 0u) continue;
+                    const uint32_t slot = at & 1u;
+                    mbar_wait(A_FULL(slot), (at >> 1) & 1u, abort_flag, p.status);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint32_t a_addr = a_tmem + slot * 64;
+                        const uint32_t lo = blo + bo[kk];
+#pragma unroll
+                        for (int j = 0; j < GS / 16; ++j)
+                            tc_mma_ts_lohi(dc[kk], a_addr + j * 8, lo + (j >> 2) * slab_step + (j & 3) * 2, DESC_HI, id0[kk],
+                                           j == 0 ? accum : 1u);
+                        if (id1[kk] != 0u) {
+#pragma unroll
+                            for (int j = 0; j < GS / 16; ++j)
+                                tc_mma_ts_lohi(dc[kk] + 256, a_addr + j * 8, lo + 256 * 8 + (j >> 2) * slab_step + (j & 3) * 2, DESC_HI,
+                                               id1[kk], j == 0 ? accum : 1u);
                         }
                         tc_commit(A_EMPTY(slot));
                     }
@@ -334,7 +351,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 for (int kk = 0; kk <= kmax; ++kk) {
                     const int sw = p.L.seg_sw[kk];
                     // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
-                    const float Mk = s1 * exp2f((float)(-(p.D.bits[kk] - p.D.bits[0]))) * two_mS;
+                    const float Mk = s1 * __int_as_float((127 - (p.D.bits[kk] - p.D.bits[0])) << 23) * two_mS;
                     const __half2 m0 = h2dup(Mk * 16777216.0f);
                     const uint32_t seg = wb + (uint32_t)p.L.seg_off[kk];
                     if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
