@@ -481,6 +481,17 @@ def test_workspace_sized_for_a_larger_batch_serves_smaller_ones(B):
         assert torch.equal(y_shared, y_own)
 
 
+@pytest.mark.parametrize("case", [
+    dict(d=512, F=512, E=128, k=8, g=128, bits=(2, 4, 8), T=64, n_shared=2),        # many experts, few tokens each
+    dict(d=256, F=384, E=4, k=2, g=128, bits=(1, 2, 3, 4, 5, 6, 7, 8), T=700),      # eight widths, grouped-GEMM kernel
+    dict(d=256, F=256, E=2, k=2, g=64, bits=(2, 4, 8), T=3000),                     # many units per expert, g = 64
+    dict(d=384, F=640, E=16, k=4, g=128, bits=(5, 6, 7, 8), T=200, n_shared=1),     # 50 tokens per expert: decode kernel, several units
+])
+def test_stress_shapes(B, case):
+    cross, err = small_layer_case(B, **case)
+    assert cross < TOL and err < TOL, (cross, err)
+
+
 def test_dense_ffn_single_expert(B):
     # E = 1, k = 1: a dense gated FFN read at a per-token width (the method applied to a dense model)
     cross, err = small_layer_case(B, d=384, F=512, E=1, k=1, g=128, bits=(2, 3, 4, 8), T=20)
