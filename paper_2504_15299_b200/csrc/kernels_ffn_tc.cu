@@ -179,6 +179,14 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // per-width constants of the dequant loop, read from shared memory instead of the kernel parameters
+    // (a dynamically indexed parameter read costs a constant-cache round trip per tile)
+    int4* seg_tab = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + 256);   // {sw, seg_off, 2^-(bits[kk]-bits[0]) bits, 0}
+    if (threadIdx.x < 8) {
+        const int kk = threadIdx.x;
+        const int db = kk < p.D.K ? p.D.bits[kk] - p.D.bits[0] : 0;
+        seg_tab[kk] = make_int4(p.L.seg_sw[kk], p.L.seg_off[kk], (127 - db) << 23, 0);
+    }
     if (warp == WARP_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
@@ -324,7 +332,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         const int r = threadIdx.x & 127;         // row of the tile = TMEM lane
         const int blk = r >> 6, rr = r & 63;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
-        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * EPI_STRIDE);
+        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (128 * 9);
         uint32_t it = 0, at = 0, ic = 0;
         __half2 acc[GS / 4];
         for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
@@ -349,11 +357,12 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 const __half2 u0 = h2dup((lo - 0.5f * s1) * two_mS);
 #pragma unroll 1
                 for (int kk = 0; kk <= kmax; ++kk) {
-                    const int sw = p.L.seg_sw[kk];
+                    const int4 tb = seg_tab[kk];
+                    const int sw = tb.x;
                     // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
-                    const float Mk = s1 * __int_as_float((127 - (p.D.bits[kk] - p.D.bits[0])) << 23) * two_mS;
+                    const float Mk = s1 * __int_as_float(tb.z) * two_mS;
                     const __half2 m0 = h2dup(Mk * 16777216.0f);
-                    const uint32_t seg = wb + (uint32_t)p.L.seg_off[kk];
+                    const uint32_t seg = wb + (uint32_t)tb.y;
                     if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
                     else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
                     if ((present >> kk) & 1u) {
@@ -379,15 +388,24 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             }
 
             // ---- epilogue: D (128 rows x ncols) -> global; the two warpgroups take alternate 16-column chunks ----
+            // While it runs the tensor pipe is idle, so it is kept short: the pieces' extents are read once,
+            // and SwiGLU is split between the two threads of a hidden unit (the gate row's thread finishes the
+            // first eight tokens of a chunk, the up row's thread the other eight).
+            int pc0[8], pcn[8], prl[8];                          // per piece: first column, columns, real columns
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                pc0[kk] = u->col0[kk]; pcn[kk] = kk <= kmax ? u->cnt[kk] : 0; prl[kk] = u->real[kk];
+            }
             mbar_wait(D_FULL, ic & 1, abort_flag, p.status);
             tc_fence_after();
             const float two_S = exp2f((float)S);
             const int ncols = u->ncols;
             for (int c0 = wg * 16; c0 < ncols; c0 += 32) {
                 int nreal = 0;
-                for (int kk = 0; kk <= kmax; ++kk) {
-                    const int rel = c0 - u->col0[kk];
-                    if (u->cnt[kk] > 0 && rel >= 0 && rel < u->cnt[kk]) nreal = min(16, max(0, u->real[kk] - rel));
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const int rel = c0 - pc0[kk];
+                    if (pcn[kk] > 0 && rel >= 0 && rel < pcn[kk]) nreal = min(16, max(0, prl[kk] - rel));
                 }
                 if (nreal == 0) continue;            // padding columns only (uniform across the warpgroup)
                 uint32_t v[16];
@@ -395,20 +413,20 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 tc_wait_ld();
                 const long long grow = u->row0 + c0;
                 if (p.mode == 0) {
-                    if (blk == 1) {
+                    // exchange: the gate thread publishes tokens 8..15, the up thread tokens 0..7
+                    const int give = blk == 0 ? 8 : 0;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) epi[rr * EPI_STRIDE + j] = __uint_as_float(v[j]) * two_S;
-                    }
+                    for (int j = 0; j < 8; ++j) epi[(blk * 64 + rr) * 9 + j] = __uint_as_float(v[give + j]) * two_S;
                     asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
-                    if (blk == 0) {
-                        __half* dst = p.hbuf + grow * p.D.F + (long long)ii.tile * 64 + rr;
+                    const int keep = blk == 0 ? 0 : 8;           // the tokens this thread finishes
+                    __half* dst = p.hbuf + (grow + keep) * p.D.F + (long long)ii.tile * 64 + rr;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (j < nreal) {
-                                const float g = __uint_as_float(v[j]) * two_S;
-                                const float up = epi[rr * EPI_STRIDE + j];
-                                dst[(long long)j * p.D.F] = __float2half_rn(g / (1.0f + __expf(-g)) * up);
-                            }
+                    for (int j = 0; j < 8; ++j) {
+                        if (keep + j < nreal) {
+                            const float mine = __uint_as_float(v[keep + j]) * two_S;
+                            const float other = epi[((1 - blk) * 64 + rr) * 9 + j];
+                            const float g = blk == 0 ? mine : other, up = blk == 0 ? other : mine;
+                            dst[(long long)j * p.D.F] = __float2half_rn(__fdividef(g, 1.0f + __expf(-g)) * up);
                         }
                     }
                     asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
@@ -602,7 +620,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
         const int b_bytes = NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
-        const int epi_bytes = 2 * 64 * EPI_STRIDE * 4;
+        const int epi_bytes = 2 * 128 * 9 * 4;            // per warpgroup: 128 rows x 8 exchanged values (+1 pad)
         const int bar_bytes = 512;
         const int budget = 224 * 1024;
         int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
