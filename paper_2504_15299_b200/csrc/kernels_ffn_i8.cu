@@ -185,17 +185,7 @@ __device__ __forceinline__ void unpack_dispatch(int sw, uint32_t seg, int rr, in
     }
 }
 
-// Compile-time description of a width list of at most four segments: nibble j of WPACK is the logical
-// width of segment j (stored 1, 2, 4 or 8 bits wide).  WPACK == 0 selects the run-time path.
-template <int WPACK>
-struct I8SegList {
-    __host__ __device__ static constexpr int w(int j) { return (WPACK >> (4 * j)) & 15; }
-    __host__ __device__ static constexpr int sw(int j) { return w(j) <= 1 ? 1 : (w(j) <= 2 ? 2 : (w(j) <= 4 ? 4 : 8)); }
-    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && w(k) != 0) ++k; return k; }
-    __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += w(i); return b; }
-    __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += w(i); return top() - b; }
-    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
-};
+template <int WPACK> using I8SegList = WidthList<WPACK>;
 
 // Output phase of one work item for one thread: scales the folded sums by the tokens' activation
 // scales, applies SwiGLU across the gate / up halves of the tile (mode 0) and writes the result.

@@ -33,6 +33,8 @@
 #include "kernels_ffn_tc.cuh"
 #include "tc_common.cuh"
 
+#include <type_traits>
+
 namespace {
 
 constexpr int TC_THREADS = 352;        // 8 dequant warps (2 warpgroups) + weight producer + activation producer + MMA issuer
@@ -140,7 +142,7 @@ __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
-template <int GS>
+template <int GS, int WPACK>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMaps maps) {
     constexpr int HALVES = GS / 64;              // 64-element K slabs of the activation tile
@@ -355,33 +357,56 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 const __half2 mh = as_h2(meta);
                 const float s1 = __low2float(mh), lo = __high2float(mh);
                 const __half2 u0 = h2dup((lo - 0.5f * s1) * two_mS);
-#pragma unroll 1
-                for (int kk = 0; kk <= kmax; ++kk) {
-                    const int4 tb = seg_tab[kk];
-                    const int sw = tb.x;
-                    // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
-                    const float Mk = s1 * __int_as_float(tb.z) * two_mS;
-                    const __half2 m0 = h2dup(Mk * 16777216.0f);
-                    const uint32_t seg = wb + (uint32_t)tb.y;
-                    if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
-                    else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
-                    if ((present >> kk) & 1u) {
-                        const int slot = at % A_SLOTS;
-                        mbar_wait(A_EMPTY(slot), ((at / A_SLOTS) & 1) ^ 1, abort_flag, p.status);
-                        tc_fence_after();
-                        const __half2 half_m = h2dup(0.5f * Mk);
-                        const uint32_t dst = a_tmem + slot * 64 + wg * (TILE_COLS / 2) + lane_addr;
+                // hands the running tile over as the tile of width index kk (Mk = M_kk * 2^-S)
+                auto write_tile = [&](float Mk) {
+                    const int slot = at % A_SLOTS;
+                    mbar_wait(A_EMPTY(slot), ((at / A_SLOTS) & 1) ^ 1, abort_flag, p.status);
+                    tc_fence_after();
+                    const __half2 half_m = h2dup(0.5f * Mk);
+                    const uint32_t dst = a_tmem + slot * 64 + wg * (TILE_COLS / 2) + lane_addr;
 #pragma unroll
-                        for (int c = 0; c < GS / 64; ++c) {
-                            uint32_t v[16];
+                    for (int c = 0; c < GS / 64; ++c) {
+                        uint32_t v[16];
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) v[j] = as_u32(__hadd2(acc[c * 16 + j], half_m));
-                            tc_st16(dst + c * 16, v);
+                        for (int j = 0; j < 16; ++j) v[j] = as_u32(__hadd2(acc[c * 16 + j], half_m));
+                        tc_st16(dst + c * 16, v);
+                    }
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(A_FULL(slot));
+                    ++at;
+                };
+                if constexpr (WPACK != 0) {
+                    // compile-time width list: storage widths, segment offsets and scale ratios are immediates
+                    using WL = WidthList<WPACK>;
+                    auto seg_step = [&](auto jc) {
+                        constexpr int J = decltype(jc)::value;
+                        if constexpr (J < WL::count()) {
+                            if (J <= kmax) {
+                                constexpr int db = WL::top() - WL::pos(J) - WL::w(0);      // bits[J] - bits[0]
+                                const float Mk = s1 * __int_as_float((127 - db) << 23) * two_mS;
+                                dequant_segment<GS, WL::sw(J), J == 0>(wb + (uint32_t)WL::seg_off(GS, J), rr, wg, acc,
+                                                                      h2dup(Mk * 16777216.0f), u0);
+                                if ((present >> J) & 1u) write_tile(Mk);
+                            }
                         }
-                        tc_wait_st();
-                        tc_fence_before();
-                        mbar_arrive(A_FULL(slot));
-                        ++at;
+                    };
+                    seg_step(std::integral_constant<int, 0>{});
+                    seg_step(std::integral_constant<int, 1>{});
+                    seg_step(std::integral_constant<int, 2>{});
+                    seg_step(std::integral_constant<int, 3>{});
+                } else {
+#pragma unroll 1
+                    for (int kk = 0; kk <= kmax; ++kk) {
+                        const int4 tb = seg_tab[kk];
+                        const int sw = tb.x;
+                        // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
+                        const float Mk = s1 * __int_as_float(tb.z) * two_mS;
+                        const __half2 m0 = h2dup(Mk * 16777216.0f);
+                        const uint32_t seg = wb + (uint32_t)tb.y;
+                        if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
+                        else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
+                        if ((present >> kk) & 1u) write_tile(Mk);
                     }
                 }
                 mbar_arrive(W_EMPTY(s));
@@ -632,16 +657,22 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;   // + slack for the 1024-byte alignment
         mark(mode == 0 ? 1 : 2);
+        // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
+        int wpack = 0;
+        if (p.L.n_seg <= 4)
+            for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
+        auto launch = [&](auto kern) -> cudaError_t {
+            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (err != cudaSuccess) return err;
+            kern<<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            return cudaSuccess;
+        };
         cudaError_t e;
-        if (D.g == 128) {
-            e = cudaFuncSetAttribute(ffn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            if (e != cudaSuccess) return e;
-            ffn_tc_kernel<128><<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
-        } else {
-            e = cudaFuncSetAttribute(ffn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-            if (e != cudaSuccess) return e;
-            ffn_tc_kernel<64><<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
-        }
+        if (D.g == 128 && wpack == 0x4112) e = launch(ffn_tc_kernel<128, 0x4112>);        // {2,3,4,8}
+        else if (D.g == 128 && wpack == 0x422) e = launch(ffn_tc_kernel<128, 0x422>);     // {2,4,8}
+        else if (D.g == 128) e = launch(ffn_tc_kernel<128, 0>);
+        else e = launch(ffn_tc_kernel<64, 0>);
+        if (e != cudaSuccess) return e;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

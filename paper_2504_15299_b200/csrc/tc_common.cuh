@@ -163,6 +163,18 @@ __device__ __forceinline__ __half2 h2dup(float v) { return __float2half2_rn(v); 
 __device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 __device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
+// Compile-time description of a width list of at most four segments: nibble j of WPACK is the logical
+// width of segment j (stored 1, 2, 4 or 8 bits wide).  WPACK == 0 selects the run-time path.
+template <int WPACK>
+struct WidthList {
+    __host__ __device__ static constexpr int w(int j) { return (WPACK >> (4 * j)) & 15; }
+    __host__ __device__ static constexpr int sw(int j) { return w(j) <= 1 ? 1 : (w(j) <= 2 ? 2 : (w(j) <= 4 ? 4 : 8)); }
+    __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && w(k) != 0) ++k; return k; }
+    __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += w(i); return b; }
+    __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += w(i); return top() - b; }
+    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
+};
+
 // exponent S of the common factor 2^-S from the header of a packed matrix
 __device__ __forceinline__ int matrix_exponent(const uint8_t* packed) {
     const PackHeader* h = reinterpret_cast<const PackHeader*>(packed);
