@@ -543,7 +543,7 @@ def run_ours(args):
     # arithmetic type of the expert kernels: the decode kernel multiplies unsigned 8-bit codes with signed
     # 8-bit activation halves (int32 accumulation, fp32 scaling), the grouped GEMM runs on fp16 tiles
     dtype = "f32" if args.path == "cuda_core" else "i8"
-    if -(-T * wl.top_k // wl.n_experts) > 64 and args.path != "cuda_core":
+    if -(-T * wl.top_k // wl.n_experts) > 40 and args.path != "cuda_core":
         dtype = "f16"
         A_tot = T * (wl.top_k + wl.n_shared)
         flops = {"gate_up": A_tot * 2 * 2 * wl.d_model * wl.d_ffn, "down": A_tot * 2 * wl.d_model * wl.d_ffn}

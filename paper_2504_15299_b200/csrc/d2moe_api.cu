@@ -138,7 +138,7 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
         // the split-K factor of the down projection falls as the batch grows: size the partial outputs for
         // the smallest batch that takes the same kernel, so that the total never shrinks when T grows
         TcPlan pl_lo;
-        const long long t_dec = 64LL * c->n_experts / c->top_k;
+        const long long t_dec = (long long)D2MOE_DECODE_MAX_AVG * c->n_experts / c->top_k;
         tc_plan(c, pl.decode ? 1 : (t_dec + 1 < T ? t_dec + 1 : T), &pl_lo);
         const int n_split_alloc = pl_lo.n_split > pl.n_split ? pl_lo.n_split : pl.n_split;
         ws->off_o = take((size_t)n_split_alloc * pl.R_alloc * c->d_model * 4);
@@ -166,7 +166,7 @@ extern "C" size_t d2moe_workspace_bytes(const d2moe_config* c, int64_t max_token
     size_t total = ws.total;
     // a call with fewer tokens may take the other expert kernel, whose buffers are laid out differently:
     // cover the largest batch of that kind as well, so that every T <= max_tokens fits
-    const long long t_dec = 64LL * c->n_experts / c->top_k;      // largest batch the decode kernel takes
+    const long long t_dec = (long long)D2MOE_DECODE_MAX_AVG * c->n_experts / c->top_k;      // largest batch the decode kernel takes
     if (t_dec >= 1 && t_dec < T) {
         d2moe_carve_workspace(c, t_dec, &ws);
         if (ws.total > total) total = ws.total;

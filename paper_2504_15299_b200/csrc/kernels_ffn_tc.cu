@@ -589,9 +589,9 @@ bool tc_path_supported(const d2moe_config* c) {
 void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     const long long A = T * c->top_k, A_tot = A + T * c->n_shared;
     const long long avg = (A + c->n_experts - 1) / c->n_experts;
-    // up to about 64 tokens per expert the 8-bit kernel (units of 32 slots, weights unpacked once per unit) is
-    // faster than the fp16 grouped GEMM (measured crossover on the Mixtral shape: between 64 and 96)
-    pl->decode = avg <= 64 ? 1 : 0;
+    // up to about 40 tokens per expert the 8-bit kernel (units of 32 slots, weights unpacked once per unit) is
+    // faster than the fp16 grouped GEMM (measured crossover on the Mixtral shape: T = 160, 40 tokens per expert)
+    pl->decode = avg <= D2MOE_DECODE_MAX_AVG ? 1 : 0;
     if (pl->decode) {
         pl->n_cap = 32;                      // token slots per unit
     } else {

@@ -26,6 +26,9 @@ struct I8Unit {
     int blk[8];    // the real blocks: first slot / 4, relative to slot0
 };
 
+// largest average number of tokens per expert that the 8-bit decode kernel takes
+#define D2MOE_DECODE_MAX_AVG 40
+
 struct TcPlan {
     int decode;             // 1: memory-bound 8-bit decode kernel (tokens laid out widest first, scales applied
                             //    to the accumulators); 0: grouped fp16 dequant-GEMM (one tile per width, any load)
