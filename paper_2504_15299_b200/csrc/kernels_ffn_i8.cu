@@ -191,7 +191,8 @@ template <int WPACK> using I8SegList = WidthList<WPACK>;
 // scales, applies SwiGLU across the gate / up halves of the tile (mode 0) and writes the result.
 // blks: byte i = first slot / 4 of the thread's block i.
 static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, int wg, int r, int n_mine, uint32_t blks,
-                                                 float (&acc)[4][4], float* epi) {
+                                                 float (&acc)[4][4], uint8_t* smem) {
+    float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
     const I8Item io = i8_item(p, item);
     const int slot0 = p.units[io.unit].slot0;
     const int blk = r >> 6, rr = r & 63;
@@ -263,9 +264,9 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     auto A_EMPTY = [&](int wg, int sl) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 4 + wg * 2 + sl); };
     auto D_FULL = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 8 + b); };
     auto D_EMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 10 + b); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * I8_MAX_NSW + 2 * I8_NSB + 12);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    const uint32_t abort_addr = smem_u32(tmem_slot + 1);
+    // tail of the 512-byte barrier block: TMEM base (488), device-status pointer (496), abort flag (504)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 488);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 504);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -278,6 +279,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
         *abort_flag = 0;
+        *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -319,7 +321,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                     const int ng = min(GPS, ii.g1 - G);
                     {
                         const int s = it % nsw;
-                        { I8S_T0(); mbar_wait_ptx(W_EMPTY(s), ((it / nsw) & 1) ^ 1, abort_addr, p.status); I8S_ADD(0); }
+                        { I8S_T0(); mbar_wait_blk(W_EMPTY(s), ((it / nsw) & 1) ^ 1); I8S_ADD(0); }
                         mbar_expect_tx(W_FULL(s), 2 * bytes * ng);
                         const uint32_t dst = wbuf + s * w_slot_bytes;
                         for (int sub = 0; sub < ng; ++sub) {
@@ -329,7 +331,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                     }
                     {
                         const int s = it % I8_NSB;
-                        { I8S_T0(); mbar_wait_ptx(B_EMPTY(s), ((it / I8_NSB) & 1) ^ 1, abort_addr, p.status); I8S_ADD(1); }
+                        { I8S_T0(); mbar_wait_blk(B_EMPTY(s), ((it / I8_NSB) & 1) ^ 1); I8S_ADD(1); }
                         mbar_expect_tx(B_FULL(s), tile_bytes + ng * xk_bytes);
                         tma_load_2d(bbuf + s * I8_B_TILE, &maps.m[mi], G * GS, 2 * slot0, B_FULL(s));
                         for (int sub = 0; sub < ng; ++sub)
@@ -367,13 +369,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int j = 0; j < 8; ++j) idesc[j] = instr_desc_i8(2 * max(u->npad[j], 8));
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
-                { I8S_T0(); mbar_wait_ptx(B_FULL(bs), bph, abort_addr, p.status); I8S_ADD(3); }
+                { I8S_T0(); mbar_wait_blk(B_FULL(bs), bph); I8S_ADD(3); }
                 const uint64_t bdesc = smem_desc_sw128(bbuf + bs * I8_B_TILE);
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
                     if (sub < ng && !I8_STREAM_ONLY) {
                         const int buf = gc & 1;
-                        { I8S_T0(); mbar_wait_ptx(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1, abort_addr, p.status); I8S_ADD(2); }
+                        { I8S_T0(); mbar_wait_blk(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1); I8S_ADD(2); }
                         tc_fence_after();
                         const uint32_t d_addr = d_tmem + buf * I8_D_COLS;
 #pragma unroll
@@ -382,7 +384,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                             for (int wg = 0; wg < 2; ++wg) {
                                 const int j0 = wg + 4 * hp, j1 = j0 + 2;
                                 if (j0 <= kmax) {
-                                    { I8S_T0(); mbar_wait_ptx(A_FULL(wg, 0), hs[wg] & 1, abort_addr, p.status); I8S_ADD(4); }
+                                    { I8S_T0(); mbar_wait_blk(A_FULL(wg, 0), hs[wg] & 1); I8S_ADD(4); }
                                     tc_fence_after();
                                     const uint32_t a_addr = a_tmem + wg * 64;
                                     if (elect_one()) {
@@ -429,14 +431,11 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
         const int blk = r >> 6, rr = r & 63;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
-        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
         const uint32_t a_base = a_tmem + wg * 64 + lane_addr;          // my two operand tiles: +0, +32
         const uint32_t d_base = d_tmem + lane_addr;
-        const uint32_t AF = A_FULL(wg, 0), AE = A_EMPTY(wg, 0);
-        const uint32_t w_addr0 = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
         uint32_t gc = 0, hs = 0;                   // groups folded / operand hand-offs so far
         uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
-        uint32_t w_addr = w_addr0;
+        uint32_t w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
         I8S_DECL();
 #ifdef D2MOE_WAIT_STATS
         const long long _tt = clock64();
@@ -461,13 +460,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             // (bits 0-1), phase (bit 2), last group of its stage (bit 3), group inside the stage (bit 4)
             auto fold = [&](uint32_t g, uint32_t pb, uint32_t meta) {
                 const int buf = g & 1;
-                { I8S_T0(); mbar_wait_ptx(D_FULL(buf), (g >> 1) & 1, abort_addr, p.status); I8S_ADD(9); }
+                { I8S_T0(); mbar_wait_blk(D_FULL(buf), (g >> 1) & 1); I8S_ADD(9); }
                 tc_fence_after();
                 I8S_T0();
                 const __half2 mh = as_h2(meta);
                 const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
                 const float lo = __high2float(mh);
-                mbar_wait_ptx(B_FULL(pb & 3), (pb >> 2) & 1, abort_addr, p.status);
+                mbar_wait_blk(B_FULL(pb & 3), (pb >> 2) & 1);
                 const uint32_t xk_addr = xkbuf + ((pb & 3) * 2 + (pb >> 4)) * I8_XK_BYTES;
                 // two rounds of two blocks: 16 accumulator registers in flight instead of 32
 #pragma unroll
@@ -507,7 +506,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             uint32_t pend_pb = 0, pend_meta = 0;
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
-                { I8S_T0(); mbar_wait_ptx(W_FULL(ws), wph, abort_addr, p.status); I8S_ADD(6); }
+                { I8S_T0(); mbar_wait_blk(W_FULL(ws), wph); I8S_ADD(6); }
                 if (I8_STREAM_ONLY) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B_EMPTY(bs));
@@ -519,13 +518,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         uint32_t meta;
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
                         auto handoff_begin = [&]() {
-                            { I8S_T0(); mbar_wait_ptx(AE, (hs & 1) ^ 1, abort_addr, p.status); I8S_ADD(7); }
+                            { I8S_T0(); mbar_wait_blk(A_EMPTY(wg, 0), (hs & 1) ^ 1); I8S_ADD(7); }
                             tc_fence_after();
                         };
                         auto handoff_end = [&]() {
                             { I8S_T0(); tc_wait_st(); I8S_ADD(8); }
                             tc_fence_before();
-                            mbar_arrive(AF);
+                            mbar_arrive(A_FULL(wg, 0));
                             ++hs;
                         };
                         if constexpr (SWPACK != 0) {
@@ -573,7 +572,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 }
                 mbar_arrive(W_EMPTY(ws));
                 w_addr += w_slot_bytes;
-                if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = w_addr0; }
+                if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
                 if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
             }
             if (pend) fold(gc - 1, pend_pb, pend_meta);
@@ -585,7 +584,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int q = 0; q < 4; ++q) out[i][q] = acc[i][q];
-            i8_write_out(p, item, wg, r, n_mine, myblks, out, epi);
+            i8_write_out(p, item, wg, r, n_mine, myblks, out, smem);
             I8S_ADD(14);
         }
 #ifdef D2MOE_WAIT_STATS
@@ -864,7 +863,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         p.nsw = nsw;
         p.smem_w_off = b_bytes;
         p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
-        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 511) & ~511;   // 512-byte aligned from the 1024-byte aligned base
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         if (mode == 1)
             i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,

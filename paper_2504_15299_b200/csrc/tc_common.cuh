@@ -103,6 +103,37 @@ __device__ __forceinline__ void mbar_wait_ptx(uint32_t bar, uint32_t parity, uin
         ::"r"(bar), "r"(parity), "r"(abort_addr), "l"(status) : "memory");
 }
 
+// The same for kernels whose barrier block is 512-byte aligned and keeps the abort flag at byte 504 and
+// the device-status pointer at byte 496 of that block: the slow path finds both from the barrier's own
+// address, so a wait keeps no register alive besides the barrier address and the parity.
+__device__ __forceinline__ void mbar_wait_blk(uint32_t bar, uint32_t parity) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u32 ab, blk;\n\t"
+        ".reg .u64 t0, t1, st;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%0], %1;\n\t"
+        "@p bra WAITB_DONE;\n\t"
+        "and.b32 blk, %0, 0xFFFFFE00;\n\t"
+        "mov.u64 t0, %%globaltimer;\n"
+        "WAITB_RETRY:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%0], %1, 4000;\n\t"
+        "@p bra WAITB_DONE;\n\t"
+        "ld.volatile.shared.u32 ab, [blk+504];\n\t"
+        "setp.ne.u32 q, ab, 0;\n\t"
+        "@q bra WAITB_DONE;\n\t"
+        "mov.u64 t1, %%globaltimer;\n\t"
+        "sub.u64 t1, t1, t0;\n\t"
+        "setp.lt.u64 q, t1, 1000000000;\n\t"
+        "@q bra WAITB_RETRY;\n\t"
+        "st.volatile.shared.u32 [blk+504], 1;\n\t"
+        "ld.shared.u64 st, [blk+496];\n\t"
+        "red.global.or.b32 [st], 2;\n"    // D2MOE_DEV_TIMEOUT
+        "WAITB_DONE:\n\t"
+        "}"
+        ::"r"(bar), "r"(parity) : "memory");
+}
+
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
