@@ -137,8 +137,8 @@ __device__ __forceinline__ void unpack_segment(uint32_t seg, int rr, int W, int 
     constexpr int NCELL = GS / 4;
     const uint32_t mask = (((1u << W) - 1u) << P) * 0x01010101u;
 
-    constexpr int NB = NCELL / 16;                           // batches of 16 cells = one tcgen05.st
-    constexpr int WPB = 16 / CPW;                            // words per batch: 8, 4, 2 for SW = 4, 2, 1 (16 for 8)
+    constexpr int NB = NCELL / 8;                            // batches of 8 cells = one tcgen05.st (few live registers)
+    constexpr int WPB = 8 / CPW;                             // words per batch: 4, 2, 1 for SW = 4, 2, 1 (8 for 8)
     constexpr int NW = NLD * WPL;
     // words are loaded batch by batch when a batch spans whole loads, otherwise once for all batches
     constexpr bool PER_BATCH = WPB >= WPL;
@@ -163,15 +163,15 @@ __device__ __forceinline__ void unpack_segment(uint32_t seg, int rr, int W, int 
 #pragma unroll
             for (int l = 0; l < WPB / WPL; ++l) load(b * (WPB / WPL) + l, w + l * WPL);
         }
-        uint32_t v[16];
+        uint32_t v[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int cell = b * 16 + i, q = PER_BATCH ? i / CPW : cell / CPW, u = cell % CPW;
+        for (int i = 0; i < 8; ++i) {
+            const int cell = b * 8 + i, q = PER_BATCH ? i / CPW : cell / CPW, u = cell % CPW;
             const int sh = P - SW * u;                       // compile-time sign when P is a constant
             const uint32_t moved = sh >= 0 ? (w[q] << (sh & 31)) : (w[q] >> ((-sh) & 31));
             v[i] = moved & mask;
         }
-        tc_st16(taddr + b * 16, v);
+        tc_st8(taddr + b * 8, v);
     }
 }
 
