@@ -433,9 +433,10 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     } else
     route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
-    // few assignments and keys: histogram, scan and scatter in one single-block launch
+    // few assignments and keys: histogram, scan and scatter in one single-block launch (beyond about a
+    // thousand warp walks the three grid-wide kernels are faster: 39 vs 10 us at 192 keys x 1536 assignments)
     const long long walks = (long long)n_keys * ((D.A + 31) / 32);
-    if (D.A <= 8192 && n_keys <= 2048 && walks <= 16384) {
+    if (D.A <= 8192 && n_keys <= 2048 && walks <= 1024) {
         const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
         group_small_kernel<<<1, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
         return cudaGetLastError();
