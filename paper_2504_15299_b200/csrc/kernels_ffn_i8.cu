@@ -303,40 +303,58 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // One producer thread feeds both rings, stage by stage (they are consumed at the same rate).
         if (lane == 0) {
             I8S_DECL();
-            uint32_t it = 0;
+            // This thread shares a scheduler with unpack warps, so its loop is kept short: source pointers and
+            // ring positions advance by addition, nothing is recomputed per stage.
+            uint32_t it = 0, ws = 0, wph = 1, bs = 0, bph = 1;         // ring positions, parity of the "empty" waits
             for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
                 const I8Item ii = i8_item(p, item);
                 const I8Unit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
                 const uint32_t bytes = (uint32_t)p.L.seg_off[kmax + 1];
                 const uint8_t *m0, *m1;
-                int rt0, rt1;
-                if (p.mode == 0) { m0 = p.P.w[3 * e + 0]; m1 = p.P.w[3 * e + 1]; rt0 = rt1 = ii.tile; }
-                else { m0 = m1 = p.P.w[3 * e + 2]; rt0 = 2 * ii.tile; rt1 = 2 * ii.tile + 1; }
+                if (p.mode == 0) {
+                    m0 = p.P.w[3 * e + 0] + d2moe_block_offset(p.L, ii.tile, ii.g0);
+                    m1 = p.P.w[3 * e + 1] + d2moe_block_offset(p.L, ii.tile, ii.g0);
+                } else {
+                    m0 = p.P.w[3 * e + 2] + d2moe_block_offset(p.L, 2 * ii.tile, ii.g0);
+                    m1 = p.P.w[3 * e + 2] + d2moe_block_offset(p.L, 2 * ii.tile + 1, ii.g0);
+                }
                 const int nslots = u->nslots, slot0 = u->slot0;
                 const int mi = nslots <= 8 ? 0 : (nslots <= 16 ? 1 : 2);        // boxes of 16, 32, 64 rows
                 const uint32_t tile_bytes = (16u << mi) * 128u;
                 const uint32_t xk_bytes = (uint32_t)nslots * 8u;
+                const uint32_t bb = (uint32_t)p.L.block_bytes;
+                const float* xk_src = p.xk + ((long long)ii.g0 * p.R_alloc + slot0) * 2;
+                const long long xk_step = p.R_alloc * 2;
+                const CUtensorMap* map = &maps.m[mi];
                 for (int G = ii.g0; G < ii.g1; G += GPS, ++it) {
                     const int ng = min(GPS, ii.g1 - G);
                     {
-                        const int s = it % nsw;
-                        { I8S_T0(); mbar_wait_blk(W_EMPTY(s), ((it / nsw) & 1) ^ 1); I8S_ADD(0); }
-                        mbar_expect_tx(W_FULL(s), 2 * bytes * ng);
-                        const uint32_t dst = wbuf + s * w_slot_bytes;
-                        for (int sub = 0; sub < ng; ++sub) {
-                            bulk_g2s(dst + (2 * sub) * p.L.block_bytes, m0 + d2moe_block_offset(p.L, rt0, G + sub), bytes, W_FULL(s));
-                            bulk_g2s(dst + (2 * sub + 1) * p.L.block_bytes, m1 + d2moe_block_offset(p.L, rt1, G + sub), bytes, W_FULL(s));
+                        { I8S_T0(); mbar_wait_blk(W_EMPTY(ws), wph); I8S_ADD(0); }
+                        mbar_expect_tx(W_FULL(ws), 2 * bytes * ng);
+                        const uint32_t dst = wbuf + ws * w_slot_bytes;
+#pragma unroll
+                        for (int sub = 0; sub < GPS; ++sub) {
+                            if (sub < ng) {
+                                bulk_g2s(dst + (2 * sub) * bb, m0, bytes, W_FULL(ws));
+                                bulk_g2s(dst + (2 * sub + 1) * bb, m1, bytes, W_FULL(ws));
+                                m0 += bb; m1 += bb;
+                            }
                         }
+                        if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1u; }
                     }
                     {
-                        const int s = it % I8_NSB;
-                        { I8S_T0(); mbar_wait_blk(B_EMPTY(s), ((it / I8_NSB) & 1) ^ 1); I8S_ADD(1); }
-                        mbar_expect_tx(B_FULL(s), tile_bytes + ng * xk_bytes);
-                        tma_load_2d(bbuf + s * I8_B_TILE, &maps.m[mi], G * GS, 2 * slot0, B_FULL(s));
-                        for (int sub = 0; sub < ng; ++sub)
-                            bulk_g2s(xkbuf + (2 * s + sub) * I8_XK_BYTES,
-                                     p.xk + ((long long)(G + sub) * p.R_alloc + slot0) * 2, xk_bytes, B_FULL(s));
+                        { I8S_T0(); mbar_wait_blk(B_EMPTY(bs), bph); I8S_ADD(1); }
+                        mbar_expect_tx(B_FULL(bs), tile_bytes + ng * xk_bytes);
+                        tma_load_2d(bbuf + bs * I8_B_TILE, map, G * GS, 2 * slot0, B_FULL(bs));
+#pragma unroll
+                        for (int sub = 0; sub < GPS; ++sub) {
+                            if (sub < ng) {
+                                bulk_g2s(xkbuf + (2 * bs + sub) * I8_XK_BYTES, xk_src, xk_bytes, B_FULL(bs));
+                                xk_src += xk_step;
+                            }
+                        }
+                        if (++bs == I8_NSB) { bs = 0; bph ^= 1u; }
                     }
                 }
             }
