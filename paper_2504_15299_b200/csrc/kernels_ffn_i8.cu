@@ -467,16 +467,19 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             uint32_t myblks = 0;                                 // byte i: first slot / 4 of my block i
 #pragma unroll
             for (int i = 0; i < 4; ++i) myblks |= (uint32_t)u->blk[min((wg == 0 ? 0 : h0) + i, 7)] << (8 * i);
-#define MYBLK(i) ((myblks >> (8 * (i))) & 255u)
+            uint32_t blk_r[4];                                   // the same, one register each (hot loop)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) blk_r[i] = (myblks >> (8 * i)) & 255u;
+#define MYBLK(i) blk_r[i]
             float acc[4][4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int s = 0; s < 4; ++s) acc[i][s] = 0.0f;
 
-            // fold the group whose accumulator is buffer `buf` into acc; pb: ring position of its sums
-            // (bits 0-1), phase (bit 2), last group of its stage (bit 3), group inside the stage (bit 4)
-            auto fold = [&](uint32_t g, uint32_t pb, uint32_t meta) {
+            // fold group g (accumulator buffer g & 1) into acc; fbs / fbph: ring position and phase of its sums,
+            // sub: group inside the stage, rel: last group of the stage (the stage is released afterwards)
+            auto fold = [&](uint32_t g, uint32_t fbs, uint32_t fbph, int sub, bool rel, uint32_t meta) {
                 const int buf = g & 1;
                 { I8S_T0(); mbar_wait_blk(D_FULL(buf), (g >> 1) & 1); I8S_ADD(9); }
                 tc_fence_after();
@@ -484,8 +487,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const __half2 mh = as_h2(meta);
                 const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
                 const float lo = __high2float(mh);
-                mbar_wait_blk(B_FULL(pb & 3), (pb >> 2) & 1);
-                const uint32_t xk_addr = xkbuf + ((pb & 3) * 2 + (pb >> 4)) * I8_XK_BYTES;
+                mbar_wait_blk(B_FULL(fbs), fbph);
+                const uint32_t xk_addr = xkbuf + (fbs * 2 + sub) * I8_XK_BYTES;
                 // two rounds of two blocks: 16 accumulator registers in flight instead of 32
 #pragma unroll
                 for (int rd = 0; rd < 2; ++rd) {
@@ -513,15 +516,17 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         }
                     }
                 }
-                if (pb & 8) {
+                if (rel) {
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(B_EMPTY(pb & 3));
+                    if (lane == 0) mbar_arrive(B_EMPTY(fbs));
                 }
                 I8S_ADD(11);
             };
 
             bool pend = false;
-            uint32_t pend_pb = 0, pend_meta = 0;
+            uint32_t pend_bs = 0, pend_bph = 0, pend_meta = 0;
+            int pend_sub = 0;
+            bool pend_rel = true;
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
                 { I8S_T0(); mbar_wait_blk(W_FULL(ws), wph); I8S_ADD(6); }
@@ -578,10 +583,10 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 handoff_end();
                             }
                         }
-                        if (pend) fold(gc - 1, pend_pb, pend_meta);
+                        if (pend) fold(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
                         pend = true;
                         pend_meta = meta;
-                        pend_pb = bs | (bph << 2) | (sub == ng - 1 ? 8u : 0u) | ((uint32_t)sub << 4);
+                        pend_bs = bs; pend_bph = bph; pend_sub = sub; pend_rel = sub == ng - 1;
                         ++gc;
 #ifdef D2MOE_WAIT_STATS
                         stat[13] += 1;
@@ -593,7 +598,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
                 if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
             }
-            if (pend) fold(gc - 1, pend_pb, pend_meta);
+            if (pend) fold(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
             I8S_T0();
