@@ -48,7 +48,7 @@ constexpr int I8_SLOTS = 32;                  // token slots per unit
 constexpr int I8_NSB = 4;                     // activation ring depth
 constexpr int I8_MAX_NSW = 8;                 // weight ring depth (upper bound)
 constexpr int I8_B_TILE = 2 * I8_SLOTS * 128; // 64 rows x 128 bytes (128 input columns)
-constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa X) per slot, one group
+constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa) per slot, one group
 constexpr int I8_B_STAGE = I8_B_TILE + 2 * I8_XK_BYTES;
 constexpr int I8_EPI_STRIDE = 17;
 constexpr float I8_XMAX = 16191.0f;           // |xq| <= 126 * 128 + 63
@@ -252,7 +252,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t w_slot_bytes = (uint32_t)(GPS * 2) * (uint32_t)p.L.block_bytes;
     const uint32_t bbuf = smem_base;
-    const uint32_t xkbuf = smem_base + I8_NSB * I8_B_TILE;   // per stage: 2 x (X, kappa X) of 32 slots
+    const uint32_t xkbuf = smem_base + I8_NSB * I8_B_TILE;   // per stage: 2 x (X, kappa) of 32 slots
     const uint32_t wbuf = smem_base + p.smem_w_off;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.smem_bar_off);
     const uint32_t bar0 = smem_u32(bars);
@@ -506,12 +506,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                             const uint32_t a = xk_addr + 32u * MYBLK(2 * rd + i);
                             asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
                             asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
+                            // the four slots of a block have one width: s1' kappa + lo once per block
+                            const float cx = fmaf(s1p, xk[1], lo);
 #pragma unroll
                             for (int s = 0; s < 4; ++s) {
                                 const int di = (int)v[i][2 * s] * 128 + (int)v[i][2 * s + 1];
-                                const float t = (float)di + xk[2 * s + 1];
-                                acc[2 * rd + i][s] = fmaf(s1p, t, acc[2 * rd + i][s]);
-                                acc[2 * rd + i][s] = fmaf(lo, xk[2 * s], acc[2 * rd + i][s]);
+                                acc[2 * rd + i][s] = fmaf(s1p, (float)di, acc[2 * rd + i][s]);
+                                acc[2 * rd + i][s] = fmaf(cx, xk[2 * s], acc[2 * rd + i][s]);
                             }
                         }
                     }
@@ -722,7 +723,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
 // Quantises one activation row per slot to 15-bit integers xq = rint(x / sigma), sigma = max|x| / 16191,
 // stored as two signed bytes per element (xq = 128 hi + lo8, lo8 in [-64, 63]) in rows 2 slot and
 // 2 slot + 1 of q, in the byte order of the operand cells (elements k, k+2, k+1, k+3), and writes
-// per group the integer sum X of the row's xq and kappa * X.  GATHER: the row of slot s is
+// per group the integer sum X of the row's xq, and kappa of the slot.  GATHER: the row of slot s is
 // x[src_token[s]] (bf16); otherwise it is row s of an fp32 buffer.  Padding slots become zeros.
 template <bool GATHER>
 __global__ void __launch_bounds__(256)
@@ -797,7 +798,7 @@ i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, c
             if (c < n_cells && (c % cpg) == 0) {
                 const int G = c / cpg;
                 float2 o;
-                o.x = (float)sum; o.y = kap * (float)sum;
+                o.x = (float)sum; o.y = kap;
                 reinterpret_cast<float2*>(xk)[(size_t)G * R_alloc + slot] = o;
             }
         }
