@@ -68,18 +68,9 @@ struct I8Params {
     long long R_alloc;
     int32_t* status;
     int smem_w_off, smem_epi_off, smem_bar_off;
-    int dbg;                  // debug builds only: bit 0 skips the MMAs, bit 1 the unpack math, bit 2 the fold math
 };
 
 struct I8Item { int unit, tile, split, g0, g1; };
-
-#if defined(D2MOE_WAIT_STATS) || defined(D2MOE_I8_DBG)
-#define I8_SKIP(bit) if (!(p.dbg & bit))      // debug builds only: leave out part of the work
-#define I8_STREAM_ONLY (p.dbg & 8)            // debug builds only: stream the rings, do nothing else
-#else
-#define I8_SKIP(bit)
-#define I8_STREAM_ONLY false
-#endif
 
 #ifdef D2MOE_WAIT_STATS
 // Debug build only: cycles per wait category, summed over all CTAs.  0 wprod.w_empty 1 bprod.b_empty
@@ -391,7 +382,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const uint64_t bdesc = smem_desc_sw128(bbuf + bs * I8_B_TILE);
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
-                    if (sub < ng && !I8_STREAM_ONLY) {
+                    if (sub < ng) {
                         const int buf = gc & 1;
                         { I8S_T0(); mbar_wait_blk(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1); I8S_ADD(2); }
                         tc_fence_after();
@@ -406,18 +397,15 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                     tc_fence_after();
                                     const uint32_t a_addr = a_tmem + wg * 64;
                                     if (elect_one()) {
-                                        I8_SKIP(1)
-                                        {
+#pragma unroll
+                                        for (int ks = 0; ks < KSTEPS; ++ks)
+                                            tc_mma_i8_ts(d_addr, a_addr + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
+                                                         idesc[j0], (j0 == 0 && ks == 0) ? 0u : 1u);
+                                        if (j1 <= kmax) {
 #pragma unroll
                                             for (int ks = 0; ks < KSTEPS; ++ks)
-                                                tc_mma_i8_ts(d_addr, a_addr + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
-                                                             idesc[j0], (j0 == 0 && ks == 0) ? 0u : 1u);
-                                            if (j1 <= kmax) {
-#pragma unroll
-                                                for (int ks = 0; ks < KSTEPS; ++ks)
-                                                    tc_mma_i8_ts(d_addr, a_addr + 32 + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
-                                                                 idesc[j1 & 7], 1u);
-                                            }
+                                                tc_mma_i8_ts(d_addr, a_addr + 32 + ks * 8, bdesc + (uint64_t)((sub * GS + ks * 32) >> 4),
+                                                             idesc[j1 & 7], 1u);
                                         }
                                         tc_commit(A_EMPTY(wg, 0));
                                     }
@@ -498,7 +486,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         if (2 * rd + i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(2 * rd + i), v[i]);
                     tc_wait_ld();
                     if (rd == 1) { tc_fence_before(); mbar_arrive(D_EMPTY(buf)); }
-                    I8_SKIP(4)
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
                         if (2 * rd + i < n_mine) {
@@ -531,13 +518,9 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
                 { I8S_T0(); mbar_wait_blk(W_FULL(ws), wph); I8S_ADD(6); }
-                if (I8_STREAM_ONLY) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(B_EMPTY(bs));
-                }
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
-                    if (sub < ng && !I8_STREAM_ONLY) {
+                    if (sub < ng) {
                         const uint32_t wb = w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes;
                         uint32_t meta;
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
@@ -557,7 +540,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 constexpr int J = decltype(jc)::value;
                                 if constexpr (J < SL::count()) {
                                     if ((J & 1) == wg && J <= kmax) {
-                                        I8_SKIP(2)
                                         unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J),
                                                                       a_base + (J >> 1) * 32);
                                     }
@@ -825,10 +807,6 @@ static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long 
 
 }  // namespace
 
-static int g_i8_dbg_mode = 0;
-#if defined(D2MOE_WAIT_STATS) || defined(D2MOE_I8_DBG)
-extern "C" int d2moe_debug_i8_set_mode(int mode) { g_i8_dbg_mode = mode; return 0; }
-#endif
 #ifdef D2MOE_WAIT_STATS
 extern "C" int d2moe_debug_i8_stats(unsigned long long* host16, int reset) {
     cudaDeviceSynchronize();
@@ -874,7 +852,6 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         p.xk = mode == 0 ? B.xk_x : B.xk_h;
         p.sigma = mode == 0 ? sigma_x : sigma_h;
         p.hbuf = B.h32; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
-        p.dbg = g_i8_dbg_mode;
         const int gps = 128 / D.g;
         const int b_bytes = I8_NSB * I8_B_STAGE;
         const int w_slot = gps * 2 * p.L.block_bytes;
