@@ -51,6 +51,10 @@ constexpr int I8_B_TILE = 2 * I8_SLOTS * 128; // 64 rows x 128 bytes (128 input 
 constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa) per slot, one group
 constexpr int I8_B_STAGE = I8_B_TILE + 2 * I8_XK_BYTES;
 constexpr int I8_EPI_STRIDE = 17;
+constexpr int I8_NSQ = 4;                     // entries of the work queue between the producer and the other warps
+// barriers: weight ring (full, empty), activation ring (full, empty), 4 + 4 hand-offs, 2 + 2 accumulators,
+// work queue (full, empty), 2 exchange barriers of the output phase
+constexpr int I8_N_BARS = 2 * I8_MAX_NSW + 2 * I8_NSB + 12 + 2 * I8_NSQ + 2;
 constexpr float I8_XMAX = 16191.0f;           // |xq| <= 126 * 128 + 63
 
 struct I8Params {
@@ -61,6 +65,7 @@ struct I8Params {
     int n_row_tiles, n_split, groups_per_split, nsw;
     const I8Unit* units;
     const int* n_units;
+    int* next_item;           // work counter of this launch: starts at the grid size (item i < grid goes to CTA i)
     const float* xk;          // [n_groups][R_alloc][2]
     const float* sigma;       // [R_alloc]
     float* hbuf;              // [R_alloc, F]
@@ -184,6 +189,9 @@ template <int WPACK> using I8SegList = WidthList<WPACK>;
 static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, int wg, int r, int n_mine, uint32_t blks,
                                                  float (&acc)[4][4], uint8_t* smem) {
     float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
+    // the warpgroup's exchange barrier (128 arrivals): two phases per work item, so the parities are always 0, 1;
+    // a bounded wait, like every other wait of the kernel
+    const uint32_t ebar = smem_u32(smem + p.smem_bar_off) + 8u * (uint32_t)(I8_N_BARS - 2 + wg);
     const I8Item io = i8_item(p, item);
     const int slot0 = p.units[io.unit].slot0;
     const int blk = r >> 6, rr = r & 63;
@@ -202,7 +210,8 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, in
 #pragma unroll
                     for (int s = 0; s < 4; ++s) epi[rr * I8_EPI_STRIDE + 4 * i + s] = acc[i][s];
         }
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+        mbar_arrive(ebar);
+        mbar_wait_blk(ebar, 0);
         if (blk == 0) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -217,7 +226,8 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, in
                 }
             }
         }
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+        mbar_arrive(ebar);
+        mbar_wait_blk(ebar, 1);
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -255,6 +265,12 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     auto A_EMPTY = [&](int wg, int sl) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 4 + wg * 2 + sl); };
     auto D_FULL = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 8 + b); };
     auto D_EMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 10 + b); };
+    auto SQ_FULL = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 12 + i); };
+    auto SQ_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 12 + I8_NSQ + i); };
+    static_assert(8 * I8_N_BARS + 4 * I8_NSQ <= 488, "barrier block");
+    // work queue entries (after the barriers): the producer takes work items from a global counter and
+    // publishes them here, so that CTAs that drew cheap items take more of them
+    volatile int* sq_item = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 8 * I8_N_BARS);
     // tail of the 512-byte barrier block: TMEM base (488), device-status pointer (496), abort flag (504)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 488);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 504);
@@ -269,6 +285,9 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         for (int wg = 0; wg < 2; ++wg)
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
+        // a queue entry is released by the issuer warp and the eight unpack / fold warps
+        for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 9); }
+        for (int wg = 0; wg < 2; ++wg) mbar_init(bar0 + 8u * (uint32_t)(I8_N_BARS - 2 + wg), 128);
         *abort_flag = 0;
         *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -297,7 +316,15 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             // This thread shares a scheduler with unpack warps, so its loop is kept short: source pointers and
             // ring positions advance by addition, nothing is recomputed per stage.
             uint32_t it = 0, ws = 0, wph = 1, bs = 0, bph = 1;         // ring positions, parity of the "empty" waits
-            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+            int item = blockIdx.x;
+            for (uint32_t qi = 0;; ++qi) {
+                const uint32_t q = qi & (I8_NSQ - 1);
+                mbar_wait_blk(SQ_EMPTY(q), ((qi / I8_NSQ) & 1u) ^ 1u);
+                if (item >= total_items) item = -1;                    // the end mark
+                sq_item[q] = item;
+                mbar_arrive(SQ_FULL(q));
+                if (item < 0) break;
+                const int next = atomicAdd(p.next_item, 1);            // in flight while this item's stages are issued
                 const I8Item ii = i8_item(p, item);
                 const I8Unit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
@@ -348,6 +375,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         if (++bs == I8_NSB) { bs = 0; bph ^= 1u; }
                     }
                 }
+                item = next;
             }
             for (int s = 0; s < nsw && s < (int)it; ++s) {      // drain: all copies issued have landed
                 const uint32_t last = it - 1 - (it - 1 - s) % nsw;
@@ -369,7 +397,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
 #ifdef D2MOE_WAIT_STATS
         const long long _tt = clock64();
 #endif
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        for (uint32_t qi = 0;; ++qi) {
+            const uint32_t q = qi & (I8_NSQ - 1);
+            mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
+            const int item = sq_item[q];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(SQ_EMPTY(q));
+            if (item < 0) break;
             const I8Item ii = i8_item(p, item);
             const I8Unit* u = p.units + ii.unit;
             const int kmax = u->kmax;
@@ -446,7 +480,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
 #ifdef D2MOE_WAIT_STATS
         const long long _tt = clock64();
 #endif
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        for (uint32_t qi = 0;; ++qi) {
+            const uint32_t q = qi & (I8_NSQ - 1);
+            mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
+            const int item = sq_item[q];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(SQ_EMPTY(q));
+            if (item < 0) break;
             const I8Item ii = i8_item(p, item);
             const I8Unit* u = p.units + ii.unit;
             const int kmax = u->kmax, nblk = u->nblk;
@@ -612,15 +652,19 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // One block.  Lays every expert's tokens out by width, widest first, each width class padded to a
 // multiple of 8 slots; cuts every expert into units of 32 slots; records per unit and segment how many
 // of its slots include the segment, and which blocks of 4 slots hold real tokens.
-// Shared memory: group_off (E K + 1 ints), then per expert its first unit (n_exp + 1 ints).
+// Then orders the units by decreasing work per group, so that the expert kernels, whose CTAs draw work
+// items from a counter, take the cheap ones last; sets both work counters (n_units[1], n_units[2]) to
+// the grid size of those kernels.
+// Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints).
 __global__ void __launch_bounds__(256)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
-               int32_t* src_token, float* kappa, int max_units, int top, int b1) {
+               int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid) {
     extern __shared__ int32_t s_prep[];
     __shared__ int s_total;
     const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
     int32_t* go = s_prep;                          // group_off
     int32_t* unit_off = s_prep + n_keys + 1;
+    int32_t* cost = unit_off + n_exp + 1;
     for (int i = threadIdx.x; i <= n_keys; i += blockDim.x) go[i] = R.group_off[i];
     __syncthreads();
     if (threadIdx.x < 32) {                       // padded slot offsets and first units (one warp scans)
@@ -647,7 +691,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         }
         if (lane == 0) {
             pad_off[n_exp] = carry; s_total = carry; unit_off[n_exp] = ucarry;
-            *n_units = min(ucarry, max_units);
+            n_units[0] = min(ucarry, max_units);
+            n_units[1] = ffn_grid; n_units[2] = ffn_grid;
         }
     }
     __syncthreads();
@@ -698,7 +743,31 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
                     if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
             }
             units[nu] = u;                        // every window starts with a real token: never empty
+            // work per group and warp: a warpgroup unpacks every other segment and folds half of the blocks
+            cost[nu] = 80 * ((u.kmax + 2) / 2) + 25 * ((u.nblk + 1) / 2);
         }
+    }
+    __syncthreads();
+    const int n = min(unit_off[n_exp], max_units);
+    if (n <= 4 * (int)blockDim.x) {              // rank by (cost descending, index ascending), then permute
+        I8Unit mine[4];
+        int rank[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = threadIdx.x + k * blockDim.x;
+            rank[k] = -1;
+            if (i < n) {
+                mine[k] = units[i];
+                const int c = cost[i];
+                int rk = 0;
+                for (int j = 0; j < n; ++j) rk += (cost[j] > c || (cost[j] == c && j < i)) ? 1 : 0;
+                rank[k] = rk;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (rank[k] >= 0) units[rank[k]] = mine[k];
     }
 }
 
@@ -829,18 +898,19 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     int8_t* qh = reinterpret_cast<int8_t*>(B.h16);
     const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
 
-    const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1) * 4;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int ffn_grid = 2 * sms;
+    const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
     i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
-                                      pl.max_units, Lgu.top, Lgu.b1);
+                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid);
     i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
                                                     qx, B.xk_x, sigma_x, device_status);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps_u8(&maps_x, qx, 2 * pl.R_alloc, D.d) || !make_maps_u8(&maps_h, qh, 2 * pl.R_alloc, D.F))
         return cudaErrorNotSupported;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
 
     for (int mode = 0; mode < 2; ++mode) {
         I8Params p;
@@ -848,7 +918,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         p.n_row_tiles = mode == 0 ? D.F / 64 : D.d / 128;
         p.n_split = mode == 0 ? 1 : pl.n_split;
         p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
-        p.units = units; p.n_units = B.n_units;
+        p.units = units; p.n_units = B.n_units; p.next_item = B.n_units + 1 + mode;
         p.xk = mode == 0 ? B.xk_x : B.xk_h;
         p.sigma = mode == 0 ? sigma_x : sigma_h;
         p.hbuf = B.h32; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
@@ -877,7 +947,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         auto launch = [&](auto kern) -> cudaError_t {
             cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
             if (err != cudaSuccess) return err;
-            kern<<<2 * sms, I8_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            kern<<<ffn_grid, I8_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
         cudaError_t e;
