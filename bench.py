@@ -29,7 +29,7 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of
 # this command (profiles/ffn_i8_kernel_mixtral_decode_T64.md); key = workload:tokens:stage:path
-NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1024431872, "mixtral_decode:T64:down:auto": 522892288}
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1044382432, "mixtral_decode:T64:down:auto": 539915144}
 
 
 def measured_peaks():
