@@ -44,7 +44,7 @@ constexpr int D_COLS = 384;            // accumulator columns (n_cap <= 320)
 constexpr int A_SLOTS = 2;             // operand tiles of GS/2 columns at TMEM columns 384 and 448
 constexpr int NSB = 2;                 // activation ring depth
 constexpr int MAX_NSW = 4;             // weight ring depth (upper bound)
-constexpr int EPI_STRIDE = 17;
+constexpr int NSQ = 4;                 // entries of the work queue between the weight producer and the other warps
 
 struct TcParams {
     MoeDims D;
@@ -54,6 +54,7 @@ struct TcParams {
     int n_cap, n_row_tiles, n_split, groups_per_split, nsw;
     const TcUnit* units;
     const int* n_units;
+    int* next_item;           // work counter of this launch: starts at the grid size (item i < grid goes to CTA i)
     __half* hbuf;             // [R, F]
     float* obuf;              // [n_split][R, d]
     long long R_alloc;
@@ -168,6 +169,14 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     const uint32_t D_EMPTY = D_FULL + 8u;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_NSW + 2 * NSB + 2 * A_SLOTS + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // Work queue (bytes 160..255 of the barrier block): the weight producer takes work items from a global
+    // counter and publishes them to the other warps, so that CTAs that drew cheap items take more of them.
+    // An entry is released by the activation producer, the issuer warp and the eight dequant warps.
+    static_assert(8 * (2 * MAX_NSW + 2 * NSB + 2 * A_SLOTS + 2) + 8 <= 160, "barrier block");
+    auto SQ_FULL = [&](uint32_t i) { return bar0 + 160u + 8u * i; };
+    auto SQ_EMPTY = [&](uint32_t i) { return bar0 + 192u + 8u * i; };
+    auto EPI_BAR = [&](int wg) { return bar0 + 224u + 8u * (uint32_t)wg; };     // SwiGLU exchange of a warpgroup (128 arrivals)
+    volatile int* sq_item = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 240);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -177,6 +186,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         for (int i = 0; i < A_SLOTS; ++i) { mbar_init(A_FULL(i), 256); mbar_init(A_EMPTY(i), 1); }
         mbar_init(D_FULL, 1);
         mbar_init(D_EMPTY, 256);
+        for (int i = 0; i < NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 10); }
+        for (int wg = 0; wg < 2; ++wg) mbar_init(EPI_BAR(wg), 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -204,12 +215,29 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     const int n_units = *p.n_units;
     const int total_items = n_units * p.n_row_tiles * p.n_split;
     const int nsw = p.nsw;
+    // next work item of a consumer: queue entry qi (one arrival per warp, or per thread for a single-thread role)
+    auto pop = [&](uint32_t qi, bool whole_warp) -> int {
+        const uint32_t q = qi & (NSQ - 1);
+        mbar_wait(SQ_FULL(q), (qi / NSQ) & 1u, abort_flag, p.status);
+        const int item = sq_item[q];
+        if (whole_warp) __syncwarp();
+        if (!whole_warp || lane == 0) mbar_arrive(SQ_EMPTY(q));
+        return item;
+    };
 
     if (warp == WARP_WPROD) {
         // ---------------- weight producer ----------------
         if (lane == 0) {
             uint32_t it = 0;
-            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+            int item = blockIdx.x;
+            for (uint32_t qi = 0;; ++qi) {
+                const uint32_t q = qi & (NSQ - 1);
+                mbar_wait(SQ_EMPTY(q), ((qi / NSQ) & 1u) ^ 1u, abort_flag, p.status);
+                if (item >= total_items) item = -1;                    // the end mark
+                sq_item[q] = item;
+                mbar_arrive(SQ_FULL(q));
+                if (item < 0) break;
+                const int next = atomicAdd(p.next_item, 1);            // in flight while this item's blocks are issued
                 const ItemInfo ii = decode_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
@@ -226,6 +254,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     bulk_g2s(dst, m0 + d2moe_block_offset(p.L, rt0, G), bytes, W_FULL(s));
                     bulk_g2s(dst + p.L.block_bytes, m1 + d2moe_block_offset(p.L, rt1, G), bytes, W_FULL(s));
                 }
+                item = next;
             }
             // drain: every copy issued must have landed before the CTA may exit
             for (int s = 0; s < nsw && s < (int)it; ++s) {
@@ -237,7 +266,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         // ---------------- activation producer ----------------
         if (lane == 0) {
             uint32_t it = 0;
-            for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+            for (uint32_t qi = 0;; ++qi) {
+                const int item = pop(qi, false);
+                if (item < 0) break;
                 const ItemInfo ii = decode_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
                 const int ncols = u->ncols;                       // multiple of 16, <= n_cap
@@ -275,7 +306,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         constexpr uint32_t DESC_HI = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
         uint32_t it = 0, at = 0, ic = 0;
         const uint32_t slab_step = (uint32_t)p.n_cap * 8u;        // second 64-column slab of a stage, in 16-byte units
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
+        for (uint32_t qi = 0;; ++qi, ++ic) {
+            const int item = pop(qi, true);
+            if (item < 0) break;
             const ItemInfo ii = decode_item(p, item);
             const TcUnit* u = p.units + ii.unit;
             const int kmax = u->kmax;
@@ -335,9 +368,11 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         const int blk = r >> 6, rr = r & 63;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (128 * 9);
-        uint32_t it = 0, at = 0, ic = 0;
+        uint32_t it = 0, at = 0, ic = 0, eph = 0;       // eph: parity of the warpgroup's next exchange barrier phase
         __half2 acc[GS / 4];
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++ic) {
+        for (uint32_t qi = 0;; ++qi, ++ic) {
+            const int item = pop(qi, true);
+            if (item < 0) break;
             const ItemInfo ii = decode_item(p, item);
             const TcUnit* u = p.units + ii.unit;
             const int e = u->e, kmax = u->kmax;
@@ -442,7 +477,11 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     const int give = blk == 0 ? 8 : 0;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) epi[(blk * 64 + rr) * 9 + j] = __uint_as_float(v[give + j]) * two_S;
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+                    // a bounded wait like every other one (after a timeout the warps of a warpgroup may leave
+                    // the queue at different items: no bar.sync inside the roles)
+                    mbar_arrive(EPI_BAR(wg));
+                    mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
+                    eph ^= 1u;
                     const int keep = blk == 0 ? 0 : 8;           // the tokens this thread finishes
                     __half* dst = p.hbuf + (grow + keep) * p.D.F + (long long)ii.tile * 64 + rr;
 #pragma unroll
@@ -454,7 +493,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                             dst[(long long)j * p.D.F] = __float2half_rn(__fdividef(g, 1.0f + __expf(-g)) * up);
                         }
                     }
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+                    mbar_arrive(EPI_BAR(wg));
+                    mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
+                    eph ^= 1u;
                 } else {
                     float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + r;
 #pragma unroll
@@ -483,8 +524,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 // most n_cap rows, and records for every assignment its padded row.
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, int32_t* pad_off,
-               int32_t* row_map, int32_t* src_token, int max_units) {
+               int32_t* row_map, int32_t* src_token, int max_units, int ffn_grid) {
     __shared__ int s_total_rows, s_n_units;
+    __shared__ int s_cost[1024];
     const int n_keys = D.E * D.K + D.n_shared;
     // 1. padded offsets (one warp scans)
     if (threadIdx.x < 32) {
@@ -549,11 +591,40 @@ tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, i
                     u.real[kk] = max(0, min(hi, a0 + n_real) - lo);
                     u.kmax = kk;
                 }
+                // work per group: one dequantised tile per width present + tensor time per column
+                int n_present = 0;
+                for (int kk = 0; kk < 8; ++kk) n_present += u.cnt[kk] > 0 ? 1 : 0;
+                if (nu < 1024) s_cost[nu] = 190 * n_present + u.ncols;
                 units[nu++] = u;
             }
         }
-        *n_units = nu;
+        n_units[0] = nu;
+        n_units[1] = ffn_grid; n_units[2] = ffn_grid;      // work counters of the two expert kernels
         s_n_units = nu;
+    }
+    __syncthreads();
+    // 4. order the units by decreasing work, so that the expert kernels, whose CTAs draw work items from a
+    //    counter, take the cheap ones last (rank by cost, ties by index; then permute)
+    const int n = s_n_units;
+    if (n <= 1024) {
+        TcUnit mine[4];
+        int rank[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = threadIdx.x + k * blockDim.x;
+            rank[k] = -1;
+            if (i < n) {
+                mine[k] = units[i];
+                const int c = s_cost[i];
+                int rk = 0;
+                for (int j = 0; j < n; ++j) rk += (s_cost[j] > c || (s_cost[j] == c && j < i)) ? 1 : 0;
+                rank[k] = rk;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (rank[k] >= 0) units[rank[k]] = mine[k];
     }
 }
 
@@ -623,16 +694,15 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
                               const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
     auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
     const int n_keys = D.E * D.K + D.n_shared;
-    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units);
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms);
     tc_gather_kernel<<<296, 256, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps(&maps_x, B.xp16, pl.R_alloc, D.d) || !make_maps(&maps_h, B.h16, pl.R_alloc, D.F))
         return cudaErrorNotSupported;
-
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
 
     for (int mode = 0; mode < 2; ++mode) {
         TcParams p;
@@ -641,7 +711,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.n_row_tiles = mode == 0 ? D.F / 64 : D.d / 128;
         p.n_split = mode == 0 ? 1 : pl.n_split;
         p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
-        p.units = B.units; p.n_units = B.n_units;
+        p.units = B.units; p.n_units = B.n_units; p.next_item = B.n_units + 1 + mode;
         p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
         const int b_bytes = NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
