@@ -676,11 +676,15 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
                                     : A_tot + 15 * (n_pieces < A_tot ? n_pieces : A_tot);
     pl->R_alloc = ((pad_rows + 255) / 256) * 256 + 256;
     pl->max_units = (int)(c->n_experts + c->n_shared + pl->R_alloc / pl->n_cap + 1);
-    // split-K of the down projection: aim for >= 4 work items per resident CTA (2 per SM, 148 SMs)
-    const long long units_est = (c->n_experts < A ? c->n_experts : A) + (long long)c->n_shared * ((T + pl->n_cap - 1) / pl->n_cap);
+    // split-K of the down projection: aim for >= 4 work items per resident CTA
+    long long units_est = (c->n_experts < A ? c->n_experts : A) + (long long)c->n_shared * ((T + pl->n_cap - 1) / pl->n_cap);
+    // prefill-sized loads: an expert spans several units (every partial output plane is written by the down
+    // projection and read again by the combine, so no more planes than the work distribution needs)
+    if (!pl->decode && units_est < A / pl->n_cap + c->n_experts / 2) units_est = A / pl->n_cap + c->n_experts / 2;
     const long long tiles = c->d_model / 128;
     const int n_groups = c->d_ffn / c->group_size;
-    long long want = (4 * 296 + units_est * tiles - 1) / (units_est * tiles);
+    const long long ctas = pl->decode ? 296 : 148;       // resident CTAs: 2 per SM (decode kernel), 1 per SM
+    long long want = ((pl->decode ? 4 : 2) * ctas + units_est * tiles - 1) / (units_est * tiles);
     if (want < 1) want = 1;
     if (want > 8) want = 8;
     if (want > n_groups / 4) want = n_groups / 4 > 0 ? n_groups / 4 : 1;
