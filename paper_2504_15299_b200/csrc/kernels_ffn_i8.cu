@@ -72,7 +72,7 @@ struct I8Params {
     float* obuf;              // [n_split][R_alloc, d]
     long long R_alloc;
     int32_t* status;
-    int smem_w_off, smem_epi_off, smem_bar_off;
+    int smem_w_off, smem_epi_off, smem_rec_off, smem_bar_off;
 };
 
 struct I8Item { int unit, tile, split, g0, g1; };
@@ -185,20 +185,25 @@ template <int WPACK> using I8SegList = WidthList<WPACK>;
 
 // Output phase of one work item for one thread: scales the folded sums by the tokens' activation
 // scales, applies SwiGLU across the gate / up halves of the tile (mode 0) and writes the result.
-// blks: byte i = first slot / 4 of the thread's block i.
-static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, int wg, int r, int n_mine, uint32_t blks,
+// blks: byte i = first slot / 4 of the thread's block i.  rec: the warp's record of the work item in shared
+// memory (words 0..31: activation scale of the unit's slots, copied asynchronously when the item began;
+// 32: first slot, 33: tile, 34: split), so that the phase starts without a trip to global memory.
+static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int r, int n_mine, uint32_t blks,
                                                  float (&acc)[4][4], uint8_t* smem) {
+    const float* rec = reinterpret_cast<const float*>(smem + p.smem_rec_off) + (threadIdx.x >> 5) * 40;
     float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
     // the warpgroup's exchange barrier (128 arrivals): two phases per work item, so the parities are always 0, 1;
     // a bounded wait, like every other wait of the kernel
     const uint32_t ebar = smem_u32(smem + p.smem_bar_off) + 8u * (uint32_t)(I8_N_BARS - 2 + wg);
-    const I8Item io = i8_item(p, item);
-    const int slot0 = p.units[io.unit].slot0;
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncwarp();
+    const int slot0 = reinterpret_cast<const int*>(rec)[32];
+    const int io_tile = reinterpret_cast<const int*>(rec)[33], io_split = reinterpret_cast<const int*>(rec)[34];
     const int blk = r >> 6, rr = r & 63;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (i < n_mine) {
-            const float4 sg = *reinterpret_cast<const float4*>(p.sigma + slot0 + 4 * ((blks >> (8 * i)) & 255u));
+            const float4 sg = *reinterpret_cast<const float4*>(rec + 4 * ((blks >> (8 * i)) & 255u));
             acc[i][0] *= sg.x; acc[i][1] *= sg.y; acc[i][2] *= sg.z; acc[i][3] *= sg.w;
         }
     }
@@ -216,7 +221,7 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, in
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 if (i < n_mine) {
-                    float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io.tile * 64 + rr;
+                    float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
 #pragma unroll
                     for (int s = 0; s < 4; ++s) {
                         const float g = acc[i][s];
@@ -232,8 +237,8 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int item, in
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (i < n_mine) {
-                float* dst = p.obuf + (long long)io.split * p.R_alloc * p.D.d
-                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io.tile * 128 + r;
+                float* dst = p.obuf + (long long)io_split * p.R_alloc * p.D.d
+                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io_tile * 128 + r;
 #pragma unroll
                 for (int s = 0; s < 4; ++s) dst[(long long)s * p.D.d] = acc[i][s];
             }
@@ -490,6 +495,18 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             const I8Item ii = i8_item(p, item);
             const I8Unit* u = p.units + ii.unit;
             const int kmax = u->kmax, nblk = u->nblk;
+            {
+                float* rec = reinterpret_cast<float*>(smem + p.smem_rec_off) + warp * 40;     // this warp's record of the item
+                const int slot0 = u->slot0;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                             ::"r"(smem_u32(rec + lane)), "l"(p.sigma + slot0 + lane) : "memory");
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                if (lane == 0) {
+                    reinterpret_cast<int*>(rec)[32] = slot0;
+                    reinterpret_cast<int*>(rec)[33] = ii.tile;
+                    reinterpret_cast<int*>(rec)[34] = ii.split;
+                }
+            }
             const int h0 = (nblk + 1) >> 1;
             const int n_mine = wg == 0 ? h0 : nblk - h0;        // my token blocks (at most 4)
             uint32_t myblks = 0;                                 // byte i: first slot / 4 of my block i
@@ -630,7 +647,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int q = 0; q < 4; ++q) out[i][q] = acc[i][q];
-            i8_write_out(p, item, wg, r, n_mine, myblks, out, smem);
+            i8_write_out(p, wg, r, n_mine, myblks, out, smem);
             I8S_ADD(14);
         }
 #ifdef D2MOE_WAIT_STATS
@@ -928,13 +945,15 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         const int epi_bytes = 2 * 64 * I8_EPI_STRIDE * 4;
         const int bar_bytes = 512;
         const int budget = 112 * 1024;
-        int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
+        const int rec_bytes = 8 * 40 * 4;                             // per unpack / fold warp: the record of its work item
+        int nsw = (budget - b_bytes - epi_bytes - rec_bytes - 128 - bar_bytes - 1024) / w_slot;
         if (nsw > I8_MAX_NSW) nsw = I8_MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
         p.nsw = nsw;
         p.smem_w_off = b_bytes;
         p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
-        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 511) & ~511;   // 512-byte aligned from the 1024-byte aligned base
+        p.smem_rec_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        p.smem_bar_off = (p.smem_rec_off + rec_bytes + 511) & ~511;   // 512-byte aligned from the 1024-byte aligned base
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         if (mode == 1)
             i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,
