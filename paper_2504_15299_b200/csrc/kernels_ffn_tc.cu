@@ -688,6 +688,10 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     if (want < 1) want = 1;
     if (want > 8) want = 8;
     if (want > n_groups / 4) want = n_groups / 4 > 0 ? n_groups / 4 : 1;
+    // equal parts balance best: the largest divisor of the number of groups up to the wanted factor, unless
+    // that halves it
+    for (long long w = want; 2 * w > want; --w)
+        if (n_groups % w == 0) { want = w; break; }
     pl->groups_per_split = (int)((n_groups + want - 1) / want);
     if (c->group_size == 64 && (pl->groups_per_split & 1)) ++pl->groups_per_split;   // whole 128-column ring stages
     pl->n_split = (n_groups + pl->groups_per_split - 1) / pl->groups_per_split;
