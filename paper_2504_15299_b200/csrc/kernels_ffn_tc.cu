@@ -684,7 +684,7 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     const long long tiles = c->d_model / 128;
     const int n_groups = c->d_ffn / c->group_size;
     const long long ctas = pl->decode ? 296 : 148;       // resident CTAs: 2 per SM (decode kernel), 1 per SM
-    long long want = ((pl->decode ? 4 : 2) * ctas + units_est * tiles - 1) / (units_est * tiles);
+    long long want = (4 * ctas + units_est * tiles - 1) / (units_est * tiles);
     if (want < 1) want = 1;
     if (want > 8) want = 8;
     if (want > n_groups / 4) want = n_groups / 4 > 0 ? n_groups / 4 : 1;
