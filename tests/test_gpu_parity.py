@@ -486,6 +486,7 @@ def test_workspace_sized_for_a_larger_batch_serves_smaller_ones(B):
     dict(d=256, F=384, E=4, k=2, g=128, bits=(1, 2, 3, 4, 5, 6, 7, 8), T=700),      # eight widths, grouped-GEMM kernel
     dict(d=256, F=256, E=2, k=2, g=64, bits=(2, 4, 8), T=3000),                     # many units per expert, g = 64
     dict(d=384, F=640, E=16, k=4, g=128, bits=(5, 6, 7, 8), T=200, n_shared=1),     # 50 tokens per expert: decode kernel, several units
+    dict(d=128, F=128, E=256, k=8, g=128, bits=(2, 4, 8), T=160, n_shared=2),       # more units (266) than threads order at once
 ])
 def test_stress_shapes(B, case):
     cross, err = small_layer_case(B, **case)
