@@ -13,7 +13,9 @@
 // and signed 8-bit activation halves (xq = 128 hi + lo8), so the CUDA cores never expand a code to
 // a floating-point weight.  What is left for them per packed word is one shift and one AND per four
 // codes (the packed layout keeps the four codes of an operand cell in the four bytes of a word), and
-// per (row, group, token) five instructions that fold the accumulator into the running output.
+// per (row, group, token) four instructions that fold the accumulator into the running output
+// (128 hi + lo8, int -> float, acc += s1' D, acc += (s1' kappa_b + lo) X_G: the bracket once per block
+// of four slots, which share a width).
 //
 //   * The tokens of a unit are laid out by width, widest first, each width class padded to 8 slots:
 //     the slots that include segment j are the first npad[j] of the unit, and the product of
@@ -25,13 +27,20 @@
 //   * The accumulator is double buffered per group: while the products of group G+1 run, the
 //     dequant threads fold group G into fp32 registers.
 //
-// CTA = 320 threads, 2 CTAs per SM (96 registers per thread).  Warps 0-3 and 4-7 are two warpgroups (thread = weight row =
-// TMEM lane): warpgroup w unpacks the segments w, w+2, ... of every group into two alternating
-// 32-column operand slots in TMEM and folds half of the unit's token blocks; warp 8 streams packed
-// blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and the per-group activation sums,
-// warp 9 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns + 4 x 32
-// operand columns.  Every wait is bounded; on expiry the CTA raises D2MOE_DEV_TIMEOUT, stops
-// waiting, drains its copies, frees its TMEM and exits.
+// CTA = 320 threads, 2 CTAs per SM (96 registers per thread).  Warps 0-3 and 4-7 are two warpgroups
+// (thread = weight row = TMEM lane): warpgroup w unpacks the segments w, w+2 of every group into its
+// two 32-column operand tiles in TMEM, hands both to the issuer at once and folds half of the unit's
+// token blocks; warp 8 streams packed blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and
+// the per-group activation sums, warp 9 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns +
+// 4 x 32 operand columns.
+//
+// Work distribution: a work item is one unit x one tile of 128 weight rows x a range of groups.  The
+// producer thread takes item numbers from a global counter (which starts at the grid size: item i < grid
+// belongs to CTA i) and publishes them to the other warps through a small queue in shared memory; the
+// units are ordered by decreasing work, so the cheap items are drawn last.
+//
+// Every wait is bounded (barriers only, no bar.sync inside the roles); on expiry the CTA raises
+// D2MOE_DEV_TIMEOUT, stops waiting, drains its copies, frees its TMEM and exits.
 #include "d2moe_common.cuh"
 #include "kernels_ffn_tc.cuh"
 #include "tc_common.cuh"

@@ -27,7 +27,9 @@
 // streams activation tiles (TMA, 128B swizzle, boxes of up to 256 rows), warp 10 issues the MMAs (the
 // whole warp runs the loop, one elected lane issues).  A unit holds up to 320 tokens, so that one
 // dequantization of a weight tile is amortised over enough tensor work to leave the kernel bound by
-// the tensor cores; an MMA covers at most 256 of a piece's columns.  Every wait is bounded: on expiry
+// the tensor cores; an MMA covers at most 256 of a piece's columns.  Work items (unit x tile) are taken
+// from a global counter by the weight producer and published to the other warps through a queue in
+// shared memory; the units are ordered by decreasing work.  Every wait is bounded: on expiry
 // the CTA raises D2MOE_DEV_TIMEOUT, stops waiting, drains and exits.
 #include "d2moe_common.cuh"
 #include "kernels_ffn_tc.cuh"
