@@ -216,6 +216,18 @@ d2moe_status d2moe_stack_layer(const d2moe_config* cfg, int64_t T, void* x_bf16,
                                int32_t* device_status, void* workspace, size_t workspace_bytes,
                                void* stream);
 
+/*
+ * Self-test of the bounded waits of the expert kernels.  Every wait of those kernels (on a shared-memory
+ * barrier that a copy, a tensor-core operation or another warp completes) gives up after one second,
+ * raises D2MOE_DEV_TIMEOUT in *device_status, and lets the kernel drain and exit, so that a lost
+ * signal costs one call, not the context.  This call launches one small block that waits on a barrier
+ * nothing ever completes - with the wait of the decode kernel (which = 0) or of the grouped-GEMM kernel
+ * (which = 1) - and then issues a second wait, which must return at once because the block's abort flag
+ * is set.  Asynchronous on the stream; takes about one second of device time; after it *device_status
+ * has D2MOE_DEV_TIMEOUT set and the device is usable as before.  device_status: device int32, required.
+ */
+d2moe_status d2moe_selftest_wait_expiry(int which, int32_t* device_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

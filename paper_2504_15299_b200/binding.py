@@ -50,7 +50,7 @@ _lib = None
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
            "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count",
-           "d2moe_route_static_scratch"]
+           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry"]
 
 
 def lib() -> ctypes.CDLL:
@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.d2moe_moe_forward_events.argtypes = [cfgp, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(_RouteIn),
                                            ctypes.POINTER(_RouteOut), vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
     L.d2moe_forward_launch_count.argtypes = [cfgp, i64, ctypes.c_int]
+    L.d2moe_selftest_wait_expiry.argtypes = [ctypes.c_int, vp, vp]
     L.d2moe_stack_layer.argtypes = [cfgp, i64, vp, vp, ctypes.c_float, ctypes.POINTER(vp),
                                     ctypes.POINTER(_RouteIn), vp, vp, sz, vp]
     for name in EXPORTS:
@@ -238,6 +239,11 @@ def route_static_scratch(cfg: Config, x: torch.Tensor, *, gate_w=None, logits=No
                                             _ptr(r.bit_idx), _ptr(r.perm), _ptr(r.inv_perm), _ptr(r.group_off),
                                             _ptr(r.device_status), _stream(stream)), "d2moe_route_static_scratch")
     return r
+
+
+def selftest_wait_expiry(which: int, device_status: torch.Tensor, stream=None) -> None:
+    """Launches the block whose bounded wait nothing satisfies (see include/d2moe.h); asynchronous."""
+    _check(lib().d2moe_selftest_wait_expiry(which, _ptr(device_status), _stream(stream)), "d2moe_selftest_wait_expiry")
 
 
 def _expert_ptr_array(expert_w: Sequence[torch.Tensor]):

@@ -332,6 +332,12 @@ extern "C" d2moe_status d2moe_moe_forward_events(const d2moe_config* c, int64_t 
                         (cudaStream_t)stream, stage_events);
 }
 
+extern "C" d2moe_status d2moe_selftest_wait_expiry(int which, int32_t* device_status, void* stream) {
+    if (!device_status) return D2MOE_ERR_NULL;
+    if (which < 0 || which > 1) return D2MOE_ERR_SHAPE;
+    return launch_wait_expiry(which, device_status, (cudaStream_t)stream) == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+}
+
 extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int routing_precomputed) {
     if (d2moe_check_config(c) != D2MOE_OK || T <= 0) return 0;
     // route, then count + scan + scatter (one launch when the load is small: the rule of launch_route)

@@ -911,6 +911,42 @@ extern "C" int d2moe_debug_i8_stats(unsigned long long* host16, int reset) {
 }
 #endif
 
+namespace {
+// One block waits on a barrier that nothing completes, with either of the two bounded waits of the
+// expert kernels; the barrier block has the layout those waits expect (status pointer at byte 496, abort
+// flag at byte 504 of a 512-byte aligned block).  A second wait follows: with the abort flag set it
+// returns at once.
+__global__ void __launch_bounds__(64)
+wait_expiry_kernel(int which, int32_t* status) {
+    __shared__ __align__(1024) uint8_t blk[1024];
+    uint8_t* b = blk + ((512u - (smem_u32(blk) & 511u)) & 511u);
+    const uint32_t bar = smem_u32(b);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(b + 504);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        *abort_flag = 0;
+        *reinterpret_cast<int32_t**>(b + 496) = status;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (which == 0) mbar_wait_blk(bar, 0);
+        else mbar_wait(bar, 0, abort_flag, status);
+    }
+    __syncthreads();
+    if (threadIdx.x == 32) {
+        if (which == 0) mbar_wait_blk(bar, 0);
+        else mbar_wait(bar, 0, abort_flag, status);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_wait_expiry(int which, int32_t* device_status, cudaStream_t st) {
+    wait_expiry_kernel<<<1, 64, 0, st>>>(which, device_status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                           const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
                           const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {

@@ -51,6 +51,7 @@ struct TcBuffers {
 };
 
 bool tc_path_supported(const d2moe_config* c);
+cudaError_t launch_wait_expiry(int which, int32_t* device_status, cudaStream_t st);
 void tc_plan(const d2moe_config* c, long long T, TcPlan* pl);
 cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                               const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,

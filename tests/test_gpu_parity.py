@@ -515,3 +515,21 @@ def test_shapes_outside_the_tensor_core_path_use_the_cuda_core_path(B, d, F, g):
         B.moe_forward(cfg, x, [x] * 9, logits=torch.zeros((1, 3), device="cuda"),
                       forced_bit_idx=torch.zeros((1, 2), dtype=torch.int8, device="cuda"))
     assert e.value.code == 4
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("which", [0, 1])
+def test_a_wait_that_nothing_satisfies_expires_and_leaves_the_device_usable(B, which):
+    # the bounded waits of the expert kernels: after one second the block raises the timeout bit and returns
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t0 = time.time()
+    B.selftest_wait_expiry(which, status)
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    assert int(status.item()) & 0x2, status
+    assert 0.9 < dt < 5.0, dt          # one expiry, not two: the second wait sees the abort flag
+    # the context is intact: a normal layer call still passes
+    cross, err = small_layer_case(B, d=128, F=128, E=2, k=1, g=64, bits=(2, 4, 8), T=4)
+    assert cross < TOL and err < TOL, (cross, err)
