@@ -55,7 +55,9 @@ def measured_tensor_peak():
 
 
 # ------------------------------------------------------------------------------------------------
-# algorithmic bytes (what the method has to read at the routed widths)
+# algorithmic bytes: what the method has to read at the routed widths - per active expert and matrix the
+# packed prefix up to the widest width routed to that expert in this call, read once, plus activations
+# in and outputs out
 # ------------------------------------------------------------------------------------------------
 def matrix_bytes(rows, cols, g, bits_read):
     return rows * cols * bits_read // 8 + rows * (cols // g) * 4
