@@ -120,6 +120,13 @@ struct RouteBufs {
     int32_t* perm; int32_t* inv_perm; int32_t* group_off;
 };
 
+// Grouping of the assignments by (expert, width) key: the single-block kernel takes the smallest loads (its
+// rule is in launch_route), one launch of a few blocks the mid-sized ones (every block counts all keys: the
+// walks per warp must stay short), histogram + scan + scatter kernels the rest.
+static inline bool d2moe_group_is_mid(long long A, long long n_keys) {
+    return A <= 12288 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 6144;
+}
+
 // Workspace carving (all offsets 256-byte aligned).
 struct Workspace {
     size_t total;

@@ -233,6 +233,68 @@ group_small_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t*
     }
 }
 
+// Mid-sized loads (a prefill batch of a few thousand assignments on a few dozen keys): one launch of a few
+// blocks.  Every block stages all keys in shared memory and counts every key itself (32 warps, a key per
+// warp at a time), so no block waits for another; block b then writes the groups of the keys b, b + grid,
+// ...  Same warp-per-key ballot walks as above: the same stable order.  smem: A keys + n_keys + 1 ints.
+__global__ void __launch_bounds__(1024)
+group_mid_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
+                 int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+    extern __shared__ int32_t s_grp[];
+    int32_t* s_keys = s_grp;
+    int32_t* s_off = s_grp + ((A + 31) & ~31);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int a = threadIdx.x; a < A; a += blockDim.x) s_keys[a] = keys[a];
+    __syncthreads();
+    for (int key = warp; key < n_keys; key += n_warps) {
+        int cnt = 0;
+        for (int base = 0; base < A; base += 32) {
+            const int a = base + lane;
+            cnt += __popc(__ballot_sync(0xffffffffu, a < A && s_keys[a] == key));
+        }
+        if (lane == 0) s_off[key] = cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int base = 0; base < n_keys; base += 32) {
+            const int i = base + lane;
+            const int v = i < n_keys ? s_off[i] : 0;
+            int incl = v;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (i < n_keys) {
+                s_off[i] = carry + incl - v;
+                if (blockIdx.x == 0) group_off[i] = carry + incl - v;
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            s_off[n_keys] = carry;
+            if (blockIdx.x == 0) group_off[n_keys] = carry;
+        }
+    }
+    __syncthreads();
+    // this block's keys, spread over its warps
+    for (int key = blockIdx.x + warp * gridDim.x; key < n_keys; key += n_warps * gridDim.x) {
+        int pos = s_off[key];
+        if (pos == s_off[key + 1]) continue;
+        for (int base = 0; base < A; base += 32) {
+            const int a = base + lane;
+            const bool m = a < A && s_keys[a] == key;
+            const unsigned bal = __ballot_sync(0xffffffffu, m);
+            if (m) {
+                const int p = pos + __popc(bal & ((1u << lane) - 1u));
+                perm[p] = a;
+                inv_perm[a] = p;
+            }
+            pos += __popc(bal);
+        }
+    }
+}
+
 // Same dot product with both vectors already in shared memory.
 __device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const __nv_bfloat16* b, int d, int lane) {
     float acc = 0.0f;
@@ -439,6 +501,14 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     if (D.A <= 8192 && n_keys <= 2048 && walks <= 1024) {
         const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
         group_small_kernel<<<1, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+        return cudaGetLastError();
+    }
+    if (d2moe_group_is_mid(D.A, n_keys)) {
+        const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
+        cudaError_t e = cudaFuncSetAttribute(group_mid_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsm);
+        if (e != cudaSuccess) return e;
+        const int blocks = n_keys < 16 ? n_keys : 16;
+        group_mid_kernel<<<blocks, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
         return cudaGetLastError();
     }
     count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);
