@@ -570,39 +570,64 @@ tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, i
         row_map[D.A + i] = row;
         src_token[row] = t;
     }
-    // 3. units (serial over experts: at most a few hundred)
-    if (threadIdx.x == 0) {
-        int nu = 0;
-        for (int e = 0; e < D.E + D.n_shared; ++e) {
-            const int key0 = e < D.E ? e * D.K : D.E * D.K + (e - D.E);
-            const int key1 = e < D.E ? key0 + D.K : key0 + 1;
-            const int p0 = pad_off[key0], p1 = pad_off[key1];
-            for (int start = p0; start < p1 && nu < max_units; start += n_cap) {
-                const int end = min(p1, start + n_cap);
-                TcUnit u;
-                u.e = e; u.row0 = start; u.ncols = end - start; u.kmax = 0;
-                for (int kk = 0; kk < 8; ++kk) { u.col0[kk] = 0; u.cnt[kk] = 0; u.real[kk] = 0; }
-                for (int key = key0; key < key1; ++key) {
-                    const int kk = e < D.E ? key - key0 : D.K - 1;
-                    const int a0 = pad_off[key], a1 = pad_off[key + 1];
-                    const int n_real = e < D.E ? R.group_off[key + 1] - R.group_off[key] : D.T;
-                    const int lo = max(a0, start), hi = min(a1, end);
-                    if (hi <= lo) continue;
-                    u.col0[kk] = lo - start;
-                    u.cnt[kk] = hi - lo;
-                    u.real[kk] = max(0, min(hi, a0 + n_real) - lo);
-                    u.kmax = kk;
-                }
-                // work per group: one dequantised tile per width present + tensor time per column
-                int n_present = 0;
-                for (int kk = 0; kk < 8; ++kk) n_present += u.cnt[kk] > 0 ? 1 : 0;
-                if (nu < 1024) s_cost[nu] = 190 * n_present + u.ncols;
-                units[nu++] = u;
+    // 3. units: a warp scans the experts' unit counts, then one thread per expert writes that expert's units
+    __shared__ int s_uoff[D2MOE_MAX_EXPERTS + 1];
+    const int n_exp = D.E + D.n_shared;
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int base = 0; base < n_exp; base += 32) {
+            const int e = base + lane;
+            int nu_e = 0;
+            if (e < n_exp) {
+                const int key0 = e < D.E ? e * D.K : D.E * D.K + (e - D.E);
+                const int key1 = e < D.E ? key0 + D.K : key0 + 1;
+                nu_e = (pad_off[key1] - pad_off[key0] + n_cap - 1) / n_cap;
             }
+            int incl = nu_e;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (e < n_exp) s_uoff[e] = carry + incl - nu_e;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
         }
-        n_units[0] = nu;
-        n_units[1] = ffn_grid; n_units[2] = ffn_grid;      // work counters of the two expert kernels
-        s_n_units = nu;
+        if (lane == 0) {
+            const int nu = min(carry, max_units);
+            s_uoff[n_exp] = carry;
+            n_units[0] = nu;
+            n_units[1] = ffn_grid; n_units[2] = ffn_grid;      // work counters of the two expert kernels
+            s_n_units = nu;
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < n_exp; e += blockDim.x) {
+        const int key0 = e < D.E ? e * D.K : D.E * D.K + (e - D.E);
+        const int key1 = e < D.E ? key0 + D.K : key0 + 1;
+        const int p0 = pad_off[key0], p1 = pad_off[key1];
+        int nu = s_uoff[e];
+        for (int start = p0; start < p1 && nu < max_units; start += n_cap, ++nu) {
+            const int end = min(p1, start + n_cap);
+            TcUnit u;
+            u.e = e; u.row0 = start; u.ncols = end - start; u.kmax = 0;
+            for (int kk = 0; kk < 8; ++kk) { u.col0[kk] = 0; u.cnt[kk] = 0; u.real[kk] = 0; }
+            for (int key = key0; key < key1; ++key) {
+                const int kk = e < D.E ? key - key0 : D.K - 1;
+                const int a0 = pad_off[key], a1 = pad_off[key + 1];
+                const int n_real = e < D.E ? R.group_off[key + 1] - R.group_off[key] : D.T;
+                const int lo = max(a0, start), hi = min(a1, end);
+                if (hi <= lo) continue;
+                u.col0[kk] = lo - start;
+                u.cnt[kk] = hi - lo;
+                u.real[kk] = max(0, min(hi, a0 + n_real) - lo);
+                u.kmax = kk;
+            }
+            // work per group: one dequantised tile per width present + tensor time per column
+            int n_present = 0;
+            for (int kk = 0; kk < 8; ++kk) n_present += u.cnt[kk] > 0 ? 1 : 0;
+            if (nu < 1024) s_cost[nu] = 190 * n_present + u.ncols;
+            units[nu] = u;
+        }
     }
     __syncthreads();
     // 4. order the units by decreasing work, so that the expert kernels, whose CTAs draw work items from a
