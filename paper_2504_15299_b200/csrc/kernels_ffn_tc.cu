@@ -657,18 +657,28 @@ tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, i
 
 // xp16[row, :] = fp16(x[src_token[row], :]) for the real rows (padding rows are never consumed:
 // a D column depends only on its own token row).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 tc_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ src_token,
                  const int32_t* __restrict__ pad_off, int n_keys, __half* __restrict__ xp16) {
     const int total_rows = pad_off[n_keys];
     for (int row = blockIdx.x; row < total_rows; row += gridDim.x) {
         const int t = src_token[row];
         if (t < 0) continue;
-        const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(x + (size_t)t * d);
-        __half2* dst = reinterpret_cast<__half2*>(xp16 + (size_t)row * d);
-        for (int i = threadIdx.x; i < d / 2; i += blockDim.x) {
-            const float2 f = __bfloat1622float2(src[i]);
-            dst[i] = __floats2half2_rn(f.x, f.y);
+        // eight elements (16 bytes) per thread and step; d is a multiple of 128 on this path
+        const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * d);
+        uint4* dst = reinterpret_cast<uint4*>(xp16 + (size_t)row * d);
+        for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+            const uint4 v = src[i];
+            uint4 o;
+            const uint32_t* vi = reinterpret_cast<const uint32_t*>(&v);
+            uint32_t* oi = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vi[k]));
+                const __half2 h = __floats2half2_rn(f.x, f.y);
+                oi[k] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            dst[i] = o;
         }
     }
 }
@@ -733,7 +743,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms);
-    tc_gather_kernel<<<296, 256, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16);
+    tc_gather_kernel<<<1184, 128, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps(&maps_x, B.xp16, pl.R_alloc, D.d) || !make_maps(&maps_h, B.h16, pl.R_alloc, D.F))
