@@ -308,6 +308,7 @@ __device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const _
 __device__ __forceinline__ void stage_row(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int d) {
     const uint4* s = reinterpret_cast<const uint4*>(src);
     uint4* t = reinterpret_cast<uint4*>(dst);
+#pragma unroll 4
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
 }
 
@@ -357,7 +358,7 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
     } else {
         for (int eb = 0; eb < E; eb += EB) {
             const int n = min(EB, E - eb);
-            for (int r = 0; r < n; ++r) stage_row(ws + (size_t)r * D.d, gate_w + (size_t)(eb + r) * D.d, D.d);
+            stage_row(ws, gate_w + (size_t)eb * D.d, n * D.d);       // the n rows are contiguous: one copy loop
             __syncthreads();
             for (int r = warp; r < n; r += 8) {
                 const float v = dot_pinned_smem(xs, ws + (size_t)r * D.d, D.d, lane);
@@ -491,7 +492,9 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
         const size_t smem = row_bytes * (1 + EB) + tail_bytes;
         cudaError_t e = cudaFuncSetAttribute(route_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        route_block_kernel<<<D.T, 256, smem, st>>>(D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status, EB);
+        // logits and widths both supplied: no dot products, one warp per token does the selection
+        const int threads = (logits_in && forced) ? 32 : 256;
+        route_block_kernel<<<D.T, threads, smem, st>>>(D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status, EB);
     } else
     route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
