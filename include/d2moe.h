@@ -202,7 +202,9 @@ d2moe_status d2moe_moe_forward_events(const d2moe_config* cfg, int64_t T, const 
                                       void* workspace, size_t workspace_bytes, void* stream,
                                       void* const* stage_events);
 
-/* Number of kernel launches one d2moe_moe_forward call enqueues for T tokens (0 on a bad config). */
+/* Number of kernel launches one d2moe_moe_forward call enqueues for T tokens (0 on a bad config), for a
+ * call that passes gate weights; with more than 16 experts a call that passes logits instead makes one
+ * launch fewer. */
 int d2moe_forward_launch_count(const d2moe_config* cfg, int64_t T, int routing_precomputed);
 
 /*

@@ -343,7 +343,10 @@ extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int 
     // route, then count + scan + scatter (one launch when the load is small: the rule of launch_route)
     const long long A = (long long)T * c->top_k, n_keys = (long long)c->n_experts * c->n_bits;
     const bool small = A <= 8192 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 1024;
-    const int route = routing_precomputed ? 0 : (small || d2moe_group_is_mid(A, n_keys) ? 2 : 4);
+    int route = routing_precomputed ? 0 : (small || d2moe_group_is_mid(A, n_keys) ? 2 : 4);
+    // more than 16 experts: the gate logits come from a tiled kernel of their own (when the caller supplies
+    // logits instead of gate weights that launch does not happen: the count is then one too high)
+    if (!routing_precomputed && c->n_experts > 16 && (size_t)c->d_model * 2 * 16 <= 200 * 1024) route += 1;
     if (use_tensor_path(c)) {
         TcPlan pl;
         tc_plan(c, T, &pl);
