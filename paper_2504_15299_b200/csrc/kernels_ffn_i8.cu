@@ -745,7 +745,17 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         src_token[slot] = t;
         kappa[slot] = 0.5f - exp2f((float)(top - b1 - 1));
     }
-    for (int e = threadIdx.x; e < n_exp; e += blockDim.x) {        // one thread per expert: its units
+    // one thread per unit (an expert with many tokens, a shared one above all, has many units): the unit's
+    // expert is the last one whose first unit is not beyond it
+    const int n_all = min(unit_off[n_exp], max_units);
+    for (int nu = threadIdx.x; nu < n_all; nu += blockDim.x) {
+        int lo_e = 0, hi_e = n_exp - 1;
+        while (lo_e < hi_e) {
+            const int mid = (lo_e + hi_e + 1) >> 1;
+            if (unit_off[mid] <= nu) lo_e = mid; else hi_e = mid - 1;
+        }
+        while (lo_e + 1 < n_exp && unit_off[lo_e + 1] <= nu) ++lo_e;       // skip experts without units
+        const int e = lo_e;
         const int p0 = pad_off[e], len_e = pad_off[e + 1] - p0;
         int cnt[8], cpad[9];                      // cpad[j]: padded slots of the classes with index >= j
         cpad[D.K] = 0;
@@ -753,8 +763,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
             cnt[j] = e < D.E ? go[e * D.K + j + 1] - go[e * D.K + j] : (j == D.K - 1 ? D.T : 0);
             cpad[j] = cpad[j + 1] + round8(cnt[j]);
         }
-        int nu = unit_off[e];
-        for (int start = 0; start < len_e && nu < max_units; start += I8_SLOTS, ++nu) {
+        {
+            const int start = (nu - unit_off[e]) * I8_SLOTS;
             const int len = min(len_e - start, I8_SLOTS);
             I8Unit u;
             u.e = e; u.slot0 = p0 + start; u.nslots = len; u.kmax = 0; u.nblk = 0;

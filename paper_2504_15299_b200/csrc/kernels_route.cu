@@ -323,8 +323,8 @@ gate_logits_kernel(int T, int E, int d, const __nv_bfloat16* __restrict__ x, con
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t0 = blockIdx.x * TB, e0 = blockIdx.y * EB;
     const int nt = min(TB, T - t0), ne = min(EB, E - e0);
-    for (int r = 0; r < nt; ++r) stage_row(xs + (size_t)r * d, x + (size_t)(t0 + r) * d, d);
-    for (int r = 0; r < ne; ++r) stage_row(ws + (size_t)r * d, gate_w + (size_t)(e0 + r) * d, d);
+    stage_row(xs, x + (size_t)t0 * d, nt * d);                 // consecutive rows are contiguous: one copy loop each
+    stage_row(ws, gate_w + (size_t)e0 * d, ne * d);
     __syncthreads();
     for (int pr = warp; pr < nt * ne; pr += 8) {
         const int tt = pr / ne, ee = pr - tt * ne;
