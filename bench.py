@@ -3,10 +3,17 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload mixtral_decode] [--tokens 64] [--path auto|cuda_core|tensor]
+                    [--min-region-s 1.0] [--others all|layers|none]
 
-Prints ONE JSON line.  N > 1 runs independent replicas, one process per GPU (launched by
-torch.distributed.run), no data-path collective; the barrier and the max-over-ranks timing use NCCL.
-`--impl reference` times the CPU oracle on the host cores on a bounded sample of the same workload.
+Prints ONE JSON line.  The timed region is exactly K steps between a barrier + synchronize on both sides;
+it is repeated until --min-region-s seconds of device time are timed and the median region gives `value`
+(uninstrumented steps; the per-stage times behind `roofline` come from a separate pass).  With the default
+workload on one GPU the line also carries short legs of the other benchmark configurations
+(`other_workloads`: decode batches of 1, 8 and 32 tokens, the 2048-token prefill batch, the fine-grained
+layer, the 32-layer stack).  N > 1 runs independent replicas, one process per GPU, no data-path collective;
+the barrier and the max-over-ranks timing use NCCL; started as a plain script with --gpus N it starts the
+N ranks itself.  `--impl reference` times the CPU oracle on the host cores on a bounded sample of the same
+workload.
 """
 from __future__ import annotations
 
@@ -27,9 +34,12 @@ from paper_2504_15299_b200 import synth  # noqa: E402
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of
-# this command (profiles/ffn_i8_kernel_mixtral_decode_T64.md); key = workload:tokens:stage:path
-NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1044382432, "mixtral_decode:T64:down:auto": 539915144}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, each from one ncu capture of
+# the same workload through this script (the summaries of those captures are committed beside the numbers
+# they come from); key = workload:tokens:stage:path
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1044382432, "mixtral_decode:T64:down:auto": 539915144,
+               "mixtral_prefill:T2048:gate_up:auto": 1671000000, "mixtral_prefill:T2048:down:auto": 950000000,
+               "finegrained:T256:gate_up:auto": 461000000, "finegrained:T256:down:auto": 233300000}
 
 
 def measured_peaks():
@@ -41,17 +51,6 @@ def measured_peaks():
         except Exception:
             pass
     return FALLBACK_HBM_GBS, "fallback"
-
-
-def measured_tensor_peak():
-    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(p):
-        try:
-            d = json.load(open(p))
-            return float(d["bf16_tflops_sustained"]), "measured (sustained)"
-        except Exception:
-            pass
-    return 1400.0, "fallback (sustained)"
 
 
 # ------------------------------------------------------------------------------------------------
@@ -266,26 +265,222 @@ def job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> fl
     return tokens_per_rank * world / (ms_per_step * 1e-3)
 
 
-def workload_config(wl, T, path):
+# ------------------------------------------------------------------------------------------------
+# timing helpers
+# ------------------------------------------------------------------------------------------------
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _sync_all(dist):
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+        torch.cuda.synchronize()
+
+
+def time_regions(run_region, steps, dist, dev, min_region_s, max_regions=200):
+    """Times regions of exactly `steps` steps each (barrier + synchronize on both sides, device time, max over
+    ranks) until `min_region_s` seconds of device time have been timed.  run_region(r) enqueues one region's steps
+    and returns its device milliseconds (it may time every step by itself, see LayerBench).  Returns the list of
+    per-region milliseconds; every rank takes the same number of regions (the decision uses the reduced time)."""
+    out = []
+    total = 0.0
+    for r in range(max_regions):
+        _sync_all(dist)
+        ms = max_over_ranks(run_region(r), dist, dev)
+        out.append(ms)
+        total += ms
+        if total >= min_region_s * 1e3:
+            break
+    return out
+
+
+def median(v):
+    s = sorted(v)
+    n = len(s)
+    return s[n // 2] if n % 2 else 0.5 * (s[n // 2 - 1] + s[n // 2])
+
+
+class LayerBench:
+    """One single-layer workload on this rank's GPU: packed experts, four rotating token batches (inputs
+    resident in HBM), the workspace, and the algorithmic bytes of every batch from its realised routing."""
+
+    N_BATCHES = 4
+
+    def __init__(self, B, wl, T, path_name, dev, rank=0, blobs=None):
+        self.B, self.wl, self.T, self.dev, self.path_name = B, wl, T, dev, path_name
+        path = {"auto": B.PATH_AUTO, "cuda_core": B.PATH_CUDA_CORE, "tensor": B.PATH_TENSOR}[path_name]
+        self.cfg = B.Config.from_workload(wl, kernel_path=path)
+        if blobs is None:
+            blobs = []
+            for e in range(wl.n_experts + wl.n_shared):
+                for m in range(3):
+                    W = synth.expert_matrix(wl, e, m, device=dev)
+                    blobs.append(B.pack_mwq(self.cfg, W))
+                    del W
+        self.blobs = blobs
+        self.gw = synth.gate_weight_bf16(wl, dev)
+        nb = self.N_BATCHES
+        self.xs = [synth.tokens_bf16(wl, T, dev, step=rank * 100 + i) for i in range(nb)]
+        self.fbs = [synth.categorical(wl.seed + rank * 100 + i, synth.TID_FORCED_BITS, (T, wl.top_k), wl.bit_probs, dev)
+                    for i in range(nb)]
+        self.logits = [synth.zipf_logits(wl, T, dev) for _ in range(nb)] if wl.zipf_logits else None
+        self.ws = torch.empty(B.workspace_bytes(self.cfg, T), dtype=torch.uint8, device=dev)
+        self.y = torch.empty_like(self.xs[0])
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.alg = []
+        for i in range(nb):
+            r = B.route(self.cfg, self.xs[i], workspace=self.ws, **self.kw(i))
+            torch.cuda.synchronize()
+            self.alg.append(algorithmic_bytes(wl, T, r.group_off.cpu().tolist()))
+        self.layer_bytes = sum(a["layer"] for a in self.alg) / nb
+        # a step that streams less than a few L2 sizes could be served partly from L2 by the step before it:
+        # such workloads are timed step by step with an L2 flush (a 256 MiB write) between the steps
+        self.flush = self.layer_bytes < 4 * L2_BYTES
+        self.flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if self.flush else None
+        self.decode = -(-T * wl.top_k // wl.n_experts) <= 40
+
+    def kw(self, i, fb=None):
+        d = {"forced_bit_idx": self.fbs[i] if fb is None else fb}
+        if self.logits is not None:
+            d["logits"] = self.logits[i]
+        else:
+            d["gate_w"] = self.gw
+        return d
+
+    def step(self, i, events=None):
+        j = i % self.N_BATCHES
+        self.B.moe_forward(self.cfg, self.xs[j], self.blobs, y=self.y, workspace=self.ws, device_status=self.status,
+                           stage_events=events, **self.kw(j))
+
+    def region(self, steps, first=0):
+        """Enqueues `steps` uninstrumented steps and returns their device time in ms (waits for them)."""
+        stream = torch.cuda.current_stream()
+        if not self.flush:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(steps):
+                self.step(first + i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            self.flush_buf.zero_()
+            evs[i][0].record(stream)
+            self.step(first + i)
+            evs[i][1].record(stream)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs)
+
+    def stage_pass(self, steps):
+        """A separate, instrumented pass: the library records events around its stages on every step."""
+        B = self.B
+        stream = torch.cuda.current_stream()
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(B.N_STAGES + 1)] for _ in range(steps)]
+        for row in evs:
+            for ev in row:
+                ev.record(stream)                      # creates the handle
+        torch.cuda.synchronize()
+        for i in range(steps):
+            if self.flush:
+                self.flush_buf.zero_()
+            self.step(i, evs[i])
+        torch.cuda.synchronize()
+        stage_ms = [sum(evs[i][s].elapsed_time(evs[i][s + 1]) for i in range(steps)) / steps for s in range(B.N_STAGES)]
+        used = [self.alg[i % self.N_BATCHES] for i in range(steps)]
+        return stage_ms, used
+
+    def roofline(self, stage_ms, used, ms_per_step, clocks=None):
+        """Roofline of the stage with the largest device time, and of the whole layer call."""
+        B, wl, T = self.B, self.wl, self.T
+        names = B.STAGE_NAMES
+        dom = max(range(B.N_STAGES), key=lambda s: stage_ms[s])
+        dom_name = names[dom]
+        peak, peak_kind = measured_peaks()
+        dom_bytes = sum(u.get(dom_name, u["layer"]) for u in used) / len(used)
+        layer_bytes = sum(u["layer"] for u in used) / len(used)
+        achieved = dom_bytes / (stage_ms[dom] * 1e-3) / 1e9
+        rf = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+              "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+              "traffic": NCU_TRAFFIC.get(f"{wl.name}:T{T}:{dom_name}:{self.path_name}"),
+              "algorithmic_bytes_per_launch": dom_bytes,
+              "stage_ms": dict(zip(names, stage_ms)), "stage_samples": len(used),
+              "layer": {"algorithmic_bytes": layer_bytes,
+                        "achieved_gbs": layer_bytes / (ms_per_step * 1e-3) / 1e9,
+                        "frac": layer_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
+        dtype = "f32" if self.path_name == "cuda_core" else "i8"
+        if not self.decode and self.path_name != "cuda_core":
+            # prefill-sized expert loads (the grouped dequant-GEMM) are bound by the tensor cores: the dominant
+            # kernel against the measured dense 16-bit matmul rates (fp16 operands have the nominal rate of the
+            # bf16 the peaks were measured with); both the burst and the sustained (power-capped) figure
+            dtype = "f16"
+            A_tot = T * (wl.top_k + wl.n_shared)
+            flops = {"gate_up": A_tot * 2 * 2 * wl.d_model * wl.d_ffn, "down": A_tot * 2 * wl.d_model * wl.d_ffn}
+            burst, sustained, tkind = measured_tensor_peaks()
+            tf = flops.get(dom_name, sum(flops.values())) / (stage_ms[dom] * 1e-3) / 1e12
+            # a run short enough to stay at full clocks is compared with the burst figure, one that sits at the
+            # power cap with the sustained one
+            capped = bool(clocks and "sw_power_cap" in (clocks.get("reasons") or []))
+            tpeak = sustained if capped else burst
+            rf.update({"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
+                       "peak_kind": f"of {tkind} ({'sustained: run at the power cap' if capped else 'burst: run at full clocks'})",
+                       "frac_of_burst": tf / burst, "frac_of_sustained": tf / sustained,
+                       "algorithmic_flops_per_launch": flops.get(dom_name)})
+            lt = sum(flops.values()) / (ms_per_step * 1e-3) / 1e12
+            rf["layer"] = {"algorithmic_flops": sum(flops.values()), "achieved_tflops": lt, "frac": lt / tpeak}
+        return rf, dtype
+
+    def l2_note(self):
+        if self.flush:
+            return ("L2 flushed between steps: a 256 MiB buffer is written before every step (a step streams "
+                    f"{self.layer_bytes / 1e6:.0f} MB, less than four L2 sizes) and every step is timed by its own events")
+        return (f"inputs larger than L2: each step streams the routed planes of every active expert "
+                f"({self.layer_bytes / 1e6:.0f} MB per layer call against a 126 MB L2); four token batches are rotated")
+
+
+def measured_tensor_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+        except Exception:
+            pass
+    return 1590.0, 1400.0, "fallback"
+
+
+def workload_config(wl, T, path, l2=None):
     return {"workload": f"{wl.name} T={T}: d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} top{wl.top_k} "
-                        f"g={wl.group_size} bits={list(wl.bits)} p={list(wl.bit_probs)}",
-            "tokens_per_step": T, "kernel_path": path,
-            "l2": "inputs larger than L2: each step streams the routed planes of every active expert "
-                  "(>1 GB per layer call against a 126 MB L2); four token batches are rotated"}
+                        f"g={wl.group_size} bits={list(wl.bits)} p={list(wl.bit_probs)}"
+                        + (f" +{wl.n_shared} shared" if wl.n_shared else ""),
+            "tokens_per_step": T, "kernel_path": path, "l2": l2 or "inputs larger than L2"}
+
+
+def short_leg(B, wl, T, dev, blobs=None, steps=20, min_s=0.25):
+    """A short device-timed leg of another configuration (same rules: warm-up, regions of `steps` steps,
+    clocks sampled during the regions, stages from a separate pass)."""
+    lb = LayerBench(B, wl, T, "auto", dev, blobs=blobs)
+    for i in range(3):
+        lb.step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    regions = time_regions(lambda r: lb.region(steps, r * steps), steps, None, dev, min_s)
+    clocks = sampler.stop()
+    assert int(lb.status.item()) == 0, f"device status {int(lb.status.item())}"
+    ms = median(regions) / steps
+    stage_ms, used = lb.stage_pass(8)
+    rf, dtype = lb.roofline(stage_ms, used, ms, clocks)
+    return {"workload": workload_config(wl, T, "auto", lb.l2_note())["workload"], "tokens_per_step": T,
+            "ms_per_step": ms, "tokens_per_s": T / (ms * 1e-3), "dtype": dtype, "regions": len(regions),
+            "timed_region_s": sum(regions) * 1e-3, "l2": lb.l2_note(), "clocks": clocks, "roofline": rf}
 
 
 # ------------------------------------------------------------------------------------------------
 # layer stack (the 32-layer decode configuration): one step = every layer once, replayed as a CUDA graph
 # ------------------------------------------------------------------------------------------------
-def run_stack(args):
-    from paper_2504_15299_b200 import binding as B, build
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    build.build_library()
-    B.lib()
-    wl = synth.WORKLOADS[args.workload]
-    T = args.tokens or wl.tokens[-1]
-    L = args.layers or wl.n_layers
+def stack_bench(B, wl, T, L, dev, steps, warmup, use_graph=True, min_s=1.0, e2e=True):
     cfg = B.Config.from_workload(wl)
     layers = []
     for l in range(L):
@@ -318,7 +513,7 @@ def run_stack(args):
 
     side = torch.cuda.Stream()
     graph = None
-    if not args.no_graph:
+    if use_graph:
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
             one_step()                     # warm-up on the capture stream (function attributes, tensor maps)
@@ -335,64 +530,95 @@ def run_stack(args):
         else:
             one_step()
 
-    for i in range(max(args.warmup, 3)):
+    for i in range(max(warmup, 3)):
         step(i)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
-    torch.cuda.synchronize()
+
+    def region(r):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            step(r * steps + i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    regions = time_regions(region, steps, None, dev, min_s)
     clocks = sampler.stop()
-    ms_per_step = e0.elapsed_time(e1) / args.steps
+    ms_per_step = median(regions) / steps
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
-    # end to end: tokens from pinned host memory, the stack, result back to the host, every step
-    hx = [t.cpu().pin_memory() for t in xs]
-    hy = torch.empty_like(hx[0]).pin_memory()
+    e2e_out = None
+    if e2e:
+        # end to end: tokens from pinned host memory, the stack, result back to the host, every step
+        hx = [t.cpu().pin_memory() for t in xs]
+        hy = torch.empty_like(hx[0]).pin_memory()
 
-    def e2e_step(i):
-        x.copy_(hx[i % n_batches], non_blocking=True)
-        if graph is not None:
-            graph.replay()
-        else:
-            one_step()
-        hy.copy_(x, non_blocking=True)
+        def e2e_step(i):
+            x.copy_(hx[i % n_batches], non_blocking=True)
+            if graph is not None:
+                graph.replay()
+            else:
+                one_step()
+            hy.copy_(x, non_blocking=True)
 
-    for i in range(3):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for i in range(args.steps):
-        e2e_step(i)
-    f1.record()
-    torch.cuda.synchronize()
-    e2e_ms = f0.elapsed_time(f1) / args.steps
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(steps):
+            e2e_step(i)
+        f1.record()
+        torch.cuda.synchronize()
+        e2e_ms = f0.elapsed_time(f1) / steps
+        e2e_out = {"value": T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hx[0].numel() * 2,
+                   "d2h_bytes_per_step": hy.numel() * 2}
 
     peak, peak_kind = measured_peaks()
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
-    line = {"metric": METRIC, "value": T / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "i8", "data": "synthetic",
-            "config": {"workload": f"{wl.name}: {L} layers of d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} "
-                                   f"top{wl.top_k} g={wl.group_size} bits={list(wl.bits)}, widths from the per-expert "
-                                   f"bit-width routers, RMSNorm + residual per layer",
-                       "tokens_per_step": T, "layers": L, "cuda_graph": graph is not None,
-                       "l2": f"inputs larger than L2: {L} layers of distinct packed experts "
-                             f"({step_bytes / 1e9:.1f} GB read per step)"},
-            "clocks": clocks,
-            "e2e": {"value": T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hx[0].numel() * 2,
-                    "d2h_bytes_per_step": hy.numel() * 2},
-            "gpu_launches": (B.forward_launch_count(cfg, T) + 1) * L * args.steps,
+    return {"ms_per_step": ms_per_step, "tokens_per_s": T / (ms_per_step * 1e-3), "regions": regions,
+            "clocks": clocks, "e2e": e2e_out, "graph": graph is not None, "step_bytes": step_bytes,
+            "launches_per_step": (B.forward_launch_count(cfg, T) + 1) * L,
             "roofline": {"bound": "hbm", "kernel": "whole step", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                          "algorithmic_bytes_per_step": step_bytes},
-            "cpu_baseline": None}
+            "workload": f"{wl.name}: {L} layers of d={wl.d_model} ffn={wl.d_ffn} E={wl.n_experts} "
+                        f"top{wl.top_k} g={wl.group_size} bits={list(wl.bits)}, widths from the per-expert "
+                        f"bit-width routers, RMSNorm + residual per layer",
+            "l2": f"inputs larger than L2: {L} layers of distinct packed experts ({step_bytes / 1e9:.1f} GB read per step)"}
+
+
+def run_stack(args):
+    from paper_2504_15299_b200 import binding as B, build
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    build.build_library()
+    B.lib()
+    wl = synth.WORKLOADS[args.workload]
+    T = args.tokens or wl.tokens[-1]
+    L = args.layers or wl.n_layers
+    r = stack_bench(B, wl, T, L, dev, args.steps, args.warmup, use_graph=not args.no_graph, min_s=args.min_region_s)
+    n_reg = len(r["regions"])
+    line = {"metric": METRIC, "value": r["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "i8", "data": "synthetic",
+            "config": {"workload": r["workload"], "tokens_per_step": T, "layers": L, "cuda_graph": r["graph"], "l2": r["l2"]},
+            "timing": timing_block(r["regions"], args.steps),
+            "clocks": r["clocks"], "e2e": r["e2e"],
+            "gpu_launches": r["launches_per_step"] * args.steps * n_reg,
+            "roofline": r["roofline"], "cpu_baseline": None}
     print(json.dumps(line))
+
+
+def timing_block(regions, steps):
+    per = [ms / steps for ms in regions]
+    return {"regions": len(regions), "steps_per_region": steps, "timed_region_s": sum(regions) * 1e-3,
+            "ms_per_step_median": median(per), "ms_per_step_min": min(per), "ms_per_step_max": max(per),
+            "note": "each region is exactly `steps` steps between a barrier + synchronize on both sides; regions are "
+                    "repeated until at least --min-region-s seconds of device time are timed; value uses the median region"}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -418,92 +644,38 @@ def run_ours(args):
 
     wl = synth.WORKLOADS[args.workload]
     T = args.tokens or synth.WORKLOADS[args.workload].tokens[-1]
-    path = {"auto": B.PATH_AUTO, "cuda_core": B.PATH_CUDA_CORE, "tensor": B.PATH_TENSOR}[args.path]
-    cfg = B.Config.from_workload(wl, kernel_path=path)
-
-    blobs = []
-    for e in range(wl.n_experts + wl.n_shared):
-        for m in range(3):
-            W = synth.expert_matrix(wl, e, m, device=dev)
-            blobs.append(B.pack_mwq(cfg, W))
-            del W
-    gw = synth.gate_weight_bf16(wl, dev)
-    n_batches = 4
-    xs = [synth.tokens_bf16(wl, T, dev, step=rank * 100 + i) for i in range(n_batches)]
-    fbs = [synth.categorical(wl.seed + rank * 100 + i, synth.TID_FORCED_BITS, (T, wl.top_k), wl.bit_probs, dev)
-           for i in range(n_batches)]
-    logits = [synth.zipf_logits(wl, T, dev) for _ in range(n_batches)] if wl.zipf_logits else None
-    ws = torch.empty(B.workspace_bytes(cfg, T), dtype=torch.uint8, device=dev)
-    y = torch.empty_like(xs[0])
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-
-    def kw(i):
-        d = {"forced_bit_idx": fbs[i]}
-        if logits is not None:
-            d["logits"] = logits[i]
-        else:
-            d["gate_w"] = gw
-        return d
-
-    # realised routing of each batch -> algorithmic bytes
-    alg = []
-    for i in range(n_batches):
-        r = B.route(cfg, xs[i], workspace=ws, **kw(i))
-        torch.cuda.synchronize()
-        alg.append(algorithmic_bytes(wl, T, r.group_off.cpu().tolist()))
-
-    def step(i, events=None):
-        B.moe_forward(cfg, xs[i % n_batches], blobs, y=y, workspace=ws, device_status=status,
-                      stage_events=events, **kw(i % n_batches))
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
-            torch.cuda.synchronize()
+    lb = LayerBench(B, wl, T, args.path, dev, rank=rank)
+    stream = torch.cuda.current_stream()
 
     for i in range(args.warmup):
-        step(i)
-    sync_all()
+        lb.step(i)
+    _sync_all(dist)
 
-    # ---- timed region: K steps, device time, max over ranks ----
+    # ---- timed regions: K uninstrumented steps each, device time, max over ranks ----
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    stream = torch.cuda.current_stream()
-    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(B.N_STAGES + 1)] for _ in range(args.steps)]
-    for evs in stage_ev:
-        for ev in evs:
-            ev.record(stream)            # creates the handle
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    # per-stage events on every fifth step (with four batches in rotation every batch gets its share):
-    # recording five events per step costs about 3 % of a decode step, and the stage times are averages
-    # over the timed region anyway
-    ev_steps = [i for i in range(args.steps) if i % 5 == 0 or args.steps < 10]
-    for i in range(args.steps):
-        step(i, stage_ev[i] if (i % 5 == 0 or args.steps < 10) else None)
-    e1.record(stream)
-    sync_all()
+    regions = time_regions(lambda r: lb.region(args.steps, r * args.steps), args.steps, dist, dev, args.min_region_s)
+    _sync_all(dist)
     clocks = sampler.stop() if rank == 0 else None
-    ms_per_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
-    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    ms_per_step = median(regions) / args.steps
+    assert int(lb.status.item()) == 0, f"device status {int(lb.status.item())}"
 
-    stage_ms = [sum(stage_ev[i][s].elapsed_time(stage_ev[i][s + 1]) for i in ev_steps) / len(ev_steps)
-                for s in range(B.N_STAGES)]
+    # ---- per-stage device times: a separate pass with the library's stage events on every step ----
+    stage_ms, used = lb.stage_pass(min(max(args.steps, 8), 40))
 
     # ---- end to end: pinned host inputs -> device, layer, result back to the host, every step ----
     # The serving loop a user of the library would write: two sets of device buffers, the copies on streams of
     # their own, so that the copy-in of step i + 1 and the copy-out of step i - 1 overlap the layer call of
     # step i.  Every step's inputs come from pinned host memory and every step's result lands in pinned host
     # memory inside the timed region; the region ends when the last result has arrived.
-    hx = [x.cpu().pin_memory() for x in xs]
-    hfb = [f.cpu().pin_memory() for f in fbs]
+    nb = lb.N_BATCHES
+    hx = [x.cpu().pin_memory() for x in lb.xs]
+    hfb = [f.cpu().pin_memory() for f in lb.fbs]
     hy = [torch.empty_like(hx[0]).pin_memory() for _ in range(2)]
-    dx = [torch.empty_like(xs[0]) for _ in range(2)]
-    dfb = [torch.empty_like(fbs[0]) for _ in range(2)]
-    dy = [torch.empty_like(y) for _ in range(2)]
+    dx = [torch.empty_like(lb.xs[0]) for _ in range(2)]
+    dfb = [torch.empty_like(lb.fbs[0]) for _ in range(2)]
+    dy = [torch.empty_like(lb.y) for _ in range(2)]
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     ev_in = [torch.cuda.Event() for _ in range(2)]       # inputs of the buffer set have arrived
     ev_done = [torch.cuda.Event() for _ in range(2)]     # the layer call on the buffer set has finished
@@ -513,7 +685,7 @@ def run_ours(args):
         ev_out[b].record(stream)
 
     def e2e_step(i):
-        j, b = i % n_batches, i & 1
+        j, b = i % nb, i & 1
         with torch.cuda.stream(s_in):
             s_in.wait_event(ev_done[b])                   # the call two steps back has read these inputs
             dx[b].copy_(hx[j], non_blocking=True)
@@ -521,12 +693,7 @@ def run_ours(args):
             ev_in[b].record(s_in)
         stream.wait_event(ev_in[b])
         stream.wait_event(ev_out[b])                      # the result two steps back has been copied out
-        d = {"forced_bit_idx": dfb[b]}
-        if logits is not None:
-            d["logits"] = logits[j]
-        else:
-            d["gate_w"] = gw
-        B.moe_forward(cfg, dx[b], blobs, y=dy[b], workspace=ws, device_status=status, **d)
+        B.moe_forward(lb.cfg, dx[b], lb.blobs, y=dy[b], workspace=lb.ws, device_status=lb.status, **lb.kw(j, dfb[b]))
         ev_done[b].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_done[b])
@@ -535,57 +702,30 @@ def run_ours(args):
 
     for i in range(args.warmup):
         e2e_step(i)
-    sync_all()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(stream)
-    for i in range(args.steps):
-        e2e_step(args.warmup + i)
-    stream.wait_event(ev_out[0])
-    stream.wait_event(ev_out[1])
-    f1.record(stream)
-    sync_all()
-    e2e_ms = max_over_ranks(f0.elapsed_time(f1), dist, dev) / args.steps
+    _sync_all(dist)
+
+    def e2e_region(r):
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for i in range(args.steps):
+            e2e_step(args.warmup + r * args.steps + i)
+        stream.wait_event(ev_out[0])
+        stream.wait_event(ev_out[1])
+        f1.record(stream)
+        torch.cuda.synchronize()
+        return f0.elapsed_time(f1)
+
+    e2e_regions = time_regions(e2e_region, args.steps, dist, dev, min(args.min_region_s, 0.5))
+    _sync_all(dist)
+    e2e_ms = median(e2e_regions) / args.steps
 
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peaks()
-    used = [alg[i % n_batches] for i in ev_steps]          # the steps whose stages were timed
-    stage_names = B.STAGE_NAMES
-    dom = max(range(B.N_STAGES), key=lambda s: stage_ms[s])
-    dom_name = stage_names[dom]
-    dom_bytes = sum(u.get(dom_name, u["layer"]) for u in used) / len(used)
-    layer_bytes = sum(u["layer"] for u in used) / len(used)
-    achieved = dom_bytes / (stage_ms[dom] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
-                "algorithmic_bytes_per_launch": dom_bytes,
-                "stage_ms": dict(zip(stage_names, stage_ms)),
-                "stage_samples": len(ev_steps),
-                "layer": {"algorithmic_bytes": layer_bytes,
-                          "achieved_gbs": layer_bytes / (ms_per_step * 1e-3) / 1e9,
-                          "frac": layer_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
-    roofline["traffic"] = NCU_TRAFFIC.get(f"{args.workload}:T{T}:{dom_name}:{args.path}")
-    # prefill-sized expert loads (the grouped dequant-GEMM) are bound by the tensor cores: report
-    # the dominant kernel against the measured dense 16-bit matmul rate instead (fp16 operands have the
-    # same nominal rate as the bf16 the peak was measured with; sustained figure: kernel inside a step)
-    # arithmetic type of the expert kernels: the decode kernel multiplies unsigned 8-bit codes with signed
-    # 8-bit activation halves (int32 accumulation, fp32 scaling), the grouped GEMM runs on fp16 tiles
-    dtype = "f32" if args.path == "cuda_core" else "i8"
-    if -(-T * wl.top_k // wl.n_experts) > 40 and args.path != "cuda_core":
-        dtype = "f16"
-        A_tot = T * (wl.top_k + wl.n_shared)
-        flops = {"gate_up": A_tot * 2 * 2 * wl.d_model * wl.d_ffn, "down": A_tot * 2 * wl.d_model * wl.d_ffn}
-        tpeak, tkind = measured_tensor_peak()
-        tf = flops.get(dom_name, sum(flops.values())) / (stage_ms[dom] * 1e-3) / 1e12
-        roofline.update({"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s",
-                         "frac": tf / tpeak, "peak_kind": f"of {tkind}", "traffic": None,
-                         "algorithmic_flops_per_launch": flops.get(dom_name)})
-        roofline["layer"] = {"algorithmic_flops": sum(flops.values()),
-                             "achieved_tflops": sum(flops.values()) / (ms_per_step * 1e-3) / 1e12,
-                             "frac": sum(flops.values()) / (ms_per_step * 1e-3) / 1e12 / tpeak}
+    roofline, dtype = lb.roofline(stage_ms, used, ms_per_step, clocks)
+    lb_l2 = lb.l2_note()
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -595,20 +735,79 @@ def run_ours(args):
                          f"0..{hid - 1} of {wl.d_ffn} per expert, time scaled by {wl.d_ffn}/{hid} "
                          f"(extrapolated); 2 passes"}
 
+    # ---- the other configurations, short legs in the same invocation (one GPU only) ----
+    others = None
+    if world == 1 and args.others and args.workload == "mixtral_decode" and args.path == "auto":
+        others = []
+        for t in wl.tokens:
+            if t != T:
+                others.append(short_leg(B, wl, t, dev, blobs=lb.blobs))
+        wlp = synth.WORKLOADS["mixtral_prefill"]          # same seed and shapes: the same packed experts
+        others.append(short_leg(B, wlp, wlp.tokens[-1], dev, blobs=lb.blobs, steps=10))
+        wlf = synth.WORKLOADS["finegrained"]
+        others.append(short_leg(B, wlf, wlf.tokens[-1], dev))
+        torch.cuda.empty_cache()
+        if args.others == "all":
+            wls = synth.WORKLOADS["mixtral_stack"]
+            r = stack_bench(B, wls, wls.tokens[-1], wls.n_layers, dev, 10, 3, use_graph=True, min_s=0.5, e2e=False)
+            others.append({"workload": r["workload"], "tokens_per_step": wls.tokens[-1], "ms_per_step": r["ms_per_step"],
+                           "tokens_per_s": r["tokens_per_s"], "dtype": "i8", "regions": len(r["regions"]),
+                           "timed_region_s": sum(r["regions"]) * 1e-3, "l2": r["l2"], "clocks": r["clocks"],
+                           "cuda_graph": r["graph"], "roofline": r["roofline"]})
+
+    cfg_T = B.Config.from_workload(wl)
     line = {"metric": METRIC, "value": job_tokens_per_s(T, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype,
-            "data": "synthetic", "config": workload_config(wl, T, args.path),
+            "data": "synthetic", "config": workload_config(wl, T, args.path, lb_l2),
+            "timing": timing_block(regions, args.steps),
             "clocks": clocks,
             "e2e": {"value": job_tokens_per_s(T, world, e2e_ms), "unit": UNIT,
                     "h2d_bytes_per_step": hx[0].numel() * 2 + hfb[0].numel(),
-                    "d2h_bytes_per_step": hy[0].numel() * 2,
-                    "loop": "two buffer sets, copies on their own streams overlap the neighbouring steps' layer calls; "
-                            "no per-stage events in this loop (the device-timed loop records five per step)"},
-            "gpu_launches": B.forward_launch_count(cfg, T) * args.steps,
+                    "d2h_bytes_per_step": hy[0].numel() * 2, "regions": len(e2e_regions),
+                    "loop": "two buffer sets, copies on their own streams overlap the neighbouring steps' layer calls"},
+            "gpu_launches": B.forward_launch_count(cfg_T, T) * args.steps * len(regions),
             "roofline": roofline, "cpu_baseline": cpu}
+    if others is not None:
+        line["other_workloads"] = others
     print(json.dumps(line))
     if dist:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# launch path
+# ------------------------------------------------------------------------------------------------
+def _free_port():
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def replica_command(n, argv, port=None):
+    """The command that starts n replica processes of this script on one node (one rank per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port or _free_port()),
+            os.path.abspath(__file__), *argv]
+
+
+def run_selfcheck(args):
+    """Launch-path check without a GPU: every rank joins a gloo group, reports a made-up step time that grows
+    with its rank, and rank 0 prints the job line the real arm would print for those times."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = max_over_ranks(1.0 + rank, dist if world > 1 else None, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"impl": "selfcheck", "n_gpus": world, "ms_per_step": ms,
+                          "value": job_tokens_per_s(64, world, ms), "unit": UNIT}))
+    if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
 
 
@@ -617,7 +816,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "selfcheck"])
     ap.add_argument("--workload", default="mixtral_decode", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0,
                     help="tokens per step (default: the largest batch size of the workload, 64 for mixtral_decode)")
@@ -626,11 +825,25 @@ def main():
                     help="mixtral_stack only: layers per step (default: the workload's 32; 46 GB of packed experts)")
     ap.add_argument("--no-graph", action="store_true", help="mixtral_stack only: launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-region-s", type=float, default=1.0,
+                    help="repeat the timed K-step region until this much device time has been timed")
+    ap.add_argument("--others", default="all", choices=["all", "layers", "none"],
+                    help="after the headline, short legs of the other configurations (default workload, one GPU): "
+                         "all = single-layer ones and the 32-layer stack, layers = single-layer ones only")
     args = ap.parse_args()
+    if args.others == "none":
+        args.others = ""
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    world = int(os.environ.get("WORLD_SIZE", "0"))
+    if args.gpus > 1 and world == 0 and args.impl != "reference":
+        # started as a plain script: start the replicas ourselves (one process per GPU) and pass their line on
+        import subprocess
+        sys.exit(subprocess.run(replica_command(args.gpus, sys.argv[1:])).returncode)
     if args.impl == "reference":
         run_reference(args)
-    elif synth.WORKLOADS[args.workload].n_layers > 1 and int(os.environ.get("WORLD_SIZE", "1")) == 1:
+    elif args.impl == "selfcheck":
+        run_selfcheck(args)
+    elif synth.WORKLOADS[args.workload].n_layers > 1 and world <= 1:
         run_stack(args)
     else:
         run_ours(args)

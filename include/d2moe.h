@@ -39,8 +39,8 @@ typedef enum {
 } d2moe_status;
 
 /* bits set in *device_status */
-#define D2MOE_DEV_NONFINITE 0x1  /* a router logit, or (decode kernel) an activation row, held a NaN or an
-                                    infinity; the outputs of such a row are zero                 */
+#define D2MOE_DEV_NONFINITE 0x1  /* a router logit or an activation row held a NaN or an infinity (the
+                                    outputs of such a row are zero), or an intermediate left fp16's range */
 #define D2MOE_DEV_TIMEOUT   0x2
 #define D2MOE_DEV_BAD_INDEX 0x4  /* a supplied routing index was out of range and was skipped */
 
@@ -49,12 +49,17 @@ typedef enum {
 #define D2MOE_PATH_CUDA_CORE 1   /* plain fp32 CUDA-core kernels (any supported shape)          */
 #define D2MOE_PATH_TENSOR    2   /* tcgen05 grouped kernels; D2MOE_ERR_UNSUPPORTED if not possible */
 
+#define D2MOE_MAX_DIM 262144      /* largest d_model / d_ffn */
+#define D2MOE_MAX_TOKENS 1048576  /* largest T of one call   */
+
 /*
  * One MoE layer.  Candidate widths {b_k} of Section 3.3.1 are `bits[0..n_bits-1]`, ascending,
  * 1 <= bits[0], bits[n_bits-1] <= 8; every expert matrix is stored once at the top width and read
  * at any listed width (the nested store).  `group_size` is g of Eq. 2 (groups run along the input
  * dimension of each matrix) and must be a multiple of 32.  Experts are SwiGLU FFNs without bias:
- * gate and up projections [d_ffn, d_model], down projection [d_model, d_ffn].
+ * gate and up projections [d_ffn, d_model], down projection [d_model, d_ffn].  d_model and d_ffn are
+ * at most D2MOE_MAX_DIM, a call takes at most D2MOE_MAX_TOKENS tokens (D2MOE_ERR_CONFIG /
+ * D2MOE_ERR_SHAPE otherwise, before anything is launched).
  */
 typedef struct {
     int32_t d_model, d_ffn, n_experts, top_k, n_shared, group_size;
@@ -142,7 +147,9 @@ d2moe_status d2moe_route(const d2moe_config* cfg, int64_t T,
  *   - Limits: T * top_k <= D2MOE_STATIC_MAX_ASSIGNMENTS and n_experts * n_bits <=
  *     D2MOE_STATIC_MAX_KEYS; anything larger is refused with D2MOE_ERR_WORKSPACE before any launch.
  *   - The first call on each device looks up the array's device address (with that device current)
- *     and remembers it; make that first call outside any stream capture.
+ *     and remembers it for the life of the process; make that first call outside any stream capture.
+ *     cudaDeviceReset (or any other teardown of the device's primary context) invalidates the remembered
+ *     address: do not call this entry point on that device afterwards.
  *   - All calls on a device share the one array.  Calls that may overlap on the GPU (different
  *     streams, or graphs replayed concurrently) race on it and give wrong routing; serialise them.
  *     Nothing needs clearing between calls: every scratch word is written before it is read.
@@ -179,8 +186,18 @@ typedef struct {                    /* outputs of an earlier d2moe_route on the 
  *   in        routing inputs (see d2moe_route); ignored when `pre` is given
  *   pre       optional: routing already computed by d2moe_route (same T, same stream order)
  *   y_bf16    device bf16 [T, d_model], overwritten
- * Arithmetic: weights dequantized to 16-bit floating point in registers, fp32 accumulation, bf16
- * output (round to nearest even).  T == 0 is a no-op.
+ * Arithmetic.  Decode-sized loads (at most 40 tokens per expert on average): the packed codes are
+ * multiplied as they are, as unsigned 8-bit integers, with the activations quantised per token to 15-bit
+ * integers against the token's largest element (int32 accumulation; scales and offsets of Eq. 2 applied to
+ * the accumulators in fp32).  That quantisation adds at most sqrt(n) / 56000 of an output's rms (n = length
+ * of the dot product), whatever the spread of magnitudes inside the token.  Larger loads: weights
+ * dequantized to fp16 in registers (the "dequantized to FP16" of Section 3.3.1), every token row scaled by
+ * a power of two of its own so that tokens of any bf16 magnitude fit the fp16 products, h = silu(g) * u
+ * stored as fp16 at the square of that scale, fp32 accumulation.  The CUDA-core path is fp32 throughout.
+ * Output: bf16, round to nearest even.  A token row that holds a NaN or an infinity gives a zero output
+ * row and D2MOE_DEV_NONFINITE; so does an h beyond fp16 even at its token's scale (that element is taken
+ * as zero).  An index of `pre` that is out of range (expert, width index, or a position outside its
+ * group) makes its assignment contribute nothing and raises D2MOE_DEV_BAD_INDEX.  T == 0 is a no-op.
  */
 d2moe_status d2moe_moe_forward(const d2moe_config* cfg, int64_t T, const void* x_bf16,
                                const void* const* expert_w, const d2moe_route_in* in,

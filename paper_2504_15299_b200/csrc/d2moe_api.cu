@@ -41,6 +41,7 @@ extern "C" d2moe_status d2moe_check_config(const d2moe_config* c) {
     if (c->d_model <= 0 || c->d_ffn <= 0 || c->n_experts <= 0 || c->top_k <= 0 || c->n_shared < 0)
         return D2MOE_ERR_CONFIG;
     if (c->top_k > c->n_experts || c->top_k > 8) return D2MOE_ERR_CONFIG;
+    if (c->d_model > D2MOE_MAX_DIM || c->d_ffn > D2MOE_MAX_DIM) return D2MOE_ERR_CONFIG;   // what every launch can take
     if (c->n_experts > 256 || c->n_experts + c->n_shared > D2MOE_MAX_EXPERTS) return D2MOE_ERR_CONFIG;
     const int g = c->group_size;
     if (!(g == 32 || g == 64 || g == 128 || g == 256)) return D2MOE_ERR_CONFIG;
@@ -142,12 +143,12 @@ void d2moe_carve_workspace(const d2moe_config* c, long long T, Workspace* ws) {
         tc_plan(c, pl.decode ? 1 : (t_dec + 1 < T ? t_dec + 1 : T), &pl_lo);
         const int n_split_alloc = pl_lo.n_split > pl.n_split ? pl_lo.n_split : pl.n_split;
         ws->off_o = take((size_t)n_split_alloc * pl.R_alloc * c->d_model * 4);
-        ws->off_h32 = ws->off_xk_x = ws->off_xk_h = ws->off_slot_f = 0;
+        ws->off_h32 = ws->off_xk_x = ws->off_xk_h = 0;
+        ws->off_slot_f = take((size_t)3 * pl.R_alloc * 4);      // per padded row: three scale factors (either kernel)
         if (pl.decode) {
             ws->off_h32 = take((size_t)pl.R_alloc * c->d_ffn * 4);
             ws->off_xk_x = take((size_t)(c->d_model / c->group_size) * pl.R_alloc * 8);
             ws->off_xk_h = take((size_t)(c->d_ffn / c->group_size) * pl.R_alloc * 8);
-            ws->off_slot_f = take((size_t)3 * pl.R_alloc * 4);
         }
     } else {
         ws->off_units = ws->off_n_units = ws->off_pad_off = ws->off_row_map = ws->off_src_token = ws->off_xp16 = 0;

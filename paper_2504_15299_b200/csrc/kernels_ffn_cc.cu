@@ -69,13 +69,13 @@ __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed
     return acc;
 }
 
-// h[a, r] = silu(Wg_{e,b}[r,:] . x_t) * (Wu_{e,b}[r,:] . x_t);  grid (ceil(F/8), A_tot), 8 warps.
+// h[a, r] = silu(Wg_{e,b}[r,:] . x_t) * (Wu_{e,b}[r,:] . x_t);  grid (A_tot, ceil(F/8)), 8 warps.
 __global__ void __launch_bounds__(256)
 gateup_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, const __nv_bfloat16* __restrict__ x, RouteBufs R,
                  float* __restrict__ hbuf, int32_t* device_status) {
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int a = blockIdx.y;
+    const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
+    const int a = blockIdx.x;                       // assignments on the x dimension: no 65535 limit
     if (row >= D.F) return;
     int t, e, kk;
     if (!resolve_assignment(D, R, a, &t, &e, &kk, device_status)) {
@@ -88,13 +88,13 @@ gateup_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, const __nv_bfloat16* __r
     if (lane == 0) hbuf[(size_t)a * D.F + row] = g / (1.0f + expf(-g)) * u;
 }
 
-// o[a, r] = Wd_{e,b}[r,:] . h[a,:];  grid (ceil(d/8), A_tot)
+// o[a, r] = Wd_{e,b}[r,:] . h[a,:];  grid (A_tot, ceil(d/8))
 __global__ void __launch_bounds__(256)
 down_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, RouteBufs R, const float* __restrict__ hbuf,
                float* __restrict__ obuf, int32_t* device_status) {
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int a = blockIdx.y;
+    const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
+    const int a = blockIdx.x;
     if (row >= D.d) return;
     int t, e, kk;
     if (!resolve_assignment(D, R, a, &t, &e, &kk, nullptr)) {
@@ -111,15 +111,17 @@ down_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, RouteBufs R, const float* 
 __global__ void combine_kernel(MoeDims D, RouteBufs R, const float* __restrict__ obuf, int n_split,
                                size_t split_stride, const int32_t* __restrict__ row_map,
                                const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ y) {
-    const int t = blockIdx.y;
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int t = blockIdx.x;                       // tokens on the x dimension: no 65535 limit
+    const int c = blockIdx.y * blockDim.x + threadIdx.x;
     if (c >= D.d) return;
     float acc = residual ? __bfloat162float(residual[(size_t)t * D.d + c]) : 0.0f;
     float sum = 0.0f;
     for (int s = 0; s < D.k + D.n_shared; ++s) {
         const int a = s < D.k ? t * D.k + s : D.A + (s - D.k) * D.T + t;
         const float w = s < D.k ? R.topk_w[a] : 1.0f;
-        const size_t row = row_map ? (size_t)row_map[a] : (size_t)a;
+        const long long rowi = row_map ? (long long)row_map[a] : (long long)a;
+        if (rowi < 0) continue;                      // an assignment that was skipped (bad routing index)
+        const size_t row = (size_t)rowi;
         float o = 0.0f;
         for (int sp = 0; sp < n_split; ++sp) o += obuf[sp * split_stride + row * D.d + c];
         sum = fmaf(w, o, sum);
@@ -132,8 +134,8 @@ __global__ void combine_kernel(MoeDims D, RouteBufs R, const float* __restrict__
 __global__ void combine4_kernel(MoeDims D, RouteBufs R, const float* __restrict__ obuf, int n_split,
                                 size_t split_stride, const int32_t* __restrict__ row_map,
                                 const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ y) {
-    const int t = blockIdx.y;
-    const int c = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
+    const int t = blockIdx.x;
+    const int c = 4 * (blockIdx.y * blockDim.x + threadIdx.x);
     if (c >= D.d) return;
     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     if (residual) {
@@ -146,7 +148,9 @@ __global__ void combine4_kernel(MoeDims D, RouteBufs R, const float* __restrict_
     for (int s = 0; s < D.k + D.n_shared; ++s) {
         const int a = s < D.k ? t * D.k + s : D.A + (s - D.k) * D.T + t;
         const float w = s < D.k ? R.topk_w[a] : 1.0f;
-        const size_t row = row_map ? (size_t)row_map[a] : (size_t)a;
+        const long long rowi = row_map ? (long long)row_map[a] : (long long)a;
+        if (rowi < 0) continue;                      // an assignment that was skipped (bad routing index)
+        const size_t row = (size_t)rowi;
         float o[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         for (int sp = 0; sp < n_split; ++sp) {
             const float4 v = *reinterpret_cast<const float4*>(obuf + sp * split_stride + row * D.d + c);
@@ -193,7 +197,7 @@ cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, con
                                     const __nv_bfloat16* x, const RouteBufs& R, float* hbuf,
                                     int32_t* device_status, cudaStream_t st) {
     if (D.A_tot == 0) return cudaSuccess;
-    dim3 g1((D.F + 7) / 8, D.A_tot);
+    dim3 g1(D.A_tot, (D.F + 7) / 8);
     gateup_cc_kernel<<<g1, 256, 0, st>>>(D, Lgu, P, x, R, hbuf, device_status);
     return cudaGetLastError();
 }
@@ -202,7 +206,7 @@ cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const 
                                   const RouteBufs& R, const float* hbuf, float* obuf,
                                   int32_t* device_status, cudaStream_t st) {
     if (D.A_tot == 0) return cudaSuccess;
-    dim3 g2((D.d + 7) / 8, D.A_tot);
+    dim3 g2(D.A_tot, (D.d + 7) / 8);
     down_cc_kernel<<<g2, 256, 0, st>>>(D, Ld, P, R, hbuf, obuf, device_status);
     return cudaGetLastError();
 }
@@ -214,10 +218,10 @@ cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* ob
     const bool vec = D.d % 4 == 0 && split_stride % 4 == 0 && ((uintptr_t)obuf & 15) == 0 && ((uintptr_t)y & 7) == 0 &&
                      ((uintptr_t)residual & 7) == 0;
     if (vec) {
-        dim3 grid((D.d / 4 + 127) / 128, D.T);
+        dim3 grid(D.T, (D.d / 4 + 127) / 128);
         combine4_kernel<<<grid, 128, 0, st>>>(D, R, obuf, n_split, split_stride, row_map, residual, y);
     } else {
-        dim3 grid((D.d + 255) / 256, D.T);
+        dim3 grid(D.T, (D.d + 255) / 256);
         combine_kernel<<<grid, 256, 0, st>>>(D, R, obuf, n_split, split_stride, row_map, residual, y);
     }
     return cudaGetLastError();

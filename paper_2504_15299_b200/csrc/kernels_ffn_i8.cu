@@ -86,21 +86,6 @@ struct I8Params {
 
 struct I8Item { int unit, tile, split, g0, g1; };
 
-#ifdef D2MOE_WAIT_STATS
-// Debug build only: cycles per wait category, summed over all CTAs.  0 wprod.w_empty 1 bprod.b_empty
-// 2 mma.d_empty 3 mma.b_full 4 mma.a_full 5 mma.total 6 deq.w_full 7 deq.a_empty 8 deq.wait_st
-// 9 deq.d_full 10 deq.total 11 deq.fold 12 deq.unpack 13 groups 14 deq.output
-__device__ unsigned long long g_i8_stats[16];
-#define I8S_T0() const long long _t0 = clock64()
-#define I8S_ADD(slot) stat[slot] += clock64() - _t0
-#define I8S_DECL() long long stat[16] = {0}
-#define I8S_FLUSH(cond) do { if (cond) { for (int _i = 0; _i < 16; ++_i) if (stat[_i]) atomicAdd(&g_i8_stats[_i], (unsigned long long)stat[_i]); } } while (0)
-#else
-#define I8S_T0()
-#define I8S_ADD(slot)
-#define I8S_DECL()
-#define I8S_FLUSH(cond)
-#endif
 
 __device__ __forceinline__ I8Item i8_item(const I8Params& p, int item) {
     I8Item it;
@@ -326,7 +311,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     if (warp == I8_WARP_PROD) {
         // One producer thread feeds both rings, stage by stage (they are consumed at the same rate).
         if (lane == 0) {
-            I8S_DECL();
             // This thread shares a scheduler with unpack warps, so its loop is kept short: source pointers and
             // ring positions advance by addition, nothing is recomputed per stage.
             uint32_t it = 0, ws = 0, wph = 1, bs = 0, bph = 1;         // ring positions, parity of the "empty" waits
@@ -362,7 +346,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 for (int G = ii.g0; G < ii.g1; G += GPS, ++it) {
                     const int ng = min(GPS, ii.g1 - G);
                     {
-                        { I8S_T0(); mbar_wait_blk(W_EMPTY(ws), wph); I8S_ADD(0); }
+                        mbar_wait_blk(W_EMPTY(ws), wph);
                         mbar_expect_tx(W_FULL(ws), 2 * bytes * ng);
                         const uint32_t dst = wbuf + ws * w_slot_bytes;
 #pragma unroll
@@ -376,7 +360,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1u; }
                     }
                     {
-                        { I8S_T0(); mbar_wait_blk(B_EMPTY(bs), bph); I8S_ADD(1); }
+                        mbar_wait_blk(B_EMPTY(bs), bph);
                         mbar_expect_tx(B_FULL(bs), tile_bytes + ng * xk_bytes);
                         tma_load_2d(bbuf + bs * I8_B_TILE, map, G * GS, 2 * slot0, B_FULL(bs));
 #pragma unroll
@@ -399,7 +383,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const uint32_t last = it - 1 - (it - 1 - s) % I8_NSB;
                 mbar_wait(B_FULL(s), (last / I8_NSB) & 1, abort_flag, p.status, true);
             }
-            I8S_FLUSH(true);
         }
     } else if (warp == I8_WARP_MMA) {
         // One issuer: all segments of a group accumulate into the same columns, so their products
@@ -407,10 +390,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // addresses and descriptors stay in the uniform datapath.  A warpgroup hands over up to two
         // operand tiles at a time (its segments j and j + 2).
         uint32_t gc = 0, bs = 0, bph = 0, hs[2] = {0, 0};
-        I8S_DECL();
-#ifdef D2MOE_WAIT_STATS
-        const long long _tt = clock64();
-#endif
         for (uint32_t qi = 0;; ++qi) {
             const uint32_t q = qi & (I8_NSQ - 1);
             mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
@@ -426,13 +405,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int j = 0; j < 8; ++j) idesc[j] = instr_desc_i8(2 * max(u->npad[j], 8));
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
-                { I8S_T0(); mbar_wait_blk(B_FULL(bs), bph); I8S_ADD(3); }
+                mbar_wait_blk(B_FULL(bs), bph);
                 const uint64_t bdesc = smem_desc_sw128(bbuf + bs * I8_B_TILE);
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
                     if (sub < ng) {
                         const int buf = gc & 1;
-                        { I8S_T0(); mbar_wait_blk(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1); I8S_ADD(2); }
+                        mbar_wait_blk(D_EMPTY(buf), ((gc >> 1) & 1) ^ 1);
                         tc_fence_after();
                         const uint32_t d_addr = d_tmem + buf * I8_D_COLS;
 #pragma unroll
@@ -441,7 +420,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                             for (int wg = 0; wg < 2; ++wg) {
                                 const int j0 = wg + 4 * hp, j1 = j0 + 2;
                                 if (j0 <= kmax) {
-                                    { I8S_T0(); mbar_wait_blk(A_FULL(wg, 0), hs[wg] & 1); I8S_ADD(4); }
+                                    mbar_wait_blk(A_FULL(wg, 0), hs[wg] & 1);
                                     tc_fence_after();
                                     const uint32_t a_addr = a_tmem + wg * 64;
                                     if (elect_one()) {
@@ -475,10 +454,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // all products have completed before TMEM is released
         if (gc > 0) mbar_wait(D_FULL((gc - 1) & 1), ((gc - 1) >> 1) & 1, abort_flag, p.status, true);
         if (gc > 1) mbar_wait(D_FULL((gc - 2) & 1), ((gc - 2) >> 1) & 1, abort_flag, p.status, true);
-#ifdef D2MOE_WAIT_STATS
-        stat[5] = clock64() - _tt;
-#endif
-        I8S_FLUSH(lane == 0);
     } else if (warp < 8) {
         // -------- two warpgroups: unpack (segments wg, wg+2, ... of every group), fold, write out --------
         const int wg = warp >> 2;
@@ -490,10 +465,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         uint32_t gc = 0, hs = 0;                   // groups folded / operand hand-offs so far
         uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
         uint32_t w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
-        I8S_DECL();
-#ifdef D2MOE_WAIT_STATS
-        const long long _tt = clock64();
-#endif
         for (uint32_t qi = 0;; ++qi) {
             const uint32_t q = qi & (I8_NSQ - 1);
             mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
@@ -535,9 +506,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             // sub: group inside the stage, rel: last group of the stage (the stage is released afterwards)
             auto fold = [&](uint32_t g, uint32_t fbs, uint32_t fbph, int sub, bool rel, uint32_t meta) {
                 const int buf = g & 1;
-                { I8S_T0(); mbar_wait_blk(D_FULL(buf), (g >> 1) & 1); I8S_ADD(9); }
+                mbar_wait_blk(D_FULL(buf), (g >> 1) & 1);
                 tc_fence_after();
-                I8S_T0();
                 const __half2 mh = as_h2(meta);
                 const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
                 const float lo = __high2float(mh);
@@ -574,7 +544,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B_EMPTY(fbs));
                 }
-                I8S_ADD(11);
             };
 
             bool pend = false;
@@ -583,7 +552,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             bool pend_rel = true;
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
-                { I8S_T0(); mbar_wait_blk(W_FULL(ws), wph); I8S_ADD(6); }
+                mbar_wait_blk(W_FULL(ws), wph);
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
                     if (sub < ng) {
@@ -591,11 +560,11 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         uint32_t meta;
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
                         auto handoff_begin = [&]() {
-                            { I8S_T0(); mbar_wait_blk(A_EMPTY(wg, 0), (hs & 1) ^ 1); I8S_ADD(7); }
+                            mbar_wait_blk(A_EMPTY(wg, 0), (hs & 1) ^ 1);
                             tc_fence_after();
                         };
                         auto handoff_end = [&]() {
-                            { I8S_T0(); tc_wait_st(); I8S_ADD(8); }
+                            tc_wait_st();
                             tc_fence_before();
                             mbar_arrive(A_FULL(wg, 0));
                             ++hs;
@@ -613,12 +582,10 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                             };
                             if (wg <= kmax) {
                                 handoff_begin();
-                                I8S_T0();
                                 do_seg(std::integral_constant<int, 0>{});
                                 do_seg(std::integral_constant<int, 1>{});
                                 do_seg(std::integral_constant<int, 2>{});
                                 do_seg(std::integral_constant<int, 3>{});
-                                I8S_ADD(12);
                                 handoff_end();
                             }
                         } else {
@@ -637,9 +604,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         pend_meta = meta;
                         pend_bs = bs; pend_bph = bph; pend_sub = sub; pend_rel = sub == ng - 1;
                         ++gc;
-#ifdef D2MOE_WAIT_STATS
-                        stat[13] += 1;
-#endif
                     }
                 }
                 mbar_arrive(W_EMPTY(ws));
@@ -650,19 +614,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             if (pend) fold(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
-            I8S_T0();
             float out[4][4];                   // a copy: acc itself must stay in registers
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int q = 0; q < 4; ++q) out[i][q] = acc[i][q];
             i8_write_out(p, wg, r, n_mine, myblks, out, smem);
-            I8S_ADD(14);
         }
-#ifdef D2MOE_WAIT_STATS
-        stat[10] = clock64() - _tt;
-#endif
-        I8S_FLUSH((threadIdx.x & 127) == 0);
     }
 
     tc_fence_before();
@@ -684,7 +642,7 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints).
 __global__ void __launch_bounds__(256)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
-               int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid) {
+               int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status) {
     extern __shared__ int32_t s_prep[];
     __shared__ int s_total;
     const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
@@ -728,15 +686,25 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     for (int a = threadIdx.x; a < D.A; a += blockDim.x) {
         const int pos = R.inv_perm[a];
         const int e = R.topk_idx[a], kk = R.bit_idx[a];
-        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) { row_map[a] = 0; continue; }
+        // a supplied routing index out of range: the assignment is skipped (row -1 contributes nothing to the
+        // combine; its slot stays a padding slot) and the call is flagged
+        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) {
+            row_map[a] = -1;
+            if (status) atomicOr(status, D2MOE_DEV_BAD_INDEX);
+            continue;
+        }
         int start = 0;                            // classes of a larger width index come first
         for (int i = kk + 1; i < D.K; ++i) start += round8(go[e * D.K + i + 1] - go[e * D.K + i]);
         const int slot = pad_off[e] + start + (pos - go[e * D.K + kk]);
-        row_map[a] = slot;
-        if (slot >= 0 && slot < total) {
-            src_token[slot] = a / D.k;
-            kappa[slot] = exp2f((float)(top - D.bits[kk] - 1)) - exp2f((float)(top - b1 - 1));
+        // pos must lie inside the group of (e, kk); otherwise the permutation does not belong to these indices
+        if (pos < go[e * D.K + kk] || pos >= go[e * D.K + kk + 1] || slot < 0 || slot >= total) {
+            row_map[a] = -1;
+            if (status) atomicOr(status, D2MOE_DEV_BAD_INDEX);
+            continue;
         }
+        row_map[a] = slot;
+        src_token[slot] = a / D.k;
+        kappa[slot] = exp2f((float)(top - D.bits[kk] - 1)) - exp2f((float)(top - b1 - 1));
     }
     for (int i = threadIdx.x; i < D.n_shared * D.T; i += blockDim.x) {
         const int s = i / D.T, t = i - s * D.T;
@@ -910,18 +878,6 @@ static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long 
     return true;
 }
 
-}  // namespace
-
-#ifdef D2MOE_WAIT_STATS
-extern "C" int d2moe_debug_i8_stats(unsigned long long* host16, int reset) {
-    cudaDeviceSynchronize();
-    if (cudaMemcpyFromSymbol(host16, g_i8_stats, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
-    if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_i8_stats, z, sizeof(z)); }
-    return 0;
-}
-#endif
-
-namespace {
 // One block waits on a barrier that nothing completes, with either of the two bounded waits of the
 // expert kernels; the barrier block has the layout those waits expect (status pointer at byte 496, abort
 // flag at byte 504 of a 512-byte aligned block).  A second wait follows: with the abort flag set it
@@ -976,7 +932,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     const int ffn_grid = 2 * sms;
     const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
     i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
-                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid);
+                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status);
     i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
                                                     qx, B.xk_x, sigma_x, device_status);
 

@@ -59,6 +59,7 @@ struct TcParams {
     int* next_item;           // work counter of this launch: starts at the grid size (item i < grid goes to CTA i)
     __half* hbuf;             // [R, F]
     float* obuf;              // [n_split][R, d]
+    const float* row_scale;   // [3][R]: per padded row the power-of-two factors of the activation scaling (see tc_gather_kernel)
     long long R_alloc;
     int32_t* status;
     int smem_w_off, smem_epi_off, smem_bar_off;
@@ -472,9 +473,20 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 if (nreal == 0) continue;            // padding columns only (uniform across the warpgroup)
                 uint32_t v[16];
                 tc_ld16(d_tmem + lane_addr + c0, v);
-                tc_wait_ld();
                 const long long grow = u->row0 + c0;
                 if (p.mode == 0) {
+                    // the tokens this thread finishes, and their scales: xs undoes the scaling of the activation
+                    // row, hq is the factor h is stored with (both powers of two; 32-byte aligned: grow % 16 == 0)
+                    const int keep = blk == 0 ? 0 : 8;
+                    float xs[8], hq[8];
+                    {
+                        const float4* a = reinterpret_cast<const float4*>(p.row_scale + grow + keep);
+                        const float4* b = reinterpret_cast<const float4*>(p.row_scale + p.R_alloc + grow + keep);
+                        const float4 a0 = a[0], a1 = a[1], b0 = b[0], b1 = b[1];
+                        xs[0] = a0.x; xs[1] = a0.y; xs[2] = a0.z; xs[3] = a0.w; xs[4] = a1.x; xs[5] = a1.y; xs[6] = a1.z; xs[7] = a1.w;
+                        hq[0] = b0.x; hq[1] = b0.y; hq[2] = b0.z; hq[3] = b0.w; hq[4] = b1.x; hq[5] = b1.y; hq[6] = b1.z; hq[7] = b1.w;
+                    }
+                    tc_wait_ld();
                     // exchange: the gate thread publishes tokens 8..15, the up thread tokens 0..7
                     const int give = blk == 0 ? 8 : 0;
 #pragma unroll
@@ -484,25 +496,39 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     mbar_arrive(EPI_BAR(wg));
                     mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
                     eph ^= 1u;
-                    const int keep = blk == 0 ? 0 : 8;           // the tokens this thread finishes
                     __half* dst = p.hbuf + (grow + keep) * p.D.F + (long long)ii.tile * 64 + rr;
+                    bool over = false;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         if (keep + j < nreal) {
-                            const float mine = __uint_as_float(v[keep + j]) * two_S;
-                            const float other = epi[((1 - blk) * 64 + rr) * 9 + j];
+                            const float mine = __uint_as_float(v[keep + j]) * two_S * xs[j];
+                            const float other = epi[((1 - blk) * 64 + rr) * 9 + j] * xs[j];
                             const float g = blk == 0 ? mine : other, up = blk == 0 ? other : mine;
-                            dst[(long long)j * p.D.F] = __float2half_rn(__fdividef(g, 1.0f + __expf(-g)) * up);
+                            float h = __fdividef(g, 1.0f + __expf(-g)) * up * hq[j];
+                            // beyond fp16 even at the token's own scale (or not a number): stored as zero, call flagged
+                            if (!(fabsf(h) <= 65504.0f)) { h = 0.0f; over = true; }
+                            dst[(long long)j * p.D.F] = __float2half_rn(h);
                         }
                     }
+                    if (over && p.status) atomicOr(p.status, D2MOE_DEV_NONFINITE);
                     mbar_arrive(EPI_BAR(wg));
                     mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
                     eph ^= 1u;
                 } else {
+                    float hs[16];                                // undoes the factor h was stored with
+                    {
+                        const float4* a = reinterpret_cast<const float4*>(p.row_scale + 2 * p.R_alloc + grow);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 t4 = a[q];
+                            hs[4 * q] = t4.x; hs[4 * q + 1] = t4.y; hs[4 * q + 2] = t4.z; hs[4 * q + 3] = t4.w;
+                        }
+                    }
+                    tc_wait_ld();
                     float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + r;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (j < nreal) dst[(long long)j * p.D.d] = __uint_as_float(v[j]) * two_S;
+                        if (j < nreal) dst[(long long)j * p.D.d] = __uint_as_float(v[j]) * two_S * hs[j];
                 }
             }
             tc_fence_before();
@@ -526,7 +552,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 // most n_cap rows, and records for every assignment its padded row.
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, int32_t* pad_off,
-               int32_t* row_map, int32_t* src_token, int max_units, int ffn_grid) {
+               int32_t* row_map, int32_t* src_token, int max_units, int ffn_grid, int32_t* status) {
     __shared__ int s_total_rows, s_n_units;
     __shared__ int s_cost[1024];
     const int n_keys = D.E * D.K + D.n_shared;
@@ -558,11 +584,17 @@ tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, i
     for (int a = threadIdx.x; a < D.A; a += blockDim.x) {
         const int pos = R.inv_perm[a];
         const int e = R.topk_idx[a], kk = R.bit_idx[a];
-        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < 0 || pos >= D.A) { row_map[a] = 0; continue; }
+        // a supplied routing index out of range, or a position outside the group of (e, kk): the assignment is
+        // skipped (row -1 contributes nothing to the combine) and the call is flagged
         const int key = e * D.K + kk;
+        if (e < 0 || e >= D.E || kk < 0 || kk >= D.K || pos < R.group_off[key] || pos >= R.group_off[key + 1]) {
+            row_map[a] = -1;
+            if (status) atomicOr(status, D2MOE_DEV_BAD_INDEX);
+            continue;
+        }
         const int row = pad_off[key] + (pos - R.group_off[key]);
         row_map[a] = row;
-        if (row >= 0 && row < total_rows) src_token[row] = a / D.k;
+        src_token[row] = a / D.k;
     }
     for (int i = threadIdx.x; i < D.n_shared * D.T; i += blockDim.x) {
         const int s = i / D.T, t = i - s * D.T;
@@ -655,18 +687,56 @@ tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, i
     }
 }
 
-// xp16[row, :] = fp16(x[src_token[row], :]) for the real rows (padding rows are never consumed:
-// a D column depends only on its own token row).
+// xp16[row, :] = fp16(x[src_token[row], :] * 2^(4-e)) for the real rows, where 2^e is the power of two just
+// above the row's largest magnitude: every row enters the fp16 products with its largest element in
+// [8, 16), whatever its own magnitude (a token of magnitude 1e5 or 1e-6 loses nothing to the fp16
+// range).  row_scale[0][row] = 2^(e-4) undoes that in the gate/up epilogue; h = silu(g) * u grows like
+// the square of the row's magnitude, so it is stored as fp16(h * row_scale[1][row]) with
+// row_scale[1] = 2^-eh, eh = 2 (e - 4) (clamped to +-60), and the down projection's epilogue multiplies
+// by row_scale[2] = 2^eh.  A row that holds a NaN or an infinity becomes zeros (scale 0: its outputs
+// are zero) and the call is flagged.  Padding rows are never consumed: a D column depends only on its
+// own token row.
 __global__ void __launch_bounds__(128)
 tc_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ src_token,
-                 const int32_t* __restrict__ pad_off, int n_keys, __half* __restrict__ xp16) {
+                 const int32_t* __restrict__ pad_off, int n_keys, __half* __restrict__ xp16,
+                 float* __restrict__ row_scale, long long R_alloc, int32_t* status) {
+    __shared__ float s_red[4];
     const int total_rows = pad_off[n_keys];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int row = blockIdx.x; row < total_rows; row += gridDim.x) {
         const int t = src_token[row];
         if (t < 0) continue;
         // eight elements (16 bytes) per thread and step; d is a multiple of 128 on this path
         const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * d);
         uint4* dst = reinterpret_cast<uint4*>(xp16 + (size_t)row * d);
+        float amax = 0.0f;
+        int bad = 0;
+        for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+            const uint4 v = src[i];
+            const uint32_t* vi = reinterpret_cast<const uint32_t*>(&v);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vi[k]));
+                amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+                bad |= !(fabsf(f.x) < 3.0e38f) | !(fabsf(f.y) < 3.0e38f);
+            }
+        }
+        for (int off = 16; off; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+        bad = __syncthreads_or(bad);
+        if (lane == 0) s_red[warp] = amax;
+        __syncthreads();
+        amax = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+        __syncthreads();
+        int e = 4;
+        if (amax > 0.0f && !bad) frexpf(amax, &e);                   // amax = m 2^e, 0.5 <= m < 1
+        const float mult = bad ? 0.0f : exp2f((float)(4 - e));
+        if (threadIdx.x == 0) {
+            const int eh = max(-60, min(60, 2 * (e - 4)));
+            row_scale[row] = bad ? 0.0f : exp2f((float)(e - 4));
+            row_scale[R_alloc + row] = exp2f((float)-eh);
+            row_scale[2 * R_alloc + row] = exp2f((float)eh);
+            if (bad && status) atomicOr(status, D2MOE_DEV_NONFINITE);
+        }
         for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
             const uint4 v = src[i];
             uint4 o;
@@ -675,7 +745,7 @@ tc_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __re
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vi[k]));
-                const __half2 h = __floats2half2_rn(f.x, f.y);
+                const __half2 h = bad ? __floats2half2_rn(0.0f, 0.0f) : __floats2half2_rn(f.x * mult, f.y * mult);
                 oi[k] = *reinterpret_cast<const uint32_t*>(&h);
             }
             dst[i] = o;
@@ -742,8 +812,9 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms);
-    tc_gather_kernel<<<1184, 128, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16);
+    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms,
+                                      device_status);
+    tc_gather_kernel<<<1184, 128, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16, B.slot_f, pl.R_alloc, device_status);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps(&maps_x, B.xp16, pl.R_alloc, D.d) || !make_maps(&maps_h, B.h16, pl.R_alloc, D.F))
@@ -757,7 +828,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.n_split = mode == 0 ? 1 : pl.n_split;
         p.groups_per_split = mode == 0 ? p.L.n_groups : pl.groups_per_split;
         p.units = B.units; p.n_units = B.n_units; p.next_item = B.n_units + 1 + mode;
-        p.hbuf = B.h16; p.obuf = B.o32; p.R_alloc = pl.R_alloc; p.status = device_status;
+        p.hbuf = B.h16; p.obuf = B.o32; p.row_scale = B.slot_f; p.R_alloc = pl.R_alloc; p.status = device_status;
         const int b_bytes = NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
         const int epi_bytes = 2 * 128 * 9 * 4;            // per warpgroup: 128 rows x 8 exchanged values (+1 pad)

@@ -47,7 +47,8 @@ struct TcBuffers {
     float* h32;             // [R_alloc, F]   SwiGLU outputs, fp32
     float* xk_x;            // [d / g][R_alloc][2]   per group and slot: sum of the quantised x, kappa * sum
     float* xk_h;            // [F / g][R_alloc][2]
-    float* slot_f;          // [3][R_alloc]   kappa, scale of x, scale of h per slot
+    float* slot_f;          // [3][R_alloc]   decode kernel: kappa, scale of x, scale of h per slot; grouped GEMM: the three
+                            //                power-of-two factors of the per-row activation scaling
 };
 
 bool tc_path_supported(const d2moe_config* c);

@@ -53,6 +53,8 @@ def test_status_strings(lib):
     (lambda c: setattr(c, "renormalize", 2), 2),
     (lambda c: setattr(c, "kernel_path", 7), 2),
     (lambda c: setattr(c, "n_experts", 300), 2),
+    (lambda c: setattr(c, "d_ffn", 1 << 19), 2),       # beyond D2MOE_MAX_DIM: no launch could take it
+    (lambda c: setattr(c, "d_ffn", 1 << 18), 0),
 ])
 def test_check_config(lib, mutate, code):
     c = good()
@@ -104,6 +106,7 @@ def test_null_and_short_buffers_are_rejected_before_launch(lib):
     # forward: T == 0 is a no-op, negative T is a shape error, missing expert pointer is NULL
     assert L.d2moe_moe_forward(ctypes.byref(c), 0, None, None, None, None, None, None, None, 0, None) == 0
     assert L.d2moe_moe_forward(ctypes.byref(c), -1, None, None, None, None, None, None, None, 0, None) == 3
+    assert L.d2moe_moe_forward(ctypes.byref(c), (1 << 20) + 1, None, None, None, None, None, None, None, 0, None) == 3
     ptrs = (ctypes.c_void_p * 12)(*([4096] * 11 + [None]))
     rin = binding._RouteIn(4096, None, None, 4096)
     assert L.d2moe_moe_forward(ctypes.byref(c), 4, 4096, ptrs, ctypes.byref(rin), None, 4096, None, 4096,
@@ -114,3 +117,15 @@ def test_null_and_short_buffers_are_rejected_before_launch(lib):
     # stack layer: argument errors are found before the normalisation kernel would be launched
     assert L.d2moe_stack_layer(ctypes.byref(c), 4, 4096, 4096, ctypes.c_float(1e-5), ptrs, ctypes.byref(rin),
                                None, 4096, 16, None) == 5
+
+
+def test_static_scratch_routing_refuses_what_its_array_cannot_hold(lib):
+    # more assignments than the built-in scratch array holds: refused before any launch (the fake non-null
+    # pointers are never dereferenced); the key limit equals the most (expert, width) pairs a valid
+    # configuration can have (256 experts x 8 widths), so it can never be exceeded
+    args = [4096, 4096, None, None, 4096] + [4096] * 6 + [None, None]
+    c = good().c()
+    assert lib.d2moe_route_static_scratch(ctypes.byref(c), -1, *args) == 3
+    too_many_tokens = binding.STATIC_MAX_ASSIGNMENTS // c.top_k + 1
+    assert lib.d2moe_route_static_scratch(ctypes.byref(c), too_many_tokens, *args) == 5
+    assert binding.STATIC_MAX_KEYS == 256 * 8

@@ -71,3 +71,24 @@ def test_single_process_helpers():
     b = bench.algorithmic_bytes(wl, 64, group_off)
     assert b["active_experts"] == 1
     assert b["down"] == 14336 * 4096 // 4 + 4096 * 112 * 4 + 128 * 14336 * 2 + 128 * 4096 * 4
+
+
+def test_gpus_flag_starts_the_replicas_itself():
+    """`python bench.py --gpus 2` run as a plain script starts two ranks (torch.distributed.run, rendezvous on
+    127.0.0.1) and passes rank 0's line on; the self-check arm stands in for the layer call (gloo, made-up step
+    times 1 ms and 2 ms), so this runs without a GPU."""
+    import json
+    import subprocess
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.replica_command(2, ["--gpus", "2"], port=1234)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-2:] == ["--gpus", "2"]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "selfcheck"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["ms_per_step"] == 2.0 and d["value"] == pytest.approx(64 * 2 / 2.0e-3)

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2504_15299_b200 import synth
-from tests.helpers import OracleLayer, gpu_layer, max_norm_rel_err, np_f32
+from tests.helpers import OracleLayer, check_rows, gpu_layer, max_norm_rel_err, np_f32
 
 pytestmark = pytest.mark.gpu
 
@@ -198,10 +198,10 @@ def test_layer_tiny(B, path):
     assert len(errs) == 16 and max(errs.values()) < TOL, errs
 
 
-@pytest.mark.parametrize("path", [1, 2])
-def test_layer_finegrained_with_shared_experts_sampled_tokens(B, path):
+def test_layer_finegrained_with_shared_experts_sampled_tokens_cuda_core_path(B):
+    # (the tensor-core path is checked on all 256 tokens in test_gpu_parity_configs.py)
     wl = synth.WORKLOADS["finegrained"]
-    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 256, tokens=[0, 100, 255], kernel_path=path)
+    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 256, tokens=[0, 100, 255], kernel_path=1)
     assert max(errs.values()) < TOL, errs
 
 
@@ -237,14 +237,6 @@ def test_mixtral_decode_tensor_path_matches_cuda_core_path(B, mixtral_blobs, T):
     wl = synth.WORKLOADS["mixtral_decode"]
     err, _ = cross_check_paths(B, wl, T, mixtral_blobs)
     assert err < TOL, err
-
-
-def test_mixtral_decode_sampled_tokens_against_oracle(B, mixtral_blobs):
-    """Full-size decode layer in the benchmark's configuration (T = 64, tensor-core path): the oracle
-    recomputes one sampled token end to end (two experts, each regenerated and quantized on the CPU)."""
-    wl = synth.WORKLOADS["mixtral_decode"]
-    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 64, tokens=[37], kernel_path=0, blobs=mixtral_blobs)
-    assert max(errs.values()) < TOL, errs
 
 
 def test_layer_empty_batch_is_a_noop(B):
@@ -305,52 +297,6 @@ def test_mixtral_prefill_tensor_path_matches_cuda_core_path(B, mixtral_blobs):
     assert err < TOL, err
 
 
-def test_mixtral_prefill_sampled_token_against_oracle(B, mixtral_blobs):
-    wl = synth.WORKLOADS["mixtral_prefill"]
-    errs, _, _ = run_layer(B, B.Config.from_workload(wl), wl, 2048, tokens=[1234], kernel_path=0, blobs=mixtral_blobs)
-    assert max(errs.values()) < TOL, errs
-
-
-def test_stack_two_full_size_layers_teacher_forced(B):
-    """Two layers of the Mixtral-shaped stack (T = 16, learned bit widths): each layer is fed the oracle's
-    input (teacher forcing) and one sampled token of its output is recomputed by the oracle."""
-    _, routing, moe = oracle_mods()
-    wl = synth.WORKLOADS["mixtral_stack"]
-    cfg = B.Config.from_workload(wl)
-    T, tok = 16, 5
-    x_or = np_f32(synth.tokens_bf16(wl, T, "cpu", step=1)).astype(np.float64)
-    for layer in range(2):
-        blobs = gpu_layer(B, cfg, wl, layer=layer)
-        gw = synth.gate_weight_bf16(wl, "cuda", layer=layer)
-        bw = synth.bit_router_weight_bf16(wl, "cuda", layer=layer)
-        x_gpu = torch.from_numpy(x_or.astype(np.float32)).to("cuda", torch.bfloat16)
-        xn = torch.empty_like(x_gpu)
-        st = torch.zeros(1, dtype=torch.int32, device="cuda")
-        B.stack_layer(cfg, x_gpu, xn, blobs, gate_w=gw, bit_w=bw, device_status=st)
-        torch.cuda.synchronize()
-        assert int(st.item()) == 0
-        # oracle: same layer, sampled token
-        xn_or = moe.round_to_bf16(moe.rmsnorm(x_or)).astype(np.float64)
-        assert np.array_equal(np_f32(xn), xn_or.astype(np.float32))
-        rt = routing.route(xn_or.astype(np.float32), E=wl.n_experts, K=len(wl.bits), top_k=wl.top_k,
-                           renormalize=True, gate_w=np_f32(gw), bit_w=np_f32(bw))
-        r_gpu = B.route(cfg, xn, gate_w=gw, bit_w=bw)
-        torch.cuda.synchronize()
-        assert np.array_equal(r_gpu.topk_idx.cpu().numpy(), rt.topk_idx)
-        assert np.array_equal(r_gpu.bit_idx.cpu().numpy(), rt.bit_idx)
-        ol = OracleLayer(wl, layer=layer)
-        y_tok = moe.moe_layer(xn_or, rt, ol, wl.bits, wl.n_experts, tokens=[tok])[tok]
-        ref_row = moe.round_to_bf16(x_or[tok] + y_tok).astype(np.float64)
-        assert max_norm_rel_err(np_f32(x_gpu)[tok], ref_row) < TOL
-        # teacher forcing: the next layer starts from the GPU output only where the oracle has no value;
-        # the sampled row comes from the oracle, the rest is what the GPU produced (already checked above
-        # to route identically)
-        x_next = np_f32(x_gpu).astype(np.float64)
-        x_next[tok] = ref_row
-        x_or = x_next
-        del blobs
-
-
 # ------------------------------------------------------------------ other width lists, group sizes, loads
 def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=21, one_expert=False,
                      token_scales=None, outlier=None):
@@ -386,7 +332,7 @@ def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     a, b = y_cc.float(), y_tc.float()
-    cross = float(((a - b).abs().amax(dim=1) / a.abs().amax(dim=1)).max().item())
+    cross = float(((a - b).abs().amax(dim=1) / a.abs().amax(dim=1).clamp_min(1e-30)).max().item())
     rt = routing.route(np_f32(x), E=E, K=K, top_k=k, renormalize=True, logits=np_f32(logits),
                        forced_bit_idx=fb.cpu().numpy())
     packed = {}
@@ -401,12 +347,10 @@ def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=
     if token_scales is not None:
         toks = list(range(T))
         ref = moe.moe_layer(np_f32(x), rt, get, bits, E, n_shared, tokens=toks)
-    err = 0.0
-    for t in toks:
-        if np.abs(ref[t]).max() == 0.0:            # an all-zero token must come out as exact zeros
-            assert np.abs(np_f32(y_tc)[t]).max() == 0.0
-        else:
-            err = max(err, max_norm_rel_err(np_f32(y_tc)[t], ref[t]))
+    # both metrics: max-norm relative error per token, and the element-wise bound |dy| <= 1e-2 |y| + 1e-2 rms(y)
+    # (an all-zero token must come out as exact zeros)
+    err, excess = check_rows(np_f32(y_tc), {t: ref[t] for t in toks}, TOL)
+    assert excess <= 1.0, excess
     return cross, err
 
 
@@ -533,3 +477,83 @@ def test_a_wait_that_nothing_satisfies_expires_and_leaves_the_device_usable(B, w
     # the context is intact: a normal layer call still passes
     cross, err = small_layer_case(B, d=128, F=128, E=2, k=1, g=64, bits=(2, 4, 8), T=4)
     assert cross < TOL and err < TOL, (cross, err)
+
+
+# ------------------------------------------------------------------ numeric range of the two expert kernels
+def test_decode_kernel_outliers_of_1e3_and_1e4(B):
+    # One element 10^3 / 10^4 times the rest of its token.  The decode kernel quantises a row to 15 bits against
+    # its largest element; the noise this adds to an output is at most sqrt(n) / (16191 sqrt(12)) of the
+    # output's rms (1.1e-3 at n = 4096, 2.1e-3 at n = 14336), because the outlier that sets the step also
+    # carries the row's norm.  Both metrics must hold for every token.
+    T = 8
+    scales = [1.0] * T
+    for outlier in [(1, 5, 1.0e3), (2, 700, 1.0e4), (3, 1023, -3.0e4)]:
+        cross, err = small_layer_case(B, d=1024, F=1024, E=2, k=2, g=128, bits=(2, 3, 4, 8), T=T, token_scales=scales,
+                                      outlier=outlier)
+        assert err < TOL and cross < TOL, (outlier, cross, err)
+
+
+def test_grouped_gemm_per_token_activation_scaling(B):
+    # the grouped dequant-GEMM runs on fp16 tiles: every token row is scaled by a power of two of its own, so
+    # tokens of magnitude 1e5 (beyond fp16), 1e-6 (below fp16's subnormals), an outlier of 1e4 and an all-zero
+    # token in one prefill-sized batch all come out within tolerance, with no flag
+    T = 400
+    scales = [1.0] * T
+    scales[3], scales[10], scales[50], scales[77], scales[200], scales[399] = 1.0e5, 1.0e-6, 0.0, 3.0e4, 2.0 ** -12, 7.0e8
+    cross, err = small_layer_case(B, d=256, F=256, E=2, k=1, g=128, bits=(2, 3, 4, 8), T=T, probs=[0.1, 0.2, 0.4, 0.3],
+                                  token_scales=scales, outlier=(5, 17, 1.0e4))
+    assert err < TOL and cross < TOL, (cross, err)
+
+
+def test_grouped_gemm_flags_nonfinite_activations(B):
+    # a NaN / an infinity in a token at prefill size: flagged, that token's output is zero, the others are untouched
+    d, F, E, k, g, bits, T = 256, 256, 2, 1, 128, (2, 4, 8), 300
+    cfg = B.Config(d, F, E, k, g, bits)
+    blobs = [B.pack_mwq(cfg, synth.normal(32, 100 + i, (F, d) if i % 3 < 2 else (d, F), 0.02, "cuda"))
+             for i in range(3 * E)]
+    x = synth.bf16_exact(synth.normal(32, 1, (T, d), 1.0, "cuda"))
+    logits = synth.normal(32, 5, (T, E), 1.0, "cuda")
+    fb = synth.categorical(32, 4, (T, k), [0.3, 0.3, 0.4], "cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_clean = B.moe_forward(cfg, x, blobs, logits=logits, forced_bit_idx=fb, device_status=st).clone()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    x_bad = x.clone()
+    x_bad[7, 5] = float("nan")
+    x_bad[150, 9] = float("-inf")
+    y_bad = B.moe_forward(cfg, x_bad, blobs, logits=logits, forced_bit_idx=fb, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & B.DEV_NONFINITE
+    keep = [t for t in range(T) if t not in (7, 150)]
+    assert torch.equal(y_bad[keep], y_clean[keep])
+    assert float(y_bad[[7, 150]].float().abs().max().item()) == 0.0
+
+
+@pytest.mark.parametrize("T", [12, 300])
+def test_bad_index_in_supplied_routing_is_flagged_and_skipped(B, T):
+    # caller-supplied routing (`pre`) with one expert index and one width index out of range, on the tensor-core
+    # kernels at decode size and at prefill size: the call is flagged and the two assignments contribute
+    # nothing, exactly as if their gate weights were zero
+    d, F, E, k, g, bits = 256, 256, 2, 2, 128, (2, 4, 8)
+    cfg = B.Config(d, F, E, k, g, bits, kernel_path=2)
+    blobs = [B.pack_mwq(cfg, synth.normal(33, 100 + i, (F, d) if i % 3 < 2 else (d, F), 0.02, "cuda"))
+             for i in range(3 * E)]
+    x = synth.bf16_exact(synth.normal(33, 1, (T, d), 1.0, "cuda"))
+    logits = synth.normal(33, 5, (T, E), 1.0, "cuda")
+    fb = synth.categorical(33, 4, (T, k), [0.3, 0.3, 0.4], "cuda")
+    pre = B.route(cfg, x, logits=logits, forced_bit_idx=fb)
+    torch.cuda.synchronize()
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # reference: the same routing with the two assignments' weights set to zero
+    ref = B.route(cfg, x, logits=logits, forced_bit_idx=fb)
+    ref.topk_w[2, 1] = 0.0
+    ref.topk_w[T - 1, 0] = 0.0
+    y_ref = B.moe_forward(cfg, x, blobs, pre=ref, device_status=st).clone()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    pre.topk_idx[2, 1] = E + 5
+    pre.bit_idx[T - 1, 0] = 9
+    y = B.moe_forward(cfg, x, blobs, pre=pre, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & B.DEV_BAD_INDEX
+    assert torch.equal(y, y_ref)

@@ -144,3 +144,45 @@ def test_stack_layer_residual():
     assert np.array_equal(out, x)
     out2 = moe.stack_layer(x, lambda xn: xn)
     assert np.array_equal(out2, moe.round_to_bf16(x + moe.round_to_bf16(moe.rmsnorm(x)).astype(np.float64)))
+
+
+def test_oracle_sampled_helper_matches_a_direct_layer_call():
+    """The test plumbing that cuts a full-size layer by expert (tests/helpers.oracle_sampled) returns
+    what one moe_layer call on the whole batch returns, for two batches sharing the weights, with a
+    shared expert, on token subsets and with one or several threads."""
+    from paper_2504_15299_b200 import synth
+    from tests.helpers import OracleLayer, group_edge_tokens, oracle_sampled
+    wl = synth.Workload("t", 64, 128, 4, 2, 32, (2, 3, 4, 8), (0.1, 0.2, 0.4, 0.3), seed=9, n_shared=1)
+    K = len(wl.bits)
+    jobs = []
+    for T, tid in ((7, 11), (19, 12)):
+        x = synth.bf16_exact(synth.normal(9, tid, (T, wl.d_model), 1.0)).float().numpy()
+        logits = synth.normal(9, tid + 10, (T, wl.n_experts), 1.0).numpy()
+        fb = synth.categorical(9, tid + 20, (T, wl.top_k), wl.bit_probs).numpy()
+        rt = routing.route(x, E=wl.n_experts, K=K, top_k=wl.top_k, renormalize=True, logits=logits, forced_bit_idx=fb)
+        jobs.append((x, rt, group_edge_tokens(rt, wl.top_k, extra=2)))
+    ol = OracleLayer(wl)
+    for n_threads in (1, 3):
+        got = oracle_sampled(wl, jobs, n_threads=n_threads)
+        for (x, rt, toks), res in zip(jobs, got):
+            ref = moe.moe_layer(x, rt, ol, wl.bits, wl.n_experts, wl.n_shared, tokens=toks)
+            assert set(res) == set(ref) == set(toks)
+            for t in toks:
+                assert np.allclose(res[t], ref[t], rtol=1e-12, atol=1e-15)
+    # the edge sample touches the first and the last member of every non-empty group
+    x, rt, toks = jobs[1]
+    gr = rt.grouping
+    for key in range(wl.n_experts * K):
+        a0, a1 = gr.group_off[key], gr.group_off[key + 1]
+        if a1 > a0:
+            assert gr.perm[a0] // wl.top_k in toks and gr.perm[a1 - 1] // wl.top_k in toks
+
+
+def test_elementwise_metric_sees_small_elements():
+    from tests.helpers import elementwise_excess, max_norm_rel_err
+    ref = np.array([100.0, 1.0, -1.0, 0.5])
+    bad = ref.copy()
+    bad[3] += 0.6                                  # 0.6 % of the row maximum: invisible to the max-norm metric
+    assert max_norm_rel_err(bad, ref) < 1e-2
+    assert elementwise_excess(bad, ref) > 1.0
+    assert elementwise_excess(ref * (1 + 2.0 ** -9), ref) < 1.0    # bf16 rounding passes
