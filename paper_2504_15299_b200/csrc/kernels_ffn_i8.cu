@@ -502,43 +502,59 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
 #pragma unroll
                 for (int s = 0; s < 4; ++s) acc[i][s] = 0.0f;
 
-            // fold group g (accumulator buffer g & 1) into acc; fbs / fbph: ring position and phase of its sums,
-            // sub: group inside the stage, rel: last group of the stage (the stage is released afterwards)
-            auto fold = [&](uint32_t g, uint32_t fbs, uint32_t fbph, int sub, bool rel, uint32_t meta) {
+            // Fold of group g (accumulator buffer g & 1) into acc, in two steps so that the tensor-memory loads are
+            // in flight while the warp does other work: fold_prefetch waits for the group's products and issues
+            // the loads of the first two blocks (it runs between the two segments the warp unpacks for the next
+            // group); fold_compute issues the loads of the other two blocks, folds the first two while those
+            // are in flight, then the rest.  fbs / fbph: ring position and phase of the group's activation sums,
+            // sub: group inside the stage, rel: last group of the stage (the stage is released afterwards).
+            uint32_t fv0[2][8], fv1[2][8];
+            auto fold_prefetch = [&](uint32_t g) {
                 const int buf = g & 1;
                 mbar_wait_blk(D_FULL(buf), (g >> 1) & 1);
                 tc_fence_after();
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    if (i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(i), fv0[i]);
+            };
+            auto fold_compute = [&](uint32_t g, uint32_t fbs, uint32_t fbph, int sub, bool rel, uint32_t meta) {
+                const int buf = g & 1;
                 const __half2 mh = as_h2(meta);
                 const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
                 const float lo = __high2float(mh);
                 mbar_wait_blk(B_FULL(fbs), fbph);
                 const uint32_t xk_addr = xkbuf + (fbs * 2 + sub) * I8_XK_BYTES;
-                // two rounds of two blocks: 16 accumulator registers in flight instead of 32
+                auto fold_block = [&](int b, const uint32_t (&v)[8]) {
+                    float xk[8];
+                    const uint32_t a = xk_addr + 32u * MYBLK(b);
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
+                    // the four slots of a block have one width: s1' kappa + lo once per block
+                    const float cx = fmaf(s1p, xk[1], lo);
 #pragma unroll
-                for (int rd = 0; rd < 2; ++rd) {
-                    uint32_t v[2][8];
+                    for (int s = 0; s < 4; ++s) {
+                        const int di = (int)v[2 * s] * 128 + (int)v[2 * s + 1];
+                        acc[b][s] = fmaf(s1p, (float)di, acc[b][s]);
+                        acc[b][s] = fmaf(cx, xk[2 * s], acc[b][s]);
+                    }
+                };
+                tc_wait_ld();                                  // the first two blocks have landed
+                if (n_mine > 2) {
 #pragma unroll
                     for (int i = 0; i < 2; ++i)
-                        if (2 * rd + i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(2 * rd + i), v[i]);
+                        if (2 + i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(2 + i), fv1[i]);
+                } else {
+                    tc_fence_before();
+                    mbar_arrive(D_EMPTY(buf));                 // nothing more to read from this buffer
+                }
+                if (0 < n_mine) fold_block(0, fv0[0]);
+                if (1 < n_mine) fold_block(1, fv0[1]);
+                if (n_mine > 2) {
                     tc_wait_ld();
-                    if (rd == 1) { tc_fence_before(); mbar_arrive(D_EMPTY(buf)); }
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        if (2 * rd + i < n_mine) {
-                            float xk[8];
-                            const uint32_t a = xk_addr + 32u * MYBLK(2 * rd + i);
-                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
-                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
-                            // the four slots of a block have one width: s1' kappa + lo once per block
-                            const float cx = fmaf(s1p, xk[1], lo);
-#pragma unroll
-                            for (int s = 0; s < 4; ++s) {
-                                const int di = (int)v[i][2 * s] * 128 + (int)v[i][2 * s + 1];
-                                acc[2 * rd + i][s] = fmaf(s1p, (float)di, acc[2 * rd + i][s]);
-                                acc[2 * rd + i][s] = fmaf(cx, xk[2 * s], acc[2 * rd + i][s]);
-                            }
-                        }
-                    }
+                    tc_fence_before();
+                    mbar_arrive(D_EMPTY(buf));
+                    fold_block(2, fv1[0]);
+                    if (3 < n_mine) fold_block(3, fv1[1]);
                 }
                 if (rel) {
                     __syncwarp();
@@ -584,11 +600,15 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 handoff_begin();
                                 do_seg(std::integral_constant<int, 0>{});
                                 do_seg(std::integral_constant<int, 1>{});
+                                if (pend) fold_prefetch(gc - 1);     // in flight during the second segment
                                 do_seg(std::integral_constant<int, 2>{});
                                 do_seg(std::integral_constant<int, 3>{});
                                 handoff_end();
+                            } else if (pend) {
+                                fold_prefetch(gc - 1);
                             }
                         } else {
+                            if (wg > kmax && pend) fold_prefetch(gc - 1);
 #pragma unroll 1
                             for (int j = wg; j <= kmax; j += 4) {
                                 handoff_begin();
@@ -596,10 +616,11 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 if (j + 2 <= kmax)
                                     unpack_dispatch<GS>(p.L.seg_sw[j + 2], wb + (uint32_t)p.L.seg_off[j + 2], rr, p.L.seg_w[j + 2],
                                                         p.L.seg_shift[j + 2], a_base + 32);
+                                if (pend && j + 4 > kmax) fold_prefetch(gc - 1);       // before the last hand-off of the group
                                 handoff_end();
                             }
                         }
-                        if (pend) fold(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
+                        if (pend) fold_compute(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
                         pend = true;
                         pend_meta = meta;
                         pend_bs = bs; pend_bph = bph; pend_sub = sub; pend_rel = sub == ng - 1;
@@ -611,7 +632,10 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
                 if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
             }
-            if (pend) fold(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
+            if (pend) {
+                fold_prefetch(gc - 1);
+                fold_compute(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
+            }
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
             float out[4][4];                   // a copy: acc itself must stay in registers
