@@ -6,7 +6,7 @@ calibration data exists here; with X proportional to the identity the Hessian fa
 and the compensation update is zero, so what is left is Eq. 2 followed by the one-bit residual
 steps of Eq. 4, which is what this file writes out.
 
-Readings taken where the paper is silent (each also listed in the design notes):
+Readings taken where the paper is silent:
 * ``round`` in Eq. 2 is round-half-to-even; the base code is clamped to [0, 2^b1 - 1].
 * Zero point is real-valued (Eq. 2 has z in R); it is stored as ``lo = -z*s``, an fp16 value rounded
   toward -inf from the group minimum, and the scale ``s1`` is the fp16 value rounded toward +inf

@@ -885,7 +885,7 @@ i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, c
 }
 
 // tensor maps over a row-major byte matrix [rows, cols], 128-byte swizzle, boxes of 128 columns x 16/32/64 rows
-static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long long cols) {
+static inline bool make_maps_u8_uncached(TmaMaps* maps, void* base, long long rows, long long cols) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     for (int i = 0; i < 3; ++i) {
@@ -900,6 +900,9 @@ static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long 
     }
     maps->m[3] = maps->m[2]; maps->m[4] = maps->m[2];
     return true;
+}
+static inline bool make_maps_u8(TmaMaps* maps, void* base, long long rows, long long cols) {
+    return cached_maps(maps, 1, base, rows, cols, [&](TmaMaps* m) { return make_maps_u8_uncached(m, base, rows, cols); });
 }
 
 // One block waits on a barrier that nothing completes, with either of the two bounded waits of the
@@ -950,10 +953,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     int8_t* qh = reinterpret_cast<int8_t*>(B.h16);
     const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
 
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int ffn_grid = 2 * sms;
+    const int ffn_grid = 2 * device_sm_count();
     const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
     i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
                                       pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status);
@@ -998,18 +998,21 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         int wpack = 0;
         if (p.L.n_seg <= 4)
             for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
-        auto launch = [&](auto kern) -> cudaError_t {
-            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        auto launch = [&](auto kc) -> cudaError_t {
+            constexpr auto kern = decltype(kc)::value;
+            cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
             if (err != cudaSuccess) return err;
             kern<<<ffn_grid, I8_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
+#define I8_KERNEL(GS_, WP_) std::integral_constant<decltype(&ffn_i8_kernel<GS_, WP_>), &ffn_i8_kernel<GS_, WP_>>{}
         cudaError_t e;
-        if (D.g == 128 && wpack == 0x4112) e = launch(ffn_i8_kernel<128, 0x4112>);        // {2,3,4,8}
-        else if (D.g == 128 && wpack == 0x422) e = launch(ffn_i8_kernel<128, 0x422>);     // {2,4,8}
-        else if (D.g == 128 && wpack == 0x1115) e = launch(ffn_i8_kernel<128, 0x1115>);   // {5,6,7,8}
-        else if (D.g == 128) e = launch(ffn_i8_kernel<128, 0>);
-        else e = launch(ffn_i8_kernel<64, 0>);
+        if (D.g == 128 && wpack == 0x4112) e = launch(I8_KERNEL(128, 0x4112));        // {2,3,4,8}
+        else if (D.g == 128 && wpack == 0x422) e = launch(I8_KERNEL(128, 0x422));     // {2,4,8}
+        else if (D.g == 128 && wpack == 0x1115) e = launch(I8_KERNEL(128, 0x1115));   // {5,6,7,8}
+        else if (D.g == 128) e = launch(I8_KERNEL(128, 0));
+        else e = launch(I8_KERNEL(64, 0));
+#undef I8_KERNEL
         if (e != cudaSuccess) return e;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;

@@ -809,9 +809,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
                               const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
     auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
     const int n_keys = D.E * D.K + D.n_shared;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = device_sm_count();
     tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms,
                                       device_status);
     tc_gather_kernel<<<1184, 128, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16, B.slot_f, pl.R_alloc, device_status);
@@ -847,17 +845,20 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         int wpack = 0;
         if (p.L.n_seg <= 4)
             for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
-        auto launch = [&](auto kern) -> cudaError_t {
-            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        auto launch = [&](auto kc) -> cudaError_t {
+            constexpr auto kern = decltype(kc)::value;
+            cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
             if (err != cudaSuccess) return err;
             kern<<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
+#define TC_KERNEL(GS_, WP_) std::integral_constant<decltype(&ffn_tc_kernel<GS_, WP_>), &ffn_tc_kernel<GS_, WP_>>{}
         cudaError_t e;
-        if (D.g == 128 && wpack == 0x4112) e = launch(ffn_tc_kernel<128, 0x4112>);        // {2,3,4,8}
-        else if (D.g == 128 && wpack == 0x422) e = launch(ffn_tc_kernel<128, 0x422>);     // {2,4,8}
-        else if (D.g == 128) e = launch(ffn_tc_kernel<128, 0>);
-        else e = launch(ffn_tc_kernel<64, 0>);
+        if (D.g == 128 && wpack == 0x4112) e = launch(TC_KERNEL(128, 0x4112));        // {2,3,4,8}
+        else if (D.g == 128 && wpack == 0x422) e = launch(TC_KERNEL(128, 0x422));     // {2,4,8}
+        else if (D.g == 128) e = launch(TC_KERNEL(128, 0));
+        else e = launch(TC_KERNEL(64, 0));
+#undef TC_KERNEL
         if (e != cudaSuccess) return e;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;

@@ -1,6 +1,7 @@
 // Dual routing (expert gate top-k + per-expert bit-width choice, Section 3.2) and the stable
 // grouping of assignments by (expert, width); its histogram is B_{j,k} of Section 3.4.3.
 #include "d2moe_common.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -16,6 +17,58 @@ __device__ __forceinline__ float dot_pinned(const __nv_bfloat16* __restrict__ a,
         acc = fmaf(__bfloat162float(a[i]), __bfloat162float(b[i]), acc);
     for (int off = 16; off; off >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, off);
     return acc;
+}
+
+// One warp: the gate of one token from its logits (lane l holds the logits of experts l, l + 32, ...).
+// k rounds of arg-max over the remaining logits, ties to the lower index (shuffle reduction); softmax over
+// all experts, gathered at the selected ones.  Outputs in every lane: sel[s], w[s] (not renormalised) and
+// their sum; a NaN or an infinity among the logits raises D2MOE_DEV_NONFINITE.
+__device__ __forceinline__ void gate_select(const float (&lg)[MAX_E_PER_LANE], int E, int k, int lane,
+                                            int (&sel)[MAX_TOPK], float (&w)[MAX_TOPK], float& wsum,
+                                            int32_t* __restrict__ device_status) {
+    bool bad = false;
+#pragma unroll
+    for (int m = 0; m < MAX_E_PER_LANE; ++m)
+        if (lane + 32 * m < E && !isfinite(lg[m])) bad = true;
+    if (__any_sync(0xffffffffu, bad) && lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_NONFINITE);
+
+    unsigned taken = 0;
+    float selv[MAX_TOPK];
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s) {
+        sel[s] = 0; selv[s] = 0.0f;
+        if (s < k) {
+            float bv = -INFINITY; int bi = 0x7fffffff;
+#pragma unroll
+            for (int m = 0; m < MAX_E_PER_LANE; ++m) {
+                const int e = lane + 32 * m;
+                if (e < E && !((taken >> m) & 1u)) {
+                    if (bi == 0x7fffffff || lg[m] > bv) { bv = lg[m]; bi = e; }
+                }
+            }
+            for (int off = 16; off; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                const bool take = (oi != 0x7fffffff) &&
+                                  (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
+                if (take) { bv = ov; bi = oi; }
+            }
+            sel[s] = bi; selv[s] = bv;
+            if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+        }
+    }
+    const float mx = selv[0];
+    float part = 0.0f;
+#pragma unroll
+    for (int m = 0; m < MAX_E_PER_LANE; ++m)
+        if (lane + 32 * m < E) part += expf(lg[m] - mx);
+    for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    wsum = 0.0f;
+#pragma unroll
+    for (int s = 0; s < MAX_TOPK; ++s) {
+        w[s] = 0.0f;
+        if (s < k) { w[s] = expf(selv[s] - mx) / part; wsum += w[s]; }
+    }
 }
 
 // One warp per token.
@@ -47,54 +100,10 @@ route_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16
                 if (m == (e >> 5) && lane == (e & 31)) lg[m] = v;
         }
     }
-    bool bad = false;
-#pragma unroll
-    for (int m = 0; m < MAX_E_PER_LANE; ++m)
-        if (lane + 32 * m < E && !isfinite(lg[m])) bad = true;
-    if (__any_sync(0xffffffffu, bad) && lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_NONFINITE);
-
-    // k rounds of arg-max over the remaining logits, ties to the lower index
-    unsigned taken = 0;
     int sel[MAX_TOPK];
-    float selv[MAX_TOPK];
-#pragma unroll
-    for (int s = 0; s < MAX_TOPK; ++s) {
-        sel[s] = 0; selv[s] = 0.0f;
-        if (s < D.k) {
-            float bv = -INFINITY; int bi = 0x7fffffff;
-#pragma unroll
-            for (int m = 0; m < MAX_E_PER_LANE; ++m) {
-                const int e = lane + 32 * m;
-                if (e < E && !((taken >> m) & 1u)) {
-                    if (bi == 0x7fffffff || lg[m] > bv) { bv = lg[m]; bi = e; }
-                }
-            }
-            for (int off = 16; off; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                const bool take = (oi != 0x7fffffff) &&
-                                  (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
-                if (take) { bv = ov; bi = oi; }
-            }
-            sel[s] = bi; selv[s] = bv;
-            if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
-        }
-    }
-
-    // softmax over all experts, gathered at the selected ones
-    const float mx = selv[0];
-    float part = 0.0f;
-#pragma unroll
-    for (int m = 0; m < MAX_E_PER_LANE; ++m)
-        if (lane + 32 * m < E) part += expf(lg[m] - mx);
-    for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
     float w[MAX_TOPK];
-    float wsum = 0.0f;
-#pragma unroll
-    for (int s = 0; s < MAX_TOPK; ++s) {
-        w[s] = 0.0f;
-        if (s < D.k) { w[s] = expf(selv[s] - mx) / part; wsum += w[s]; }
-    }
+    float wsum;
+    gate_select(lg, E, D.k, lane, sel, w, wsum, device_status);
 
     // bit-width choice per selected expert
 #pragma unroll
@@ -180,65 +189,13 @@ __global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ ke
     }
 }
 
-// Decode-sized loads: the three steps above in one block, keys staged in shared memory (same
-// warp-per-key ballot walks, so the result is the same stable order).  smem: A keys + n_keys + 1 ints.
+// Small and mid-sized loads: histogram, scan and scatter in one launch.  Every block stages all keys in shared
+// memory and counts every key itself (32 warps, a key per warp at a time), so no block waits for another;
+// block b then writes the groups of the keys b, b + grid, ...  One block for decode-sized loads, a few
+// blocks for a prefill batch of a few thousand assignments on a few dozen keys.  Same warp-per-key ballot
+// walks as the three kernels above: the same stable order.  smem: A keys + n_keys + 1 ints.
 __global__ void __launch_bounds__(1024)
-group_small_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
-                   int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
-    extern __shared__ int32_t s_grp[];
-    int32_t* s_keys = s_grp;
-    int32_t* s_off = s_grp + ((A + 31) & ~31);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int a = threadIdx.x; a < A; a += blockDim.x) s_keys[a] = keys[a];
-    __syncthreads();
-    for (int key = warp; key < n_keys; key += n_warps) {
-        int cnt = 0;
-        for (int base = 0; base < A; base += 32) {
-            const int a = base + lane;
-            cnt += __popc(__ballot_sync(0xffffffffu, a < A && s_keys[a] == key));
-        }
-        if (lane == 0) s_off[key] = cnt;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        int carry = 0;
-        for (int base = 0; base < n_keys; base += 32) {
-            const int i = base + lane;
-            const int v = i < n_keys ? s_off[i] : 0;
-            int incl = v;
-            for (int off = 1; off < 32; off <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += o;
-            }
-            if (i < n_keys) { s_off[i] = carry + incl - v; group_off[i] = carry + incl - v; }
-            carry += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (lane == 0) { s_off[n_keys] = carry; group_off[n_keys] = carry; }
-    }
-    __syncthreads();
-    for (int key = warp; key < n_keys; key += n_warps) {
-        int pos = s_off[key];
-        if (pos == s_off[key + 1]) continue;
-        for (int base = 0; base < A; base += 32) {
-            const int a = base + lane;
-            const bool m = a < A && s_keys[a] == key;
-            const unsigned bal = __ballot_sync(0xffffffffu, m);
-            if (m) {
-                const int p = pos + __popc(bal & ((1u << lane) - 1u));
-                perm[p] = a;
-                inv_perm[a] = p;
-            }
-            pos += __popc(bal);
-        }
-    }
-}
-
-// Mid-sized loads (a prefill batch of a few thousand assignments on a few dozen keys): one launch of a few
-// blocks.  Every block stages all keys in shared memory and counts every key itself (32 warps, a key per
-// warp at a time), so no block waits for another; block b then writes the groups of the keys b, b + grid,
-// ...  Same warp-per-key ballot walks as above: the same stable order.  smem: A keys + n_keys + 1 ints.
-__global__ void __launch_bounds__(1024)
-group_mid_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
+group_block_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
                  int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
     extern __shared__ int32_t s_grp[];
     int32_t* s_keys = s_grp;
@@ -373,49 +330,16 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
     int sel[MAX_TOPK];
     if (warp == 0) {
         float lg[MAX_E_PER_LANE];
-        bool bad = false;
 #pragma unroll
         for (int m = 0; m < MAX_E_PER_LANE; ++m) {
             const int e = lane + 32 * m;
             lg[m] = e < E ? lg_s[e] : -INFINITY;
-            if (e < E && !isfinite(lg[m])) bad = true;
         }
-        if (__any_sync(0xffffffffu, bad) && lane == 0 && device_status) atomicOr(device_status, D2MOE_DEV_NONFINITE);
-        unsigned taken = 0;
-        float selv[MAX_TOPK];
+        gate_select(lg, E, D.k, lane, sel, w, wsum, device_status);
+        if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < MAX_TOPK; ++s) {
-            sel[s] = 0; selv[s] = 0.0f;
-            if (s < D.k) {
-                float bv = -INFINITY; int bi = 0x7fffffff;
-#pragma unroll
-                for (int m = 0; m < MAX_E_PER_LANE; ++m) {
-                    const int e = lane + 32 * m;
-                    if (e < E && !((taken >> m) & 1u)) {
-                        if (bi == 0x7fffffff || lg[m] > bv) { bv = lg[m]; bi = e; }
-                    }
-                }
-                for (int off = 16; off; off >>= 1) {
-                    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                    const bool take = (oi != 0x7fffffff) && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
-                    if (take) { bv = ov; bi = oi; }
-                }
-                sel[s] = bi; selv[s] = bv;
-                if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
-                if (lane == 0) sel_s[s] = bi;
-            }
-        }
-        const float mx = selv[0];
-        float part = 0.0f;
-#pragma unroll
-        for (int m = 0; m < MAX_E_PER_LANE; ++m)
-            if (lane + 32 * m < E) part += expf(lg[m] - mx);
-        for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-#pragma unroll
-        for (int s = 0; s < MAX_TOPK; ++s) {
-            w[s] = 0.0f;
-            if (s < D.k) { w[s] = expf(selv[s] - mx) / part; wsum += w[s]; }
+            for (int s = 0; s < MAX_TOPK; ++s)
+                if (s < D.k) sel_s[s] = sel[s];
         }
     }
     __syncthreads();
@@ -482,7 +406,7 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
         if (!logits_in && D.E > 16 && logits_ws && 16 * row_bytes <= budget) {
             const int TB = 8, EBL = 8;
             const size_t lsm = (size_t)(TB + EBL) * row_bytes;
-            cudaError_t e = cudaFuncSetAttribute(gate_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsm);
+            cudaError_t e = ensure_dynamic_smem<&gate_logits_kernel>((int)lsm);
             if (e != cudaSuccess) return e;
             dim3 grid((D.T + TB - 1) / TB, (D.E + EBL - 1) / EBL);
             gate_logits_kernel<<<grid, 256, lsm, st>>>(D.T, D.E, D.d, x, gate_w, logits_ws, TB, EBL);
@@ -490,7 +414,7 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
             gate_w = nullptr;
         }
         const size_t smem = row_bytes * (1 + EB) + tail_bytes;
-        cudaError_t e = cudaFuncSetAttribute(route_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = ensure_dynamic_smem<&route_block_kernel>((int)smem);
         if (e != cudaSuccess) return e;
         // logits and widths both supplied: no dot products, one warp per token does the selection
         const int threads = (logits_in && forced) ? 32 : 256;
@@ -501,17 +425,13 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     // few assignments and keys: histogram, scan and scatter in one single-block launch (beyond about a
     // thousand warp walks the three grid-wide kernels are faster: 39 vs 10 us at 192 keys x 1536 assignments)
     const long long walks = (long long)n_keys * ((D.A + 31) / 32);
-    if (D.A <= 8192 && n_keys <= 2048 && walks <= 1024) {
+    const bool small = D.A <= 8192 && n_keys <= 2048 && walks <= 1024;
+    if (small || d2moe_group_is_mid(D.A, n_keys)) {
         const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
-        group_small_kernel<<<1, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
-        return cudaGetLastError();
-    }
-    if (d2moe_group_is_mid(D.A, n_keys)) {
-        const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
-        cudaError_t e = cudaFuncSetAttribute(group_mid_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsm);
+        cudaError_t e = ensure_dynamic_smem<&group_block_kernel>((int)gsm);
         if (e != cudaSuccess) return e;
-        const int blocks = n_keys < 16 ? n_keys : 16;
-        group_mid_kernel<<<blocks, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+        const int blocks = small ? 1 : (n_keys < 16 ? n_keys : 16);
+        group_block_kernel<<<blocks, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
         return cudaGetLastError();
     }
     count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);

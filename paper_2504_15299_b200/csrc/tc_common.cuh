@@ -243,7 +243,57 @@ static inline EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-static inline bool make_maps(TmaMaps* maps, void* base, long long rows, long long cols) {
+// ------------------------------------------------------------------------------------------------
+// Host: per-process caches, so that a layer call does not repeat driver queries whose answer cannot change
+// ------------------------------------------------------------------------------------------------
+// number of SMs of the current device
+static inline int device_sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int sms = 148;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cached[dev] = sms;
+    }
+    return cached[dev];
+}
+
+// raises the dynamic shared-memory limit of kernel Kern on the current device when a launch needs more than
+// any earlier one did (the attribute is per device and sticks)
+template <auto Kern>
+static inline cudaError_t ensure_dynamic_smem(int bytes) {
+    static int set[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (set[dev] >= bytes) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) set[dev] = bytes;
+    return e;
+}
+
+// the tensor maps of the last few (buffer, shape) pairs this thread built: a serving loop calls with the same
+// workspace every step, so its maps are encoded once
+struct TmaMapCacheEntry { const void* base; long long rows, cols; int kind, dev; TmaMaps maps; };
+template <typename Build>
+static inline bool cached_maps(TmaMaps* out, int kind, void* base, long long rows, long long cols, Build build) {
+    static thread_local TmaMapCacheEntry cache[8];
+    static thread_local int next = 0, used = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    for (int i = 0; i < used; ++i) {
+        const TmaMapCacheEntry& c = cache[i];
+        if (c.base == base && c.rows == rows && c.cols == cols && c.kind == kind && c.dev == dev) { *out = c.maps; return true; }
+    }
+    if (!build(out)) return false;
+    TmaMapCacheEntry& c = cache[next];
+    c.base = base; c.rows = rows; c.cols = cols; c.kind = kind; c.dev = dev; c.maps = *out;
+    next = (next + 1) & 7;
+    if (used < 8) ++used;
+    return true;
+}
+
+static inline bool make_maps_uncached(TmaMaps* maps, void* base, long long rows, long long cols) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     for (int i = 0; i < 5; ++i) {
@@ -259,3 +309,6 @@ static inline bool make_maps(TmaMaps* maps, void* base, long long rows, long lon
     return true;
 }
 
+static inline bool make_maps(TmaMaps* maps, void* base, long long rows, long long cols) {
+    return cached_maps(maps, 0, base, rows, cols, [&](TmaMaps* m) { return make_maps_uncached(m, base, rows, cols); });
+}
