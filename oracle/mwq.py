@@ -12,9 +12,17 @@ Readings taken where the paper is silent:
   toward -inf from the group minimum, and the scale ``s1`` is the fp16 value rounded toward +inf
   from (max - lo)/(2^b1 - 1), so the base grid always covers the group.  s1 == 0 becomes 2^-14.
 * Eq. 4 with Q in {+1,-1}: Q = sign of the residual, sign(0) = +1.
-* Residual scales are tied, s_j = s1 * 2^-(j+1) for the j-th extra bit (the expected absolute
-  residual of a uniform residual on a cell of width s_{j-1}*2), which makes the b-bit code the
-  b most significant bits of the top-width code.
+* Residual scales, default (``scale_mode = 0``): tied, s_j = s1 * 2^-(j+1) for the j-th extra bit
+  (the expected absolute residual of a uniform residual on a cell of width s_{j-1}*2), which makes
+  the b-bit code the b most significant bits of the top-width code.
+* Residual scales, ``scale_mode = 1``: free, one scale per (row, group) and extra bit, as Eq. 4 and
+  Eq. 5 print them.  Eq. 5 picks s_{b_k} to minimise || R X - s Q X ||; without calibration data
+  (X proportional to the identity) and with Q = sign(R) the minimiser is the mean absolute residual
+  of the group, s_j = mean_G |R|, which is what is stored (rounded to the nearest fp16; the paper
+  does not say how scales are stored).  The mean is an fp32 sum in a pinned order (32 strided
+  partial sums, then a butterfly) so that the stored scales, and with them every later bit, are
+  reproducible bit for bit.  The codes stay nested either way: the bits up to width b do not depend
+  on later steps.
 * The reconstruction rule printed below Eq. 5 has a garbled summation index; it is read as
   W_hat_{b_k} = W_hat_{b_1} + sum_i s_{b_i} Q_{W_{b_i}}.
 * Width lists that skip widths (2,4,8) run every one-bit step internally and expose only the
@@ -23,7 +31,7 @@ Readings taken where the paper is silent:
 from __future__ import annotations
 
 from dataclasses import dataclass
-from typing import List, Sequence, Tuple
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -55,12 +63,15 @@ class MWQTensor:
     code : uint8 [rows, cols], the top-width code (``bits[-1]`` significant bits).
     s1   : fp32 [rows, cols/g], base scale (an fp16-representable value).
     lo   : fp32 [rows, cols/g], base offset = -z*s of Eq. 2 (an fp16-representable value).
+    s_extra : None (tied residual scales) or fp32 [rows, cols/g, top - b1]: the free scale of every
+           extra bit, s_extra[..., j-1] = s_j of Eq. 4 (fp16-representable values).
     """
     code: np.ndarray
     s1: np.ndarray
     lo: np.ndarray
     bits: Tuple[int, ...]
     group_size: int
+    s_extra: Optional[np.ndarray] = None
 
     @property
     def top(self) -> int:
@@ -76,13 +87,33 @@ def check_bits(bits: Sequence[int]) -> None:
     assert all(bits[i] < bits[i + 1] for i in range(len(bits) - 1)), "widths must ascend"
 
 
-def quantize(W: np.ndarray, bits: Sequence[int], group_size: int) -> MWQTensor:
+def sum_pinned(a: np.ndarray) -> np.ndarray:
+    """fp32 sum over the last axis in the pinned order: partial sum l takes elements l, l+32, ... in
+    ascending order, then a butterfly over the 32 partial sums (offsets 16, 8, 4, 2, 1)."""
+    a = np.ascontiguousarray(a, dtype=F32)
+    n = a.shape[-1]
+    if n % 32:
+        a = np.concatenate([a, np.zeros(a.shape[:-1] + (32 - n % 32,), dtype=F32)], axis=-1)
+    a = a.reshape(a.shape[:-1] + (-1, 32))
+    acc = np.zeros(a.shape[:-2] + (32,), dtype=F32)
+    for m in range(a.shape[-2]):
+        acc = (acc + a[..., m, :]).astype(F32)
+    lanes = np.arange(32)
+    for off in (16, 8, 4, 2, 1):
+        acc = (acc + acc[..., lanes ^ off]).astype(F32)
+    return acc[..., 0]
+
+
+def quantize(W: np.ndarray, bits: Sequence[int], group_size: int, scale_mode: int = 0) -> MWQTensor:
     """MWQ of W [rows, cols] with groups of ``group_size`` along the input (column) axis.
 
     Step 1 is the per-group asymmetric b1-bit quantization of Eq. 2; steps 2.. are the binary
-    residual quantization of Eq. 4, one bit per step up to the top width.  All arithmetic is fp32
-    with one rounding per operation (numpy does not contract a*b+c).
+    residual quantization of Eq. 4, one bit per step up to the top width, with tied scales
+    (``scale_mode = 0``) or with the free per-step scale of Eq. 5 (``scale_mode = 1``, see the
+    module docstring).  All arithmetic is fp32 with one rounding per operation (numpy does not
+    contract a*b+c).
     """
+    assert scale_mode in (0, 1)
     check_bits(bits)
     W = np.ascontiguousarray(W, dtype=F32)
     rows, cols = W.shape
@@ -104,14 +135,21 @@ def quantize(W: np.ndarray, bits: Sequence[int], group_size: int) -> MWQTensor:
     What = (lo_b + Q * s1_b).astype(F32)              # (Q - z) * s
     R = (Wg - What).astype(F32)
     code = Q.astype(np.int32)
+    s_extra = np.zeros((rows, cols // g, top - b1), dtype=F32) if scale_mode == 1 else None
     for j in range(1, top - b1 + 1):
-        s_j = (s1_b * F32(2.0 ** -(j + 1))).astype(F32)   # exact: power-of-two multiple
+        if scale_mode == 0:
+            s_j = (s1_b * F32(2.0 ** -(j + 1))).astype(F32)   # exact: power-of-two multiple
+        else:
+            # Eq. 5 without calibration data: argmin_s ||R - s sign(R)||^2 = mean |R| over the group
+            mean_abs = (sum_pinned(np.abs(R)) / F32(g)).astype(F32)
+            s_extra[:, :, j - 1] = mean_abs.astype(np.float16).astype(F32)
+            s_j = s_extra[:, :, j - 1][:, :, None]
         bit = R >= 0                                       # Eq. 4, Q in {+1,-1}
         What = (What + np.where(bit, s_j, -s_j)).astype(F32)
         R = (Wg - What).astype(F32)
         code = code * 2 + bit.astype(np.int32)
     assert code.min() >= 0 and code.max() < (1 << top)
-    return MWQTensor(code.reshape(rows, cols).astype(np.uint8), s1, lo, tuple(bits), g)
+    return MWQTensor(code.reshape(rows, cols).astype(np.uint8), s1, lo, tuple(bits), g, s_extra)
 
 
 def slice_code(q: MWQTensor, b: int) -> np.ndarray:
@@ -133,14 +171,16 @@ def dequantize(q: MWQTensor, b: int) -> np.ndarray:
     W = lo + base.astype(np.float64) * s1
     for j in range(1, b - q.b1 + 1):
         bit = (code >> (q.top - q.b1 - j)) & 1
-        W = W + np.where(bit == 1, 1.0, -1.0) * (s1 * 2.0 ** -(j + 1))
+        s_j = s1 * 2.0 ** -(j + 1) if q.s_extra is None else q.s_extra[:, :, j - 1].astype(np.float64)[:, :, None]
+        W = W + np.where(bit == 1, 1.0, -1.0) * s_j
     return W.reshape(rows, cols)
 
 
 def dequantize_closed_form(q: MWQTensor, b: int) -> np.ndarray:
     """Same weights from the sliced integer code alone: with q_b = code >> (top-b) and
     s_b = s1 / 2^(b-b1), W_hat_b = (lo - s1/2) + s_b * (q_b + 1/2), the midpoint of cell q_b of a
-    uniform grid of 2^b cells.  Used to pin ``dequantize`` (two independent formulas)."""
+    uniform grid of 2^b cells.  Used to pin ``dequantize`` (two independent formulas).  Tied scales only."""
+    assert q.s_extra is None
     rows, cols = q.code.shape
     g = q.group_size
     qb = slice_code(q, b).reshape(rows, cols // g, g).astype(np.float64)

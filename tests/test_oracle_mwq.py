@@ -237,3 +237,99 @@ def test_code_round_trip_on_random_weights():
         s_b = s1 / 2.0 ** (b - 2)
         cell = np.floor((mwq.dequantize(q, b) - (lo - s1 / 2)) / s_b).astype(np.int64)
         assert np.array_equal(cell, mwq.slice_code(q, b).astype(np.int64))
+
+
+# ---------------------------------------------------------------- free per-level scales (Eq. 4 and Eq. 5, scale_mode = 1)
+def test_sum_pinned_is_an_exact_sum_on_integers_and_order_sensitive():
+    a = rng.integers(-1000, 1000, size=(5, 7, 96)).astype(F32)
+    assert np.array_equal(mwq.sum_pinned(a), a.sum(axis=-1, dtype=np.float64).astype(F32))
+    # an input where a plain left-to-right fp32 sum gives another float than the pinned order
+    x = np.zeros(64, dtype=F32)
+    x[0], x[1], x[33] = F32(2.0 ** 24), F32(1.0), F32(1.0)
+    seq = F32(0)
+    for v in x:
+        seq = F32(seq + v)
+    assert seq == F32(2.0 ** 24)                      # each 1.0 is absorbed on its own
+    assert mwq.sum_pinned(x) == F32(2.0 ** 24 + 2.0)  # pinned: partial sum 1 holds 1.0 + 1.0, and 2^24 + 2 is exact
+    # whatever the order, the result stays within n ulps of the fp64 sum
+    y = np.abs(gaussian(3, 256, seed=11))
+    assert np.allclose(mwq.sum_pinned(y), y.sum(axis=-1, dtype=np.float64), rtol=1e-6)
+
+
+def test_free_scales_share_the_base_step_and_keep_the_codes_nested():
+    W = gaussian(16, 256, seed=21)
+    bits = (2, 3, 4, 8)
+    tied = mwq.quantize(W, bits, 64)
+    free = mwq.quantize(W, bits, 64, scale_mode=1)
+    # Eq. 2 is untouched: base code, scale and offset are those of the tied mode
+    assert np.array_equal(free.s1, tied.s1) and np.array_equal(free.lo, tied.lo)
+    assert np.array_equal(mwq.slice_code(free, 2), mwq.slice_code(tied, 2))
+    # the first residual bit only depends on the sign of the base residual: also shared
+    assert np.array_equal(mwq.slice_code(free, 3), mwq.slice_code(tied, 3))
+    assert free.s_extra.shape == (16, 4, 6)
+    assert np.array_equal(free.s_extra.astype(np.float16).astype(F32), free.s_extra)      # fp16-representable
+    # truncated lists give the MSB prefix of the codes and the prefix of the scales
+    for n in range(1, len(bits)):
+        part = mwq.quantize(W, bits[:n], 64, scale_mode=1)
+        assert np.array_equal(part.code, mwq.slice_code(free, bits[n - 1]))
+        assert np.array_equal(part.s_extra, free.s_extra[:, :, :bits[n - 1] - 2])
+
+
+def test_free_scale_is_the_least_squares_scale_of_the_sign_code():
+    """Eq. 5 with X = I and Q = sign(R): argmin_s ||R - s Q||^2 = mean |R|.  Brute force: recompute the residual
+    before every step from the stored codes and scales, and check that no fp16 neighbour of the stored scale
+    (nor any scale of a fine grid) gives a smaller squared error."""
+    W = gaussian(6, 128, seed=22)
+    bits, g = (2, 8), 32
+    q = mwq.quantize(W, bits, g, scale_mode=1)
+    Wg = W.reshape(6, 4, g).astype(np.float64)
+    code = q.code.reshape(6, 4, g).astype(np.int64)
+    What = q.lo.astype(np.float64)[:, :, None] + (code >> 6) * q.s1.astype(np.float64)[:, :, None]
+    for j in range(1, 7):
+        R = Wg - What
+        sign = np.where(((code >> (6 - j)) & 1) == 1, 1.0, -1.0)
+        assert np.array_equal(sign, np.where(R >= 0, 1.0, -1.0))            # Eq. 4: Q = sign(R)
+        s = q.s_extra[:, :, j - 1].astype(np.float64)
+        err = lambda sc: ((R - sc[:, :, None] * sign) ** 2).sum(axis=2)
+        best = err(s)
+        h = q.s_extra[:, :, j - 1].astype(np.float16)
+        for nb in (np.nextafter(h, np.float16(np.inf)), np.nextafter(h, np.float16(-np.inf))):
+            assert np.all(best <= err(nb.astype(np.float64)) * (1 + 1e-12))
+        # the error is a parabola in the scale with its minimum at mean |R|; the stored scale is that value rounded to
+        # fp16, i.e. at most g (2^-11 s)^2 above the minimum: no scale of a fine grid does better than that
+        slack = g * (2.0 ** -11 * s) ** 2
+        for f in np.linspace(0.0, 3.0, 61):
+            assert np.all(best <= err(s * f) + slack)
+        assert np.allclose(s, np.abs(R).mean(axis=2), rtol=2.0 ** -10)       # = mean |R| up to fp16 rounding
+        What = What + s[:, :, None] * sign
+
+
+def test_free_scales_never_increase_the_error_and_dequantize_is_additive():
+    W = gaussian(8, 256, seed=23)
+    q = mwq.quantize(W, (2, 3, 4, 8), 128, scale_mode=1)
+    prev = None
+    for b in range(2, 9):
+        Wb = mwq.dequantize(q, b)
+        e = ((Wb - W) ** 2).reshape(8, 2, 128).sum(axis=2)
+        if prev is not None:
+            assert np.all(e <= prev * (1 + 1e-3))          # each step's scale minimises that step's error (fp16-rounded)
+        prev = e
+    # additive rule written out for one weight
+    r, c, g = 3, 200, 128
+    G, top, b1 = c // g, 8, 2
+    code = int(q.code[r, c])
+    w = float(q.lo[r, G]) + (code >> 6) * float(q.s1[r, G])
+    for j in range(1, 7):
+        w += (1.0 if (code >> (6 - j)) & 1 else -1.0) * float(q.s_extra[r, G, j - 1])
+    assert mwq.dequantize(q, 8)[r, c] == pytest.approx(w, rel=1e-15)
+
+
+def test_free_scales_approach_the_tied_ones_on_uniform_residuals():
+    # weights spread uniformly over the base grid's range: the mean absolute residual of a uniform residual on a cell
+    # of width c is c / 4, so s_1 ~ s1 / 4, s_2 ~ s1 / 8, ...: the free scales fall back on the tied ones
+    r = np.random.default_rng(24)
+    W = r.uniform(-1.0, 1.0, size=(4, 4096)).astype(F32)
+    q = mwq.quantize(W, (2, 8), 256, scale_mode=1)
+    for j in range(1, 4):
+        ratio = q.s_extra[:, :, j - 1] / (q.s1 * 2.0 ** -(j + 1))
+        assert np.all(np.abs(ratio - 1.0) < 0.15), (j, ratio.min(), ratio.max())
