@@ -31,7 +31,7 @@ typedef enum {
     D2MOE_ERR_NULL = 1,        /* a required pointer is NULL                                  */
     D2MOE_ERR_CONFIG = 2,      /* d2moe_config is inconsistent                                */
     D2MOE_ERR_SHAPE = 3,       /* a size does not fit the configuration                       */
-    D2MOE_ERR_UNSUPPORTED = 4, /* valid but not built (e.g. scale_mode 1)                     */
+    D2MOE_ERR_UNSUPPORTED = 4, /* valid but not possible (e.g. D2MOE_PATH_TENSOR on an odd shape) */
     D2MOE_ERR_WORKSPACE = 5,   /* workspace or output buffer too small                        */
     D2MOE_ERR_CUDA = 6,        /* a CUDA runtime call or launch failed                        */
     D2MOE_ERR_TIMEOUT = 7,     /* device_status bit: a bounded device-side wait ran out       */
@@ -65,8 +65,12 @@ typedef struct {
     int32_t d_model, d_ffn, n_experts, top_k, n_shared, group_size;
     int32_t n_bits, bits[8];
     int32_t renormalize;   /* 1: weights of the selected experts are divided by their sum       */
-    int32_t scale_mode;    /* 0: tied residual scales s_j = s1 / 2^(j+1).  1 (free per-level
-                              scales of Eq. 5) is not built: D2MOE_ERR_UNSUPPORTED               */
+    int32_t scale_mode;    /* 0: tied residual scales s_j = s1 / 2^(j+1) (the b-bit code is then a uniform
+                              b-bit grid).  1: free scales, as Eq. 4 / Eq. 5 print them: every extra bit
+                              has its own fp16 scale per (row, group), s_j = mean |residual| of the group
+                              (the minimiser of Eq. 5 without calibration data); the codes stay nested.
+                              With free scales every batch size runs on the fp16 grouped GEMM (or the
+                              CUDA-core path): the 8-bit decode kernel needs the tied form.            */
     int32_t kernel_path;   /* D2MOE_PATH_*                                                      */
     int32_t reserved[3];   /* must be 0                                                         */
 } d2moe_config;
@@ -81,14 +85,16 @@ d2moe_status d2moe_check_config(const d2moe_config* cfg);
  * total = header + code bytes + metadata bytes; code_bytes and meta_bytes (either may be NULL) give
  * the split: code_bytes = rows_padded*cols*bits[n_bits-1]/8 when every segment width is 1, 2, 4 or 8
  * bits (segments of 3 / 5..7 bits are stored in 4 / 8), metadata = one (fp16 scale, fp16 offset)
- * pair per row and group.  The nested store costs the top width only, whatever n_bits is.
+ * pair per row and group, plus, with scale_mode 1, one fp16 scale per extra bit (bits[n_bits-1] -
+ * bits[0] of them) per row and group.  The nested store costs the top width only, whatever n_bits is.
  */
 d2moe_status d2moe_packed_bytes(const d2moe_config* cfg, int64_t rows, int64_t cols,
                                 size_t* total_bytes, size_t* code_bytes, size_t* meta_bytes);
 
 /*
  * MWQ quantization and packing of one matrix (Section 3.3.1: Eq. 2 base step at bits[0], then one
- * binary residual step of Eq. 4 per extra bit up to bits[n_bits-1], tied scales, calibration-free).
+ * binary residual step of Eq. 4 per extra bit up to bits[n_bits-1], scales per cfg->scale_mode,
+ * calibration-free).
  *   W       device, fp32 [rows, cols] row-major, finite, |W| < 65504
  *   packed  device, packed_bytes >= d2moe_packed_bytes(); 256-byte aligned; layout is private to
  *           this library (bit-plane segments tiled for the expert kernels) and versioned by a header.
@@ -105,6 +111,14 @@ d2moe_status d2moe_pack_mwq(const d2moe_config* cfg, const float* W, int64_t row
 d2moe_status d2moe_unpack_codes(const d2moe_config* cfg, const void* packed, int64_t rows,
                                 int64_t cols, int bits, uint8_t* codes, float* scale, float* offset,
                                 void* stream);
+
+/*
+ * Test hook for scale_mode 1: the free scale of every residual step of Eq. 4, s_extra[(r * (cols /
+ * group_size) + G) * n_steps + j - 1] = s_j of row r, group G, n_steps = bits[n_bits-1] - bits[0]
+ * (device fp32, values are fp16-representable).  D2MOE_ERR_CONFIG when cfg->scale_mode != 1.
+ */
+d2moe_status d2moe_unpack_scales(const d2moe_config* cfg, const void* packed, int64_t rows, int64_t cols,
+                                 float* s_extra, void* stream);
 
 /* Workspace (device bytes) d2moe_route and d2moe_moe_forward need for up to max_tokens tokens. */
 size_t d2moe_workspace_bytes(const d2moe_config* cfg, int64_t max_tokens);

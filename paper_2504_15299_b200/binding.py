@@ -50,7 +50,7 @@ _lib = None
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
            "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count",
-           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry"]
+           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry", "d2moe_unpack_scales"]
 
 
 def lib() -> ctypes.CDLL:
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
     L.d2moe_packed_bytes.argtypes = [cfgp, i64, i64, ctypes.POINTER(sz), ctypes.POINTER(sz), ctypes.POINTER(sz)]
     L.d2moe_pack_mwq.argtypes = [cfgp, vp, i64, i64, vp, sz, vp]
     L.d2moe_unpack_codes.argtypes = [cfgp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
+    L.d2moe_unpack_scales.argtypes = [cfgp, vp, i64, i64, vp, vp]
     L.d2moe_workspace_bytes.restype = sz
     L.d2moe_workspace_bytes.argtypes = [cfgp, i64]
     L.d2moe_route.argtypes = [cfgp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -114,9 +115,9 @@ class Config:
         return c
 
     @staticmethod
-    def from_workload(wl, kernel_path: int = PATH_AUTO) -> "Config":
+    def from_workload(wl, kernel_path: int = PATH_AUTO, scale_mode: int = 0) -> "Config":
         return Config(wl.d_model, wl.d_ffn, wl.n_experts, wl.top_k, wl.group_size, tuple(wl.bits),
-                      n_shared=wl.n_shared, renormalize=wl.renormalize, kernel_path=kernel_path)
+                      n_shared=wl.n_shared, renormalize=wl.renormalize, kernel_path=kernel_path, scale_mode=scale_mode)
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -176,6 +177,15 @@ def unpack_codes(cfg: Config, packed: torch.Tensor, rows: int, cols: int, bits: 
     _check(lib().d2moe_unpack_codes(ctypes.byref(cfg.c()), _ptr(packed), rows, cols, bits, _ptr(codes),
                                     _ptr(scale), _ptr(offset), _stream(stream)), "d2moe_unpack_codes")
     return codes, scale, offset
+
+
+def unpack_scales(cfg: Config, packed: torch.Tensor, rows: int, cols: int, stream=None) -> torch.Tensor:
+    """scale_mode 1: the free scale of every residual step, fp32 [rows, cols / g, top - b1]."""
+    n_steps = cfg.bits[-1] - cfg.bits[0]
+    out = torch.empty((rows, cols // cfg.group_size, n_steps), dtype=torch.float32, device=packed.device)
+    _check(lib().d2moe_unpack_scales(ctypes.byref(cfg.c()), _ptr(packed), rows, cols, _ptr(out), _stream(stream)),
+           "d2moe_unpack_scales")
+    return out
 
 
 @dataclass

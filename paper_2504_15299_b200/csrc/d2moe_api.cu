@@ -51,8 +51,7 @@ extern "C" d2moe_status d2moe_check_config(const d2moe_config* c) {
     for (int i = 1; i < c->n_bits; ++i)
         if (c->bits[i] <= c->bits[i - 1]) return D2MOE_ERR_CONFIG;
     if (c->renormalize != 0 && c->renormalize != 1) return D2MOE_ERR_CONFIG;
-    if (c->scale_mode == 1) return D2MOE_ERR_UNSUPPORTED;
-    if (c->scale_mode != 0) return D2MOE_ERR_CONFIG;
+    if (c->scale_mode != 0 && c->scale_mode != 1) return D2MOE_ERR_CONFIG;
     if (c->kernel_path < 0 || c->kernel_path > 2) return D2MOE_ERR_CONFIG;
     for (int i = 0; i < 3; ++i)
         if (c->reserved[i] != 0) return D2MOE_ERR_CONFIG;
@@ -67,10 +66,11 @@ extern "C" d2moe_status d2moe_packed_bytes(const d2moe_config* c, int64_t rows, 
     if (rows <= 0 || cols <= 0 || cols % c->group_size || rows > (1 << 24) || cols > (1 << 24))
         return D2MOE_ERR_SHAPE;
     PackLayout L;
-    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols);
+    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols, c->scale_mode);
     const size_t n_blocks = (size_t)L.n_rt * L.n_groups;
-    const size_t meta = n_blocks * D2MOE_TILE_ROWS * 4;
-    const size_t code = n_blocks * (size_t)(L.block_bytes - D2MOE_TILE_ROWS * 4);
+    const size_t n_steps = c->scale_mode == 1 ? (size_t)(L.top - L.b1) : 0;       // free scales: one fp16 per extra bit
+    const size_t meta = n_blocks * D2MOE_TILE_ROWS * (4 + 2 * n_steps);
+    const size_t code = n_blocks * (size_t)L.block_bytes - meta;
     *total_bytes = D2MOE_HEADER_BYTES + meta + code;
     if (code_bytes) *code_bytes = code;
     if (meta_bytes) *meta_bytes = meta;
@@ -86,7 +86,7 @@ extern "C" d2moe_status d2moe_pack_mwq(const d2moe_config* c, const float* W, in
     if (packed_bytes < need) return D2MOE_ERR_WORKSPACE;
     if (((uintptr_t)packed & 255) != 0) return D2MOE_ERR_SHAPE;
     PackLayout L;
-    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols);
+    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols, c->scale_mode);
     cudaError_t e = launch_pack(L, c->bits, c->n_bits, W, (uint8_t*)packed, (cudaStream_t)stream);
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
@@ -100,8 +100,21 @@ extern "C" d2moe_status d2moe_unpack_codes(const d2moe_config* c, const void* pa
     if (!packed || !codes) return D2MOE_ERR_NULL;
     if (bits < c->bits[0] || bits > c->bits[c->n_bits - 1]) return D2MOE_ERR_SHAPE;
     PackLayout L;
-    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols);
+    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols, c->scale_mode);
     cudaError_t e = launch_unpack(L, (const uint8_t*)packed, bits, codes, scale, offset, (cudaStream_t)stream);
+    return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+}
+
+extern "C" d2moe_status d2moe_unpack_scales(const d2moe_config* c, const void* packed, int64_t rows,
+                                            int64_t cols, float* s_extra, void* stream) {
+    size_t need = 0;
+    d2moe_status s = d2moe_packed_bytes(c, rows, cols, &need, nullptr, nullptr);
+    if (s != D2MOE_OK) return s;
+    if (c->scale_mode != 1) return D2MOE_ERR_CONFIG;
+    if (!packed || !s_extra) return D2MOE_ERR_NULL;
+    PackLayout L;
+    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols, c->scale_mode);
+    cudaError_t e = launch_unpack_scales(L, (const uint8_t*)packed, s_extra, (cudaStream_t)stream);
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
 
@@ -276,8 +289,8 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     memset(&P, 0, sizeof(P));
     for (int i = 0; i < 3 * n_exp; ++i) P.w[i] = (const uint8_t*)expert_w[i];
     PackLayout Lgu, Ld;
-    d2moe_make_layout(Lgu, c->bits, c->n_bits, c->group_size, c->d_ffn, c->d_model);
-    d2moe_make_layout(Ld, c->bits, c->n_bits, c->group_size, c->d_model, c->d_ffn);
+    d2moe_make_layout(Lgu, c->bits, c->n_bits, c->group_size, c->d_ffn, c->d_model, c->scale_mode);
+    d2moe_make_layout(Ld, c->bits, c->n_bits, c->group_size, c->d_model, c->d_ffn, c->scale_mode);
 
     if (use_tensor_path(c)) {
         TcPlan pl;

@@ -34,6 +34,12 @@
 //   bytes 0 and 2, and the pair (k+2, k+3) from bytes 1 and 3 after a shift by 8.
 //
 // A call at width bits[kk] needs meta and segments 0..kk of a block: one contiguous prefix.
+//
+// Free per-step residual scales (scale_mode 1, Eq. 4 / Eq. 5): segment j >= 1 adds w_j one-bit steps, each
+// with its own fp16 scale per (row, group).  Those scales sit directly in front of the segment's codes,
+//   block = meta | segment 0 | scales of segment 1 | segment 1 | scales of segment 2 | segment 2 | ...
+// as w_j planes of 64 fp16 values (step l of the segment, row r at byte (l*64 + r)*2), so that a call at
+// width bits[kk] still reads one contiguous prefix.
 // ------------------------------------------------------------------------------------------------
 struct PackLayout {
     int rows, cols, g, n_groups, rows_pad, n_rt;
@@ -44,6 +50,9 @@ struct PackLayout {
     int seg_cs[D2MOE_MAX_SEG];     // chunk size in bytes
     int seg_off[D2MOE_MAX_SEG + 1];// byte offset of segment j inside a block; [n_seg] = block size
     int block_bytes;
+    int scale_mode;                // 0 tied residual scales, 1 free (one fp16 scale per row, group and extra bit)
+    int seg_sc_off[D2MOE_MAX_SEG]; // scale_mode 1: byte offset of the scales of segment j (j >= 1) inside a block
+    int seg_lv0[D2MOE_MAX_SEG];    // first residual step (0-based) that segment j adds; it adds seg_w[j] steps (j >= 1)
 };
 
 struct PackHeader {
@@ -52,14 +61,16 @@ struct PackHeader {
     int32_t bits[8];
     uint32_t s1_max_bits;          // bit pattern of the largest fp32 s1 in the matrix
     uint32_t wabs_max_bits;        // bit pattern of the largest |W| in the matrix
-    uint32_t pad[48];
+    int32_t scale_mode;
+    uint32_t pad[47];
 };
 static_assert(sizeof(PackHeader) == D2MOE_HEADER_BYTES, "header size");
 
 __host__ __device__ inline int d2moe_storage_width(int w) { return w <= 1 ? 1 : (w <= 2 ? 2 : (w <= 4 ? 4 : 8)); }
 
 __host__ __device__ inline void d2moe_make_layout(PackLayout& L, const int* bits, int n_bits, int g,
-                                                  long long rows, long long cols) {
+                                                  long long rows, long long cols, int scale_mode = 0) {
+    L.scale_mode = scale_mode;
     L.rows = (int)rows; L.cols = (int)cols; L.g = g; L.n_groups = (int)(cols / g);
     L.rows_pad = (int)((rows + D2MOE_TILE_ROWS - 1) / D2MOE_TILE_ROWS * D2MOE_TILE_ROWS);
     L.n_rt = L.rows_pad / D2MOE_TILE_ROWS;
@@ -72,10 +83,14 @@ __host__ __device__ inline void d2moe_make_layout(PackLayout& L, const int* bits
             L.seg_shift[j] = L.top - bits[j];
             int row_bytes = g * L.seg_sw[j] / 8;
             L.seg_cs[j] = row_bytes < 16 ? row_bytes : 16;
+            L.seg_lv0[j] = j == 0 ? 0 : bits[j - 1] - bits[0];
+            L.seg_sc_off[j] = off;
+            if (scale_mode == 1 && j >= 1) off += D2MOE_TILE_ROWS * 2 * L.seg_w[j];
             L.seg_off[j] = off;
             off += D2MOE_TILE_ROWS * row_bytes;
         } else {
             L.seg_w[j] = L.seg_sw[j] = L.seg_shift[j] = L.seg_cs[j] = 0; L.seg_off[j] = off;
+            L.seg_sc_off[j] = off; L.seg_lv0[j] = 0;
         }
     }
     L.seg_off[n_bits < D2MOE_MAX_SEG ? n_bits : D2MOE_MAX_SEG] = off;
@@ -94,6 +109,18 @@ __host__ __device__ inline int d2moe_elem_word(const PackLayout& L, int j, int r
     int ob = 4 * m, cs = L.seg_cs[j];
     int c = ob / cs, within = ob - c * cs;
     return L.seg_off[j] + (c * D2MOE_TILE_ROWS + r) * cs + within;
+}
+
+// scale_mode 1: byte offset (inside a block) of the fp16 scale of residual step `level` (0-based) of row r
+__host__ __device__ inline int d2moe_level_offset(const PackLayout& L, int level, int r) {
+    int j = 1;
+    while (j + 1 < L.n_seg && L.seg_lv0[j + 1] <= level) ++j;
+    return L.seg_sc_off[j] + ((level - L.seg_lv0[j]) * D2MOE_TILE_ROWS + r) * 2;
+}
+
+// bytes of a block that a call at width index kk reads: meta and segments 0..kk (with their scales)
+__host__ __device__ inline int d2moe_prefix_bytes(const PackLayout& L, int kk) {
+    return kk + 1 < L.n_seg ? L.seg_sc_off[kk + 1] : L.block_bytes;
 }
 
 __host__ __device__ inline size_t d2moe_block_offset(const PackLayout& L, int rt, int G) {
@@ -144,6 +171,7 @@ cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const 
                         cudaStream_t st);
 cudaError_t launch_unpack(const PackLayout& L, const uint8_t* packed, int bits, uint8_t* codes,
                           float* scale, float* offset, cudaStream_t st);
+cudaError_t launch_unpack_scales(const PackLayout& L, const uint8_t* packed, float* s_extra, cudaStream_t st);
 
 // kernels_route.cu
 cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,

@@ -48,6 +48,14 @@ __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed
         const float sb = s1 * inv;
         const float base = lo - 0.5f * s1;
         const VT* vg = v + (size_t)G * L.g;
+        // free residual scales (Eq. 4 / Eq. 5): the additive rule W_hat = lo + s1 Q + sum over the steps of (+-) s_l
+        const int n_lv = width - L.b1;
+        float sl[7];
+        if (L.scale_mode == 1) {
+#pragma unroll
+            for (int l = 0; l < 7; ++l)
+                sl[l] = l < n_lv ? __half2float(*reinterpret_cast<const __half*>(blk + d2moe_level_offset(L, l, r))) : 0.0f;
+        }
         for (int i = lane; i < L.g / 2; i += 32) {      // pair (2i, 2i+1)
             unsigned q0 = 0, q1 = 0;
             for (int j = 0; j <= kk; ++j) {
@@ -59,8 +67,21 @@ __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed
                 q1 |= ((word >> (bitpos + 16)) & mask) << L.seg_shift[j];
             }
             q0 >>= b; q1 >>= b;
-            const float w0 = fmaf(sb, (float)q0 + 0.5f, base);
-            const float w1 = fmaf(sb, (float)q1 + 0.5f, base);
+            float w0, w1;
+            if (L.scale_mode == 1) {
+                w0 = fmaf(s1, (float)(q0 >> n_lv), lo);
+                w1 = fmaf(s1, (float)(q1 >> n_lv), lo);
+#pragma unroll
+                for (int l = 0; l < 7; ++l) {
+                    if (l < n_lv) {
+                        w0 += ((q0 >> (n_lv - 1 - l)) & 1u) ? sl[l] : -sl[l];
+                        w1 += ((q1 >> (n_lv - 1 - l)) & 1u) ? sl[l] : -sl[l];
+                    }
+                }
+            } else {
+                w0 = fmaf(sb, (float)q0 + 0.5f, base);
+                w1 = fmaf(sb, (float)q1 + 0.5f, base);
+            }
             acc = fmaf(w0, to_f32(vg[2 * i]), acc);
             acc = fmaf(w1, to_f32(vg[2 * i + 1]), acc);
         }

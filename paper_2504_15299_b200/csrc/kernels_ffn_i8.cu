@@ -326,7 +326,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const I8Item ii = i8_item(p, item);
                 const I8Unit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
-                const uint32_t bytes = (uint32_t)p.L.seg_off[kmax + 1];
+                const uint32_t bytes = (uint32_t)d2moe_prefix_bytes(p.L, kmax);
                 const uint8_t *m0, *m1;
                 if (p.mode == 0) {
                     m0 = p.P.w[3 * e + 0] + d2moe_block_offset(p.L, ii.tile, ii.g0);

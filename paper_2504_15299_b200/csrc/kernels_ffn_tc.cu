@@ -117,6 +117,63 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, 
     }
 }
 
+// Free residual scales (scale_mode 1): a segment after the first adds W one-bit steps, each with its own scale, so
+// its codes are folded in bit by bit: U += (2 s_l) bit_l for every step l of the segment (the constant - s_l of
+// W_hat = ... + s_l (2 bit_l - 1) is added when the tile is written).  mb[pos]: multiplier of a bit at position pos
+// of its byte lane, 2 s_l 2^(24 - S - pos) for the step that bit belongs to (0 for the unused bits of the field).
+template <int GS, int SW>
+__device__ __forceinline__ void dequant_segment_bits(uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], int W,
+                                                     const __half2 (&mb)[8]) {
+    constexpr int ROW_BYTES = GS * SW / 8;
+    constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
+    constexpr int HB = ROW_BYTES / 2;
+    constexpr int LD = HB < 16 ? HB : 16;
+    constexpr int NLD = HB / LD;
+    constexpr int WPL = LD / 4;
+    constexpr int PER = 16 / SW;
+#pragma unroll
+    for (int l = 0; l < NLD; ++l) {
+        uint32_t w[WPL];
+        const int off = half * HB + l * LD;
+        const int c = off / CS, within = off % CS;
+        const uint32_t addr = seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS + within);
+        if constexpr (WPL == 4) {
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+        } else if constexpr (WPL == 2) {
+            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr));
+        } else {
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[0]) : "r"(addr));
+        }
+#pragma unroll
+        for (int q = 0; q < WPL; ++q) {
+            const uint32_t lo8 = w[q], hi8 = w[q] >> 8;
+#pragma unroll
+            for (int e = 0; e < PER; ++e) {
+                const uint32_t src = (e & 1) ? hi8 : lo8;
+                const int i = (l * WPL + q) * PER + e;
+#pragma unroll
+                for (int t = 0; t < SW; ++t) {
+                    if (t < W) {
+                        const int pos = (e >> 1) * SW + t;
+                        acc[i] = __hfma2(as_h2(src & (0x00010001u << pos)), mb[pos], acc[i]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int GS>
+__device__ __forceinline__ void dequant_bits_dispatch(int sw, uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], int W,
+                                                      const __half2 (&mb)[8]) {
+    switch (sw) {
+        case 1: dequant_segment_bits<GS, 1>(seg, rr, half, acc, W, mb); break;
+        case 2: dequant_segment_bits<GS, 2>(seg, rr, half, acc, W, mb); break;
+        case 4: dequant_segment_bits<GS, 4>(seg, rr, half, acc, W, mb); break;
+        default: dequant_segment_bits<GS, 8>(seg, rr, half, acc, W, mb); break;
+    }
+}
+
 template <int GS, bool FIRST>
 __device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], __half2 m0, __half2 u0) {
     switch (sw) {
@@ -197,11 +254,11 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     }
     // per-width constants of the dequant loop, read from shared memory instead of the kernel parameters
     // (a dynamically indexed parameter read costs a constant-cache round trip per tile)
-    int4* seg_tab = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + 256);   // {sw, seg_off, 2^-(bits[kk]-bits[0]) bits, 0}
+    int4* seg_tab = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + 256);   // {sw, seg_off, 2^-(bits[kk]-bits[0]) bits, logical width | offset of the segment's scales << 4}
     if (threadIdx.x < 8) {
         const int kk = threadIdx.x;
         const int db = kk < p.D.K ? p.D.bits[kk] - p.D.bits[0] : 0;
-        seg_tab[kk] = make_int4(p.L.seg_sw[kk], p.L.seg_off[kk], (127 - db) << 23, 0);
+        seg_tab[kk] = make_int4(p.L.seg_sw[kk], p.L.seg_off[kk], (127 - db) << 23, p.L.seg_w[kk] | (p.L.seg_sc_off[kk] << 4));
     }
     if (warp == WARP_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -244,7 +301,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 const ItemInfo ii = decode_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
-                const uint32_t bytes = (uint32_t)p.L.seg_off[kmax + 1];
+                const uint32_t bytes = (uint32_t)d2moe_prefix_bytes(p.L, kmax);
                 const uint8_t *m0, *m1;
                 int rt0, rt1;
                 if (p.mode == 0) { m0 = p.P.w[3 * e + 0]; m1 = p.P.w[3 * e + 1]; rt0 = rt1 = ii.tile; }
@@ -395,12 +452,13 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 const __half2 mh = as_h2(meta);
                 const float s1 = __low2float(mh), lo = __high2float(mh);
                 const __half2 u0 = h2dup((lo - 0.5f * s1) * two_mS);
-                // hands the running tile over as the tile of width index kk (Mk = M_kk * 2^-S)
-                auto write_tile = [&](float Mk) {
+                // hands the running tile over as the tile of a width index; addend: what the tile lacks of W_hat 2^-S
+                // (tied scales: half a step of that width, M_kk / 2)
+                auto write_tile = [&](float addend) {
                     const int slot = at % A_SLOTS;
                     mbar_wait(A_EMPTY(slot), ((at / A_SLOTS) & 1) ^ 1, abort_flag, p.status);
                     tc_fence_after();
-                    const __half2 half_m = h2dup(0.5f * Mk);
+                    const __half2 half_m = h2dup(addend);
                     const uint32_t dst = a_tmem + slot * 64 + wg * (TILE_COLS / 2) + lane_addr;
 #pragma unroll
                     for (int c = 0; c < GS / 64; ++c) {
@@ -425,7 +483,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                                 const float Mk = s1 * __int_as_float((127 - db) << 23) * two_mS;
                                 dequant_segment<GS, WL::sw(J), J == 0>(wb + (uint32_t)WL::seg_off(GS, J), rr, wg, acc,
                                                                       h2dup(Mk * 16777216.0f), u0);
-                                if ((present >> J) & 1u) write_tile(Mk);
+                                if ((present >> J) & 1u) write_tile(0.5f * Mk);
                             }
                         }
                     };
@@ -434,6 +492,38 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     seg_step(std::integral_constant<int, 2>{});
                     seg_step(std::integral_constant<int, 3>{});
                 } else {
+                    if (p.L.scale_mode == 1) {
+                        // free residual scales: W_hat = lo + s1 Q + sum over the steps of s_l (2 bit_l - 1)
+                        float cneg = 0.0f;                       // - sum of the scales of the steps folded in so far, times 2^-S
+#pragma unroll 1
+                        for (int kk = 0; kk <= kmax; ++kk) {
+                            const int4 tb = seg_tab[kk];
+                            const int sw = tb.x;
+                            const uint32_t seg = wb + (uint32_t)tb.y;
+                            if (kk == 0) {
+                                dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, h2dup(s1 * two_mS * 16777216.0f), h2dup(lo * two_mS));
+                            } else {
+                                const int W = tb.w & 15;
+                                const uint32_t sc = wb + (uint32_t)(tb.w >> 4) + 2u * rr;       // this row's scales of the segment
+                                __half2 mb[8];
+#pragma unroll
+                                for (int pos = 0; pos < 8; ++pos) {
+                                    const int t = pos % sw;               // bit of the field; its step: W - 1 - t (most significant first)
+                                    float m = 0.0f;
+                                    if (t < W) {
+                                        unsigned short raw;
+                                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc + (uint32_t)((W - 1 - t) * D2MOE_TILE_ROWS * 2)));
+                                        const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
+                                        m = 2.0f * sl * __int_as_float((127 + 24 - pos) << 23);
+                                        if (pos < sw) cneg -= sl;         // each step once
+                                    }
+                                    mb[pos] = h2dup(m);
+                                }
+                                dequant_bits_dispatch<GS>(sw, seg, rr, wg, acc, W, mb);
+                            }
+                            if ((present >> kk) & 1u) write_tile(cneg);
+                        }
+                    } else {
 #pragma unroll 1
                     for (int kk = 0; kk <= kmax; ++kk) {
                         const int4 tb = seg_tab[kk];
@@ -444,7 +534,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                         const uint32_t seg = wb + (uint32_t)tb.y;
                         if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
                         else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
-                        if ((present >> kk) & 1u) write_tile(Mk);
+                        if ((present >> kk) & 1u) write_tile(0.5f * Mk);
+                    }
                     }
                 }
                 mbar_arrive(W_EMPTY(s));
@@ -769,7 +860,9 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl) {
     const long long avg = (A + c->n_experts - 1) / c->n_experts;
     // up to about 40 tokens per expert the 8-bit kernel (units of 32 slots, weights unpacked once per unit) is
     // faster than the fp16 grouped GEMM (measured crossover on the Mixtral shape: T = 160, 40 tokens per expert)
-    pl->decode = avg <= D2MOE_DECODE_MAX_AVG ? 1 : 0;
+    // (the 8-bit kernel folds one scale per group into its integer accumulators, which needs the tied residual
+    // scales: with free scales every load takes the grouped GEMM)
+    pl->decode = (avg <= D2MOE_DECODE_MAX_AVG && c->scale_mode == 0) ? 1 : 0;
     if (pl->decode) {
         pl->n_cap = 32;                      // token slots per unit
     } else {
@@ -843,7 +936,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         int wpack = 0;
-        if (p.L.n_seg <= 4)
+        if (p.L.n_seg <= 4 && p.L.scale_mode == 0)       // (their segment offsets are compile-time: tied-scale layout)
             for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
         auto launch = [&](auto kc) -> cudaError_t {
             constexpr auto kern = decltype(kc)::value;

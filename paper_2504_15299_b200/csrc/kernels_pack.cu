@@ -12,6 +12,7 @@ __global__ void pack_header_kernel(PackHeader* h, PackLayout L, int n_bits,
         h->rows = L.rows; h->cols = L.cols; h->g = L.g; h->n_bits = n_bits;
         int b[8] = {b0, b1, b2, b3, b4, b5, b6, b7};
         for (int i = 0; i < 8; ++i) h->bits[i] = b[i];
+        h->scale_mode = L.scale_mode;
         // s1_max_bits and wabs_max_bits were zeroed by the memset that precedes this kernel
     }
 }
@@ -35,7 +36,11 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
         const long long row = (long long)rt * D2MOE_TILE_ROWS + r;
         if (row >= L.rows) {                                // padding rows: zero codes, zero meta
             for (int k = lane; k < g; k += 32) codes[r * g + k] = 0;
-            if (lane == 0) reinterpret_cast<uint32_t*>(blk)[r] = 0u;
+            if (lane == 0) {
+                reinterpret_cast<uint32_t*>(blk)[r] = 0u;
+                if (L.scale_mode == 1)
+                    for (int l = 0; l < L.top - L.b1; ++l) *reinterpret_cast<uint16_t*>(blk + d2moe_level_offset(L, l, r)) = 0;
+            }
             continue;
         }
         const float* src = W + row * (long long)L.cols + (long long)G * g;
@@ -50,22 +55,65 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
         __half s1_h = __float2half_ru(__fdiv_rn(__fsub_rn(wmax, lo), levels));
         float s1 = __half2float(s1_h);
         if (s1 == 0.0f) { s1 = 6.103515625e-05f; s1_h = __float2half_rn(s1); }   // 2^-14
-        for (int k = lane; k < g; k += 32) {
-            const float w = src[k];
-            float q = rintf(__fdiv_rn(__fsub_rn(w, lo), s1));
-            q = fminf(fmaxf(q, 0.0f), levels);
-            float what = __fadd_rn(lo, __fmul_rn(q, s1));
-            float res = __fsub_rn(w, what);
-            int code = (int)q;
-            float sj = __fmul_rn(s1, 0.25f);                 // s_1 = s1 * 2^-2
-            for (int j = 1; j <= L.top - L.b1; ++j) {
-                const bool bit = res >= 0.0f;
-                what = __fadd_rn(what, bit ? sj : -sj);
-                res = __fsub_rn(w, what);
-                code = code * 2 + (bit ? 1 : 0);
-                sj = __fmul_rn(sj, 0.5f);
+        if (L.scale_mode == 0) {
+            for (int k = lane; k < g; k += 32) {
+                const float w = src[k];
+                float q = rintf(__fdiv_rn(__fsub_rn(w, lo), s1));
+                q = fminf(fmaxf(q, 0.0f), levels);
+                float what = __fadd_rn(lo, __fmul_rn(q, s1));
+                float res = __fsub_rn(w, what);
+                int code = (int)q;
+                float sj = __fmul_rn(s1, 0.25f);                 // s_1 = s1 * 2^-2
+                for (int j = 1; j <= L.top - L.b1; ++j) {
+                    const bool bit = res >= 0.0f;
+                    what = __fadd_rn(what, bit ? sj : -sj);
+                    res = __fsub_rn(w, what);
+                    code = code * 2 + (bit ? 1 : 0);
+                    sj = __fmul_rn(sj, 0.5f);
+                }
+                codes[r * g + k] = (uint8_t)code;
             }
-            codes[r * g + k] = (uint8_t)code;
+        } else {
+            // free per-step scales: every step needs the group's mean absolute residual first, so the lane keeps
+            // its elements (k = lane, lane + 32, ...: at most 8) in registers and the steps run over the whole group
+            float wv[8], wh[8], rs[8];
+            int cd[8];
+            const int n_el = g >> 5;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                if (e < n_el) {
+                    const float w = src[lane + 32 * e];
+                    float q = rintf(__fdiv_rn(__fsub_rn(w, lo), s1));
+                    q = fminf(fmaxf(q, 0.0f), levels);
+                    wv[e] = w;
+                    wh[e] = __fadd_rn(lo, __fmul_rn(q, s1));
+                    rs[e] = __fsub_rn(w, wh[e]);
+                    cd[e] = (int)q;
+                }
+            }
+            for (int j = 1; j <= L.top - L.b1; ++j) {
+                // mean |R| in the pinned order: this lane's elements ascending, then the butterfly
+                float part = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (e < n_el) part = __fadd_rn(part, fabsf(rs[e]));
+                for (int off = 16; off; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
+                const __half sj_h = __float2half_rn(__fdiv_rn(part, (float)g));
+                const float sj = __half2float(sj_h);
+                if (lane == 0) *reinterpret_cast<__half*>(blk + d2moe_level_offset(L, j - 1, r)) = sj_h;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if (e < n_el) {
+                        const bool bit = rs[e] >= 0.0f;
+                        wh[e] = __fadd_rn(wh[e], bit ? sj : -sj);
+                        rs[e] = __fsub_rn(wv[e], wh[e]);
+                        cd[e] = cd[e] * 2 + (bit ? 1 : 0);
+                    }
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                if (e < n_el) codes[r * g + lane + 32 * e] = (uint8_t)cd[e];
         }
         if (lane == 0) {
             __half2 m = __halves2half2(s1_h, lo_h);          // low half = s1, high half = lo
@@ -130,7 +178,30 @@ __global__ void unpack_kernel(PackLayout L, const uint8_t* __restrict__ packed, 
     }
 }
 
+// scale_mode 1: the free scale of every residual step, s_extra[row, G, level]
+__global__ void unpack_scales_kernel(PackLayout L, const uint8_t* __restrict__ packed, float* __restrict__ s_extra) {
+    const int n_lv = L.top - L.b1;
+    const long long n = (long long)L.rows * L.n_groups * n_lv;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int l = (int)(idx % n_lv);
+        const long long rg = idx / n_lv;
+        const int G = (int)(rg % L.n_groups), row = (int)(rg / L.n_groups);
+        const int rt = row / D2MOE_TILE_ROWS, r = row - rt * D2MOE_TILE_ROWS;
+        const uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
+        s_extra[idx] = __half2float(*reinterpret_cast<const __half*>(blk + d2moe_level_offset(L, l, r)));
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_unpack_scales(const PackLayout& L, const uint8_t* packed, float* s_extra, cudaStream_t st) {
+    const long long n = (long long)L.rows * L.n_groups * (L.top - L.b1);
+    if (n == 0) return cudaSuccess;
+    int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+    unpack_scales_kernel<<<blocks, 256, 0, st>>>(L, packed, s_extra);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const float* W, uint8_t* packed,
                         cudaStream_t st) {

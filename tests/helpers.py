@@ -34,9 +34,9 @@ def gpu_layer(binding, cfg, wl, layer: int = 0, device="cuda"):
 class OracleLayer:
     """Oracle-side experts, quantized lazily from the same seeded weights (CPU)."""
 
-    def __init__(self, wl, layer: int = 0):
+    def __init__(self, wl, layer: int = 0, scale_mode: int = 0):
         from oracle import mwq
-        self.wl, self.layer, self._mwq = wl, layer, mwq
+        self.wl, self.layer, self._mwq, self.scale_mode = wl, layer, mwq, scale_mode
         self.cache = {}
         self.raw_cache = {}
 
@@ -47,7 +47,8 @@ class OracleLayer:
 
     def __call__(self, e: int):
         if e not in self.cache:
-            self.cache[e] = tuple(self._mwq.quantize(W, self.wl.bits, self.wl.group_size) for W in self.raw(e))
+            self.cache[e] = tuple(self._mwq.quantize(W, self.wl.bits, self.wl.group_size, self.scale_mode)
+                                  for W in self.raw(e))
             self.raw_cache.pop(e, None)
         return self.cache[e]
 
@@ -104,7 +105,7 @@ def oracle_threads() -> int:
 
 
 def oracle_sampled(wl, jobs: Sequence[Tuple[np.ndarray, object, Iterable[int]]], layer: int = 0,
-                   gen_device: str = "cpu", n_threads: Optional[int] = None) -> List[Dict[int, np.ndarray]]:
+                   gen_device: str = "cpu", n_threads: Optional[int] = None, scale_mode: int = 0) -> List[Dict[int, np.ndarray]]:
     """Oracle layer outputs for token samples of several batches that share one layer's weights.
 
     jobs: (x fp32 [T, d] bf16-exact, oracle Routing of that batch, tokens wanted).  Returns one
@@ -131,7 +132,7 @@ def oracle_sampled(wl, jobs: Sequence[Tuple[np.ndarray, object, Iterable[int]]],
     part: Dict[Tuple[int, int, int], np.ndarray] = {}       # (job, token, slot or -1-shared) -> weighted expert output
 
     def expert_task(e: int, raw):
-        triple = tuple(mwq.quantize(W, wl.bits, wl.group_size) for W in raw)
+        triple = tuple(mwq.quantize(W, wl.bits, wl.group_size, scale_mode) for W in raw)
         del raw
         rows = rows_of[e]
         xs = np.stack([jobs[j][0][t] for j, t, _ in rows])

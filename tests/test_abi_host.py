@@ -49,7 +49,8 @@ def test_status_strings(lib):
     (lambda c: setattr(c, "group_size", 48), 2),
     (lambda c: setattr(c, "group_size", 128), 0),
     (lambda c: setattr(c, "d_model", 200), 2),
-    (lambda c: setattr(c, "scale_mode", 1), 4),
+    (lambda c: setattr(c, "scale_mode", 1), 0),
+    (lambda c: setattr(c, "scale_mode", 2), 2),
     (lambda c: setattr(c, "renormalize", 2), 2),
     (lambda c: setattr(c, "kernel_path", 7), 2),
     (lambda c: setattr(c, "n_experts", 300), 2),
@@ -76,6 +77,10 @@ def test_packed_bytes_is_the_top_width_only(lib):
     assert binding.packed_bytes(good(), 100, 256)[1] == 128 * 256
     with pytest.raises(binding.D2MoEError):
         binding.packed_bytes(good(), 64, 100)
+    # free residual scales: the same code bytes, six more fp16 scales per (row, group)
+    free = binding.Config(256, 512, 4, 2, 64, (2, 3, 4, 8), scale_mode=1)
+    t1, c1, m1 = binding.packed_bytes(free, rows, cols)
+    assert c1 == code and m1 == rows * (cols // 64) * (4 + 2 * 6) and t1 == 256 + c1 + m1
 
 
 def test_null_and_short_buffers_are_rejected_before_launch(lib):

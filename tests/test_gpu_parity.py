@@ -299,13 +299,13 @@ def test_mixtral_prefill_tensor_path_matches_cuda_core_path(B, mixtral_blobs):
 
 # ------------------------------------------------------------------ other width lists, group sizes, loads
 def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=21, one_expert=False,
-                     token_scales=None, outlier=None):
+                     token_scales=None, outlier=None, scale_mode=0):
     """Random small layer through the tensor-core path, the CUDA-core path and the oracle."""
     _, routing, moe = oracle_mods()
     from oracle import mwq
     K = len(bits)
-    cfg_tc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=0)
-    cfg_cc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=1)
+    cfg_tc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=0, scale_mode=scale_mode)
+    cfg_cc = B.Config(d, F, E, k, g, tuple(bits), n_shared=n_shared, kernel_path=1, scale_mode=scale_mode)
     raw = {}
     blobs = []
     for e in range(E + n_shared):
@@ -339,7 +339,7 @@ def small_layer_case(B, *, d, F, E, k, g, bits, T, n_shared=0, probs=None, seed=
 
     def get(e):
         if e not in packed:
-            packed[e] = tuple(mwq.quantize(W, bits, g) for W in raw[e])
+            packed[e] = tuple(mwq.quantize(W, bits, g, scale_mode) for W in raw[e])
         return packed[e]
 
     toks = sorted(set([0, T // 2, T - 1]))
@@ -557,3 +557,33 @@ def test_bad_index_in_supplied_routing_is_flagged_and_skipped(B, T):
     torch.cuda.synchronize()
     assert int(st.item()) & B.DEV_BAD_INDEX
     assert torch.equal(y, y_ref)
+
+
+# ------------------------------------------------------------------ free per-step residual scales (scale_mode 1)
+@pytest.mark.parametrize("bits,g,rows,cols", [((2, 3, 4, 8), 128, 256, 512), ((2, 4, 8), 64, 130, 256), ((2, 8), 32, 64, 96),
+                                              ((1, 2, 3, 4, 5, 6, 7, 8), 256, 64, 512), ((3, 5), 64, 100, 128), ((4, 8), 128, 192, 1408)])
+def test_pack_free_scales_bit_exact(B, bits, g, rows, cols):
+    # codes, base scale / offset and every per-step scale of Eq. 4 / Eq. 5 against the oracle, bit for bit
+    mwq, _, _ = oracle_mods()
+    cfg = B.Config(cols, cols, 2, 1, g, bits, scale_mode=1)
+    W = synth.normal(12, 5, (rows, cols), 0.02, "cuda")
+    blob = B.pack_mwq(cfg, W)
+    q = mwq.quantize(np_f32(W), bits, g, scale_mode=1)
+    for b in range(bits[0], bits[-1] + 1):
+        codes, s1, lo = B.unpack_codes(cfg, blob, rows, cols, b)
+        assert np.array_equal(codes.cpu().numpy(), mwq.slice_code(q, b)), f"width {b}"
+    assert np.array_equal(np_f32(s1), q.s1) and np.array_equal(np_f32(lo), q.lo)
+    assert np.array_equal(np_f32(B.unpack_scales(cfg, blob, rows, cols)), q.s_extra)
+
+
+@pytest.mark.parametrize("case", [
+    dict(d=256, F=384, E=4, k=2, g=128, bits=(2, 3, 4, 8), T=24),                      # decode-sized: grouped GEMM all the same
+    dict(d=256, F=256, E=2, k=1, g=128, bits=(2, 3, 4, 8), T=400, probs=[0.1, 0.2, 0.4, 0.3]),
+    dict(d=256, F=384, E=4, k=2, g=64, bits=(2, 4, 8), T=50, n_shared=1),
+    dict(d=256, F=256, E=2, k=2, g=128, bits=(1, 2, 3, 4, 5, 6, 7, 8), T=300),
+    dict(d=128, F=128, E=2, k=1, g=64, bits=(3, 5), T=7),
+    dict(d=192, F=256, E=3, k=2, g=64, bits=(2, 8), T=9),                              # CUDA-core path only (d % 128 != 0)
+])
+def test_free_scales_layer_against_oracle(B, case):
+    cross, err = small_layer_case(B, scale_mode=1, **case)
+    assert cross < TOL and err < TOL, (cross, err)

@@ -193,3 +193,42 @@ def test_stack_all_layers_against_oracle_and_graph_replay(B):
     assert len(widths_seen) > 1
     for l, (mn, el, ce, _) in enumerate(res):
         assert mn < TOL and el <= 1.0 and ce < TOL, (l, mn, el, ce)
+
+
+def test_mixtral_free_scales_decode_and_prefill_against_oracle_sample(B):
+    """Free per-step residual scales (Eq. 4 / Eq. 5, scale_mode 1) at full size: the Mixtral-shaped layer repacked
+    with one scale per extra bit, a 64-token decode batch and the 2048-token prefill batch (both on the grouped
+    dequant-GEMM, which folds the codes in bit by bit), against the oracle on group-edge token samples."""
+    wl = synth.WORKLOADS["mixtral_decode"]
+    wlp = synth.WORKLOADS["mixtral_prefill"]
+    cfg = B.Config.from_workload(wl, scale_mode=1)
+    blobs = gpu_layer(B, cfg, wl)
+    gw = synth.gate_weight_bf16(wl, "cuda")
+    jobs, ys, names = [], [], []
+    T = 64
+    x = synth.tokens_bf16(wl, T, "cuda")
+    fb = synth.forced_bit_idx(wl, T, "cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = B.moe_forward(cfg, x, blobs, gate_w=gw, forced_bit_idx=fb, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    rt = oracle_route(wl, x, gate_w=gw, forced=fb)
+    jobs.append((np_f32(x), rt, group_edge_tokens(rt, wl.top_k)[::2]))
+    ys.append(np_f32(y)); names.append("mixtral_decode T=64 free scales")
+    T = 2048
+    x = synth.tokens_bf16(wlp, T, "cuda")
+    fb = synth.forced_bit_idx(wlp, T, "cuda")
+    lg = synth.zipf_logits(wlp, T, "cuda")
+    y = B.moe_forward(B.Config.from_workload(wlp, scale_mode=1), x, blobs, logits=lg, forced_bit_idx=fb, device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    rt = oracle_route(wlp, x, logits=lg, forced=fb)
+    jobs.append((np_f32(x), rt, group_edge_tokens(rt, wlp.top_k)))
+    ys.append(np_f32(y)); names.append("mixtral_prefill T=2048 free scales")
+    del blobs
+    torch.cuda.empty_cache()
+    refs = oracle_sampled(wl, jobs, gen_device="cuda", scale_mode=1)
+    for name, yg, ref in zip(names, ys, refs):
+        mn, el = check_rows(yg, ref, TOL)
+        report(name, tokens_checked=len(ref), max_norm_rel_err=mn, elementwise_excess=el)
+        assert mn < TOL and el <= 1.0, (name, mn, el)
