@@ -58,11 +58,13 @@ def measured_peaks():
 # packed prefix up to the widest width routed to that expert in this call, read once, plus activations
 # in and outputs out
 # ------------------------------------------------------------------------------------------------
-def matrix_bytes(rows, cols, g, bits_read):
-    return rows * cols * bits_read // 8 + rows * (cols // g) * 4
+def matrix_bytes(rows, cols, g, bits_read, scale_steps=0):
+    """codes at the width read + (fp16 scale, fp16 offset) per row and group (+ one fp16 scale per extra bit read
+    when the residual scales are free)."""
+    return rows * cols * bits_read // 8 + rows * (cols // g) * (4 + 2 * scale_steps)
 
 
-def algorithmic_bytes(wl, T, group_off):
+def algorithmic_bytes(wl, T, group_off, scale_mode=0):
     """Bytes per layer call from the realised routing: every plane of an active expert up to the
     largest width routed to it is read once; plus activations in/out and the h round trip."""
     K = len(wl.bits)
@@ -78,8 +80,9 @@ def algorithmic_bytes(wl, T, group_off):
         else:
             b = wl.bits[-1]
         active += 1
-        gu += 2 * matrix_bytes(wl.d_ffn, wl.d_model, wl.group_size, b)
-        dn += matrix_bytes(wl.d_model, wl.d_ffn, wl.group_size, b)
+        steps = b - wl.bits[0] if scale_mode == 1 else 0
+        gu += 2 * matrix_bytes(wl.d_ffn, wl.d_model, wl.group_size, b, steps)
+        dn += matrix_bytes(wl.d_model, wl.d_ffn, wl.group_size, b, steps)
     A_tot = T * (wl.top_k + wl.n_shared)
     io_gu = A_tot * wl.d_model * 2 + A_tot * wl.d_ffn * 2       # gathered x in, h out (16-bit)
     io_dn = A_tot * wl.d_ffn * 2 + A_tot * wl.d_model * 4       # h in, expert outputs out (fp32)
@@ -307,10 +310,10 @@ class LayerBench:
 
     N_BATCHES = 4
 
-    def __init__(self, B, wl, T, path_name, dev, rank=0, blobs=None):
-        self.B, self.wl, self.T, self.dev, self.path_name = B, wl, T, dev, path_name
+    def __init__(self, B, wl, T, path_name, dev, rank=0, blobs=None, scale_mode=0):
+        self.B, self.wl, self.T, self.dev, self.path_name, self.scale_mode = B, wl, T, dev, path_name, scale_mode
         path = {"auto": B.PATH_AUTO, "cuda_core": B.PATH_CUDA_CORE, "tensor": B.PATH_TENSOR}[path_name]
-        self.cfg = B.Config.from_workload(wl, kernel_path=path)
+        self.cfg = B.Config.from_workload(wl, kernel_path=path, scale_mode=scale_mode)
         if blobs is None:
             blobs = []
             for e in range(wl.n_experts + wl.n_shared):
@@ -332,13 +335,13 @@ class LayerBench:
         for i in range(nb):
             r = B.route(self.cfg, self.xs[i], workspace=self.ws, **self.kw(i))
             torch.cuda.synchronize()
-            self.alg.append(algorithmic_bytes(wl, T, r.group_off.cpu().tolist()))
+            self.alg.append(algorithmic_bytes(wl, T, r.group_off.cpu().tolist(), scale_mode))
         self.layer_bytes = sum(a["layer"] for a in self.alg) / nb
         # a step that streams less than a few L2 sizes could be served partly from L2 by the step before it:
         # such workloads are timed step by step with an L2 flush (a 256 MiB write) between the steps
         self.flush = self.layer_bytes < 4 * L2_BYTES
         self.flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if self.flush else None
-        self.decode = -(-T * wl.top_k // wl.n_experts) <= 40
+        self.decode = -(-T * wl.top_k // wl.n_experts) <= 40 and scale_mode == 0
 
     def kw(self, i, fb=None):
         d = {"forced_bit_idx": self.fbs[i] if fb is None else fb}
@@ -410,7 +413,10 @@ class LayerBench:
                         "achieved_gbs": layer_bytes / (ms_per_step * 1e-3) / 1e9,
                         "frac": layer_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
         dtype = "f32" if self.path_name == "cuda_core" else "i8"
-        if not self.decode and self.path_name != "cuda_core":
+        small_load = -(-T * wl.top_k // wl.n_experts) <= 40       # decode-sized: bound by the bytes whichever kernel runs
+        if self.scale_mode == 1 and small_load and self.path_name != "cuda_core":
+            dtype = "f16"
+        if not self.decode and not small_load and self.path_name != "cuda_core":
             # prefill-sized expert loads (the grouped dequant-GEMM) are bound by the tensor cores: the dominant
             # kernel against the measured dense 16-bit matmul rates (fp16 operands have the nominal rate of the
             # bf16 the peaks were measured with); both the burst and the sustained (power-capped) figure
@@ -457,10 +463,10 @@ def workload_config(wl, T, path, l2=None):
             "tokens_per_step": T, "kernel_path": path, "l2": l2 or "inputs larger than L2"}
 
 
-def short_leg(B, wl, T, dev, blobs=None, steps=20, min_s=0.25):
+def short_leg(B, wl, T, dev, blobs=None, steps=20, min_s=0.25, scale_mode=0):
     """A short device-timed leg of another configuration (same rules: warm-up, regions of `steps` steps,
     clocks sampled during the regions, stages from a separate pass)."""
-    lb = LayerBench(B, wl, T, "auto", dev, blobs=blobs)
+    lb = LayerBench(B, wl, T, "auto", dev, blobs=blobs, scale_mode=scale_mode)
     for i in range(3):
         lb.step(i)
     torch.cuda.synchronize()
@@ -472,7 +478,9 @@ def short_leg(B, wl, T, dev, blobs=None, steps=20, min_s=0.25):
     ms = median(regions) / steps
     stage_ms, used = lb.stage_pass(8)
     rf, dtype = lb.roofline(stage_ms, used, ms, clocks)
-    return {"workload": workload_config(wl, T, "auto", lb.l2_note())["workload"], "tokens_per_step": T,
+    return {"workload": workload_config(wl, T, "auto", lb.l2_note())["workload"]
+                        + (" free per-step residual scales (scale_mode 1)" if scale_mode else ""),
+            "blobs": lb.blobs, "tokens_per_step": T,
             "ms_per_step": ms, "tokens_per_s": T / (ms * 1e-3), "dtype": dtype, "regions": len(regions),
             "timed_region_s": sum(regions) * 1e-3, "l2": lb.l2_note(), "clocks": clocks, "roofline": rf}
 
@@ -644,7 +652,7 @@ def run_ours(args):
 
     wl = synth.WORKLOADS[args.workload]
     T = args.tokens or synth.WORKLOADS[args.workload].tokens[-1]
-    lb = LayerBench(B, wl, T, args.path, dev, rank=rank)
+    lb = LayerBench(B, wl, T, args.path, dev, rank=rank, scale_mode=args.scale_mode)
     stream = torch.cuda.current_stream()
 
     for i in range(args.warmup):
@@ -737,7 +745,7 @@ def run_ours(args):
 
     # ---- the other configurations, short legs in the same invocation (one GPU only) ----
     others = None
-    if world == 1 and args.others and args.workload == "mixtral_decode" and args.path == "auto":
+    if world == 1 and args.others and args.workload == "mixtral_decode" and args.path == "auto" and args.scale_mode == 0:
         others = []
         for t in wl.tokens:
             if t != T:
@@ -746,6 +754,12 @@ def run_ours(args):
         others.append(short_leg(B, wlp, wlp.tokens[-1], dev, blobs=lb.blobs, steps=10))
         wlf = synth.WORKLOADS["finegrained"]
         others.append(short_leg(B, wlf, wlf.tokens[-1], dev))
+        # the same Mixtral-shaped layer with free per-step residual scales (Eq. 4 / Eq. 5): repacked, both batch sizes
+        leg = short_leg(B, wl, T, dev, scale_mode=1)
+        others.append(leg)
+        others.append(short_leg(B, wlp, wlp.tokens[-1], dev, blobs=leg["blobs"], steps=10, scale_mode=1))
+        for o in others:
+            o.pop("blobs", None)
         torch.cuda.empty_cache()
         if args.others == "all":
             wls = synth.WORKLOADS["mixtral_stack"]
@@ -755,7 +769,7 @@ def run_ours(args):
                            "timed_region_s": sum(r["regions"]) * 1e-3, "l2": r["l2"], "clocks": r["clocks"],
                            "cuda_graph": r["graph"], "roofline": r["roofline"]})
 
-    cfg_T = B.Config.from_workload(wl)
+    cfg_T = B.Config.from_workload(wl, scale_mode=args.scale_mode)
     line = {"metric": METRIC, "value": job_tokens_per_s(T, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype,
@@ -825,6 +839,8 @@ def main():
                     help="mixtral_stack only: layers per step (default: the workload's 32; 46 GB of packed experts)")
     ap.add_argument("--no-graph", action="store_true", help="mixtral_stack only: launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scale-mode", type=int, default=0, choices=[0, 1],
+                    help="0: tied residual scales; 1: free per-step scales (Eq. 4 / Eq. 5)")
     ap.add_argument("--min-region-s", type=float, default=1.0,
                     help="repeat the timed K-step region until this much device time has been timed")
     ap.add_argument("--others", default="all", choices=["all", "layers", "none"],
