@@ -261,6 +261,59 @@ d2moe_status d2moe_stack_layer(const d2moe_config* cfg, int64_t T, void* x_bf16,
  */
 d2moe_status d2moe_selftest_wait_expiry(int which, int32_t* device_status, void* stream);
 
+/*
+ * ---- Host-side planning of the bit-width-aware I/O-compute pipeline (Section 3.4) ----
+ * For deployments where the experts do not all stay in GPU memory (on one B200 they do; the layer kernels
+ * above never need this).  Plain host functions: no kernel, no device memory, every array is the caller's.
+ *
+ * With the nested store an expert is loaded segment by segment: segment k holds what width bits[k] adds
+ * to width bits[k-1]; a request at width index k reads segments 0..k.  B is the host matrix B_{j,k} of
+ * Section 3.4.3, row-major [n_experts][n_bits]: requests of expert j at width index k in this layer (the
+ * histogram of d2moe_route's group_off).
+ */
+typedef struct { int32_t expert, segment; } d2moe_plan_item;
+#define D2MOE_PLAN_HEBF  0   /* Hottest-Expert-Bit-First */
+#define D2MOE_PLAN_BY_ID 1   /* sequential baseline: ascending expert id, ascending width */
+
+/*
+ * Load order of the segments one layer needs (for every expert with a request: segments 0..its largest
+ * requested width index).  D2MOE_PLAN_HEBF (Section 3.4.3, "Solution"): one queue per expert in ascending
+ * width; the head with the highest frequency is taken next, frequency of (j, k) = requests that read
+ * segment k of expert j = sum over k' >= k of B[j][k'], ties to the lower expert id.  Every expert's
+ * segments appear in ascending width (constraint 6b).  queue: caller array of `capacity` items
+ * (n_experts * n_bits always suffices; D2MOE_ERR_WORKSPACE if too small); *n_items receives the length.
+ */
+d2moe_status d2moe_plan_load_order(int32_t n_experts, int32_t n_bits, const int32_t* B, int32_t policy,
+                                   d2moe_plan_item* queue, int32_t capacity, int32_t* n_items);
+
+/*
+ * The two-queue pipeline of Eq. 6 for a given load order: loads run back to back, item s taking
+ * t_io[segment]; the compute of item s (its B[j][k] requests, t_comp[k] each) starts when both its load
+ * (constraint 6a) and the compute of item s-1 have finished; the time the compute queue stood idle is
+ * T_wait (constraint 6c).  t_io, t_comp: host double [n_bits] (the offline profile of Section 3.4.2).
+ * *makespan: when both queues are done; *wait (may be NULL): summed T_wait.  An order that loads a
+ * segment before the one below it is rejected (D2MOE_ERR_SHAPE).
+ */
+d2moe_status d2moe_plan_simulate(int32_t n_experts, int32_t n_bits, const int32_t* B,
+                                 const d2moe_plan_item* queue, int32_t n_items, const double* t_io,
+                                 const double* t_comp, double* makespan, double* wait);
+
+/*
+ * One layer step of the memory-budget scheduler (Algorithm 2).  `resident`: segments now in GPU memory,
+ * `need`: segments the coming layer needs, `budget`: M in bytes.  Needed segments that are resident stay;
+ * the others are loaded after enough other segments have been released - highest width first, then the
+ * oldest layer, then the lowest expert id ("high bit-width expert weights are released ... low bit-width
+ * weights are also released as needed").  Outputs (caller arrays of `capacity` entries each): the new
+ * resident list, the loads and the releases.  D2MOE_ERR_WORKSPACE if the layer's own segments exceed the
+ * budget or an output array is too small.
+ */
+typedef struct { int32_t layer, expert, segment, reserved; int64_t bytes; } d2moe_segment;
+d2moe_status d2moe_plan_budget_step(const d2moe_segment* resident, int32_t n_resident,
+                                    const d2moe_segment* need, int32_t n_need, int64_t budget,
+                                    d2moe_segment* new_resident, int32_t* n_new,
+                                    d2moe_segment* loads, int32_t* n_loads,
+                                    d2moe_segment* evictions, int32_t* n_evictions, int32_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

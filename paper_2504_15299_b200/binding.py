@@ -35,6 +35,15 @@ class _Config(ctypes.Structure):
                 ("kernel_path", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
+class _PlanItem(ctypes.Structure):
+    _fields_ = [("expert", ctypes.c_int32), ("segment", ctypes.c_int32)]
+
+
+class _Segment(ctypes.Structure):
+    _fields_ = [("layer", ctypes.c_int32), ("expert", ctypes.c_int32), ("segment", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("bytes", ctypes.c_int64)]
+
+
 class _RouteIn(ctypes.Structure):
     _fields_ = [("gate_w_bf16", ctypes.c_void_p), ("logits", ctypes.c_void_p),
                 ("bit_w_bf16", ctypes.c_void_p), ("forced_bit_idx", ctypes.c_void_p)]
@@ -50,7 +59,7 @@ _lib = None
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
            "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count",
-           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry", "d2moe_unpack_scales"]
+           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry", "d2moe_unpack_scales", "d2moe_plan_load_order", "d2moe_plan_simulate", "d2moe_plan_budget_step"]
 
 
 def lib() -> ctypes.CDLL:
@@ -70,6 +79,14 @@ def lib() -> ctypes.CDLL:
     L.d2moe_pack_mwq.argtypes = [cfgp, vp, i64, i64, vp, sz, vp]
     L.d2moe_unpack_codes.argtypes = [cfgp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
     L.d2moe_unpack_scales.argtypes = [cfgp, vp, i64, i64, vp, vp]
+    i32p, dp = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double)
+    L.d2moe_plan_load_order.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, ctypes.c_int32, ctypes.POINTER(_PlanItem),
+                                        ctypes.c_int32, i32p]
+    L.d2moe_plan_simulate.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, ctypes.POINTER(_PlanItem), ctypes.c_int32, dp, dp,
+                                      dp, dp]
+    segp = ctypes.POINTER(_Segment)
+    L.d2moe_plan_budget_step.argtypes = [segp, ctypes.c_int32, segp, ctypes.c_int32, ctypes.c_int64, segp, i32p, segp, i32p,
+                                         segp, i32p, ctypes.c_int32]
     L.d2moe_workspace_bytes.restype = sz
     L.d2moe_workspace_bytes.argtypes = [cfgp, i64]
     L.d2moe_route.argtypes = [cfgp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -314,3 +331,43 @@ def stack_layer(cfg: Config, x: torch.Tensor, xn: torch.Tensor, expert_w: Sequen
                                    _expert_ptr_array(expert_w), ctypes.byref(rin), _ptr(device_status),
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "d2moe_stack_layer")
     return x
+
+
+# ---- host-side pipeline planning (Section 3.4): marshalling of plain Python lists ----
+PLAN_HEBF, PLAN_BY_ID = 0, 1
+
+
+def _flat_B(B):
+    E, K = len(B), len(B[0])
+    arr = (ctypes.c_int32 * (E * K))(*[int(v) for row in B for v in row])
+    return E, K, arr
+
+
+def plan_load_order(B, policy: int = PLAN_HEBF) -> List[Tuple[int, int]]:
+    E, K, arr = _flat_B(B)
+    q = (_PlanItem * (E * K))()
+    n = ctypes.c_int32()
+    _check(lib().d2moe_plan_load_order(E, K, arr, policy, q, E * K, ctypes.byref(n)), "d2moe_plan_load_order")
+    return [(q[i].expert, q[i].segment) for i in range(n.value)]
+
+
+def plan_simulate(B, order: Sequence[Tuple[int, int]], t_io: Sequence[float], t_comp: Sequence[float]) -> Tuple[float, float]:
+    E, K, arr = _flat_B(B)
+    q = (_PlanItem * max(len(order), 1))(*[_PlanItem(j, k) for j, k in order])
+    io, comp = (ctypes.c_double * K)(*t_io), (ctypes.c_double * K)(*t_comp)
+    span, wait = ctypes.c_double(), ctypes.c_double()
+    _check(lib().d2moe_plan_simulate(E, K, arr, q, len(order), io, comp, ctypes.byref(span), ctypes.byref(wait)),
+           "d2moe_plan_simulate")
+    return span.value, wait.value
+
+
+def plan_budget_step(resident, need, budget: int):
+    """resident / need: lists of (layer, expert, segment, bytes); returns (new resident, loads, evictions)."""
+    cap = len(resident) + len(need) + 1
+    mk = lambda v: (_Segment * max(len(v), 1))(*[_Segment(l, e, k, 0, b) for l, e, k, b in v])
+    out = [(_Segment * cap)() for _ in range(3)]
+    ns = [ctypes.c_int32() for _ in range(3)]
+    _check(lib().d2moe_plan_budget_step(mk(resident), len(resident), mk(need), len(need), budget, out[0], ctypes.byref(ns[0]),
+                                        out[1], ctypes.byref(ns[1]), out[2], ctypes.byref(ns[2]), cap), "d2moe_plan_budget_step")
+    conv = lambda a, n: [(a[i].layer, a[i].expert, a[i].segment, a[i].bytes) for i in range(n.value)]
+    return conv(out[0], ns[0]), conv(out[1], ns[1]), conv(out[2], ns[2])

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2moe.so")
-SOURCES = ["d2moe_api.cu", "kernels_pack.cu", "kernels_route.cu", "kernels_ffn_cc.cu", "kernels_ffn_tc.cu", "kernels_ffn_i8.cu"]
+SOURCES = ["d2moe_api.cu", "kernels_pack.cu", "kernels_route.cu", "kernels_ffn_cc.cu", "kernels_ffn_tc.cu", "kernels_ffn_i8.cu", "planner.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 
