@@ -83,8 +83,8 @@ d2moe_status d2moe_check_config(const d2moe_config* cfg);
 /*
  * Size in bytes of the packed form of one [rows, cols] matrix (cols % group_size == 0).
  * total = header + code bytes + metadata bytes; code_bytes and meta_bytes (either may be NULL) give
- * the split: code_bytes = rows_padded*cols*bits[n_bits-1]/8 when every segment width is 1, 2, 4 or 8
- * bits (segments of 3 / 5..7 bits are stored in 4 / 8), metadata = one (fp16 scale, fp16 offset)
+ * the split: code_bytes = rows_padded*cols*bits[n_bits-1]/8 for every width list (a width step of 3, 5,
+ * 6 or 7 bits is stored as fields of 2+1, 4+1, 4+2, 4+2+1 bits), metadata = one (fp16 scale, fp16 offset)
  * pair per row and group, plus, with scale_mode 1, one fp16 scale per extra bit (bits[n_bits-1] -
  * bits[0] of them) per row and group.  The nested store costs the top width only, whatever n_bits is.
  */

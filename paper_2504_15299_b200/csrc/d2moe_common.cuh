@@ -43,16 +43,20 @@
 // ------------------------------------------------------------------------------------------------
 struct PackLayout {
     int rows, cols, g, n_groups, rows_pad, n_rt;
-    int n_seg, top, b1;
-    int seg_w[D2MOE_MAX_SEG];      // logical width of segment j
-    int seg_sw[D2MOE_MAX_SEG];     // storage width (1, 2, 4, 8)
+    int n_seg, top, b1;            // n_seg: stored segments (a width step of 3, 5, 6 or 7 bits is stored as 2+1, 4+1, 4+2, 4+2+1)
+    int seg_w[D2MOE_MAX_SEG];      // width of stored segment j: 1, 2, 4 or 8 bits
+    int seg_sw[D2MOE_MAX_SEG];     // storage width (= seg_w)
     int seg_shift[D2MOE_MAX_SEG];  // position of the segment inside the top-width code
     int seg_cs[D2MOE_MAX_SEG];     // chunk size in bytes
     int seg_off[D2MOE_MAX_SEG + 1];// byte offset of segment j inside a block; [n_seg] = block size
+    int seg_kk[D2MOE_MAX_SEG];     // width index whose step the segment belongs to
+    int n_widths;                  // number of listed widths
+    int last_seg[D2MOE_MAX_SEG];   // width index kk -> its last stored segment (a call at bits[kk] reads segments 0..last_seg[kk])
     int block_bytes;
     int scale_mode;                // 0 tied residual scales, 1 free (one fp16 scale per row, group and extra bit)
-    int seg_sc_off[D2MOE_MAX_SEG]; // scale_mode 1: byte offset of the scales of segment j (j >= 1) inside a block
-    int seg_lv0[D2MOE_MAX_SEG];    // first residual step (0-based) that segment j adds; it adds seg_w[j] steps (j >= 1)
+    int w_sc_off[D2MOE_MAX_SEG];   // scale_mode 1: byte offset of the scales of width step kk (kk >= 1) inside a block
+    int w_lv0[D2MOE_MAX_SEG];      // first residual step (0-based) of width step kk; it has bits[kk] - bits[kk-1] steps
+    int w_end[D2MOE_MAX_SEG];      // end of what a call at width index kk reads (bytes from the start of the block)
 };
 
 struct PackHeader {
@@ -66,35 +70,44 @@ struct PackHeader {
 };
 static_assert(sizeof(PackHeader) == D2MOE_HEADER_BYTES, "header size");
 
-__host__ __device__ inline int d2moe_storage_width(int w) { return w <= 1 ? 1 : (w <= 2 ? 2 : (w <= 4 ? 4 : 8)); }
-
 __host__ __device__ inline void d2moe_make_layout(PackLayout& L, const int* bits, int n_bits, int g,
                                                   long long rows, long long cols, int scale_mode = 0) {
     L.scale_mode = scale_mode;
     L.rows = (int)rows; L.cols = (int)cols; L.g = g; L.n_groups = (int)(cols / g);
     L.rows_pad = (int)((rows + D2MOE_TILE_ROWS - 1) / D2MOE_TILE_ROWS * D2MOE_TILE_ROWS);
     L.n_rt = L.rows_pad / D2MOE_TILE_ROWS;
-    L.n_seg = n_bits; L.top = bits[n_bits - 1]; L.b1 = bits[0];
-    int off = D2MOE_TILE_ROWS * 4, prev = 0;
+    L.top = bits[n_bits - 1]; L.b1 = bits[0]; L.n_widths = n_bits;
     for (int j = 0; j < D2MOE_MAX_SEG; ++j) {
-        if (j < n_bits) {
-            L.seg_w[j] = bits[j] - prev; prev = bits[j];
-            L.seg_sw[j] = d2moe_storage_width(L.seg_w[j]);
-            L.seg_shift[j] = L.top - bits[j];
-            int row_bytes = g * L.seg_sw[j] / 8;
-            L.seg_cs[j] = row_bytes < 16 ? row_bytes : 16;
-            L.seg_lv0[j] = j == 0 ? 0 : bits[j - 1] - bits[0];
-            L.seg_sc_off[j] = off;
-            if (scale_mode == 1 && j >= 1) off += D2MOE_TILE_ROWS * 2 * L.seg_w[j];
-            L.seg_off[j] = off;
-            off += D2MOE_TILE_ROWS * row_bytes;
-        } else {
-            L.seg_w[j] = L.seg_sw[j] = L.seg_shift[j] = L.seg_cs[j] = 0; L.seg_off[j] = off;
-            L.seg_sc_off[j] = off; L.seg_lv0[j] = 0;
-        }
+        L.seg_w[j] = L.seg_sw[j] = L.seg_shift[j] = L.seg_cs[j] = L.seg_kk[j] = 0;
+        L.last_seg[j] = 0; L.w_sc_off[j] = L.w_lv0[j] = L.w_end[j] = 0;
     }
-    L.seg_off[n_bits < D2MOE_MAX_SEG ? n_bits : D2MOE_MAX_SEG] = off;
-    if (n_bits == D2MOE_MAX_SEG) L.seg_off[D2MOE_MAX_SEG] = off;
+    int off = D2MOE_TILE_ROWS * 4, prev = 0, n = 0;
+    for (int kk = 0; kk < n_bits; ++kk) {
+        int w = bits[kk] - prev;                       // the step of this width: stored as power-of-two sub-fields, widest first
+        L.w_lv0[kk] = kk == 0 ? 0 : prev - bits[0];
+        L.w_sc_off[kk] = off;
+        if (scale_mode == 1 && kk >= 1) off += D2MOE_TILE_ROWS * 2 * w;
+        int pos = bits[kk] - prev;                     // bits of the step not yet stored
+        for (int f = 8; f >= 1; f >>= 1) {
+            if (pos >= f && n < D2MOE_MAX_SEG) {
+                pos -= f;
+                L.seg_w[n] = L.seg_sw[n] = f;
+                L.seg_shift[n] = L.top - bits[kk] + pos;
+                const int row_bytes = g * f / 8;
+                L.seg_cs[n] = row_bytes < 16 ? row_bytes : 16;
+                L.seg_off[n] = off;
+                L.seg_kk[n] = kk;
+                off += D2MOE_TILE_ROWS * row_bytes;
+                ++n;
+            }
+        }
+        L.last_seg[kk] = n - 1;
+        L.w_end[kk] = off;
+        prev = bits[kk];
+        (void)w;
+    }
+    L.n_seg = n;
+    for (int j = n; j <= D2MOE_MAX_SEG; ++j) L.seg_off[j] = off;
     L.block_bytes = off;
 }
 
@@ -113,15 +126,13 @@ __host__ __device__ inline int d2moe_elem_word(const PackLayout& L, int j, int r
 
 // scale_mode 1: byte offset (inside a block) of the fp16 scale of residual step `level` (0-based) of row r
 __host__ __device__ inline int d2moe_level_offset(const PackLayout& L, int level, int r) {
-    int j = 1;
-    while (j + 1 < L.n_seg && L.seg_lv0[j + 1] <= level) ++j;
-    return L.seg_sc_off[j] + ((level - L.seg_lv0[j]) * D2MOE_TILE_ROWS + r) * 2;
+    int kk = 1;
+    while (kk + 1 < L.n_widths && L.w_lv0[kk + 1] <= level) ++kk;
+    return L.w_sc_off[kk] + ((level - L.w_lv0[kk]) * D2MOE_TILE_ROWS + r) * 2;
 }
 
-// bytes of a block that a call at width index kk reads: meta and segments 0..kk (with their scales)
-__host__ __device__ inline int d2moe_prefix_bytes(const PackLayout& L, int kk) {
-    return kk + 1 < L.n_seg ? L.seg_sc_off[kk + 1] : L.block_bytes;
-}
+// bytes of a block that a call at width index kk reads: meta and the segments (with their scales) of widths 0..kk
+__host__ __device__ inline int d2moe_prefix_bytes(const PackLayout& L, int kk) { return L.w_end[kk]; }
 
 __host__ __device__ inline size_t d2moe_block_offset(const PackLayout& L, int rt, int G) {
     return (size_t)D2MOE_HEADER_BYTES + ((size_t)rt * L.n_groups + G) * (size_t)L.block_bytes;

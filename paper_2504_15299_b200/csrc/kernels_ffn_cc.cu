@@ -37,7 +37,8 @@ template <typename VT>
 __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed, int row, int kk,
                          const VT* __restrict__ v, int lane) {
     const int rt = row / D2MOE_TILE_ROWS, r = row - rt * D2MOE_TILE_ROWS;
-    const int b = L.seg_shift[kk];                      // top - bits[kk]
+    const int last = L.last_seg[kk];                    // the call reads stored segments 0..last
+    const int b = L.seg_shift[last];                    // top - bits[kk]
     const int width = L.top - b;
     const float inv = 1.0f / (float)(1 << (width - L.b1));
     float acc = 0.0f;
@@ -58,7 +59,7 @@ __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed
         }
         for (int i = lane; i < L.g / 2; i += 32) {      // pair (2i, 2i+1)
             unsigned q0 = 0, q1 = 0;
-            for (int j = 0; j <= kk; ++j) {
+            for (int j = 0; j <= last; ++j) {
                 int bitpos;
                 const int wo = d2moe_elem_word(L, j, r, 2 * i, &bitpos);
                 const uint32_t word = *reinterpret_cast<const uint32_t*>(blk + wo);

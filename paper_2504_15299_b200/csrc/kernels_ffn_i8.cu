@@ -85,6 +85,7 @@ struct I8Params {
 };
 
 struct I8Item { int unit, tile, split, g0, g1; };
+struct I8SegMap { int n_seg; int seg_kk[8]; };   // stored segment -> width index of the step it belongs to
 
 
 __device__ __forceinline__ I8Item i8_item(const I8Params& p, int item) {
@@ -161,6 +162,62 @@ __device__ __forceinline__ void unpack_segment(uint32_t seg, int rr, int W, int 
             const uint32_t moved = sh >= 0 ? (w[q] << (sh & 31)) : (w[q] >> ((-sh) & 31));
             v[i] = moved & mask;
         }
+        tc_st8(taddr + b * 8, v);
+    }
+}
+
+// Eight operand cells (batch b of a row's GS/4 cells) from one stored field of FW bits per code at bit PF of its
+// byte; FIRST: the cells are set, otherwise the field is OR-ed into them (one three-input logic operation).
+template <int GS, int FW, bool FIRST>
+__device__ __forceinline__ void field_batch(uint32_t seg, int rr, int PF, int b, uint32_t (&v)[8]) {
+    constexpr int ROW_BYTES = GS * FW / 8;
+    constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
+    constexpr int CPW = 8 / FW;                              // cells per word
+    constexpr int WPB = FW;                                  // words per batch of 8 cells
+    uint32_t w[WPB];
+    auto addr_of = [&](int m) {                              // shared address of the row's word m
+        const int ob = 4 * m, c = ob / CS, within = ob % CS;
+        return seg + (uint32_t)((c * D2MOE_TILE_ROWS + rr) * CS + within);
+    };
+    if constexpr (WPB == 8) {
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr_of(8 * b)));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(addr_of(8 * b + 4)));
+    } else if constexpr (WPB == 4) {
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr_of(4 * b)));
+    } else if constexpr (WPB == 2) {
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr_of(2 * b)));
+    } else {
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[0]) : "r"(addr_of(b)));
+    }
+    const uint32_t mask = (((1u << FW) - 1u) << PF) * 0x01010101u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int q = i / CPW, u = i % CPW;
+        const int sh = PF - FW * u;
+        const uint32_t moved = sh >= 0 ? (w[q] << (sh & 31)) : (w[q] >> ((-sh) & 31));
+        v[i] = FIRST ? (moved & mask) : ((moved & mask) | v[i]);
+    }
+}
+
+// One width step of W bits (stored as fields of 8, 4, 2, 1 bits, widest first, one after the other in the block) of
+// one row -> GS/4 operand cells with the step's value at bit P of every byte: the fields are merged in registers, so
+// a step is one operand tile whatever its width.
+template <int GS, int W>
+__device__ __forceinline__ void unpack_step(uint32_t seg, int rr, int P, uint32_t taddr) {
+    constexpr int F0 = W >= 8 ? 8 : (W >= 4 ? 4 : (W >= 2 ? 2 : 1));
+    constexpr int R1 = W - F0;
+    constexpr int F1 = R1 >= 4 ? 4 : (R1 >= 2 ? 2 : (R1 >= 1 ? 1 : 0));
+    constexpr int R2 = R1 - F1;
+    constexpr int F2 = R2 >= 2 ? 2 : (R2 >= 1 ? 1 : 0);
+    constexpr int R3 = R2 - F2;                              // 0 or 1
+    constexpr int FB = D2MOE_TILE_ROWS * GS / 8;             // bytes of a one-bit field
+#pragma unroll
+    for (int b = 0; b < GS / 32; ++b) {
+        uint32_t v[8];
+        field_batch<GS, F0, true>(seg, rr, P + R1, b, v);
+        if constexpr (F1 > 0) field_batch<GS, F1, false>(seg + F0 * FB, rr, P + R2, b, v);
+        if constexpr (F2 > 0) field_batch<GS, F2, false>(seg + (F0 + F1) * FB, rr, P + R3, b, v);
+        if constexpr (R3 > 0) field_batch<GS, 1, false>(seg + (F0 + F1 + F2) * FB, rr, P, b, v);
         tc_st8(taddr + b * 8, v);
     }
 }
@@ -326,7 +383,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const I8Item ii = i8_item(p, item);
                 const I8Unit* u = p.units + ii.unit;
                 const int e = u->e, kmax = u->kmax;
-                const uint32_t bytes = (uint32_t)d2moe_prefix_bytes(p.L, kmax);
+                // kmax: the unit's last width step (specialised kernels: a step is one operand) or its last stored segment
+                const uint32_t bytes = (uint32_t)(SWPACK != 0 ? d2moe_prefix_bytes(p.L, kmax) : p.L.seg_off[kmax + 1]);
                 const uint8_t *m0, *m1;
                 if (p.mode == 0) {
                     m0 = p.P.w[3 * e + 0] + d2moe_block_offset(p.L, ii.tile, ii.g0);
@@ -415,7 +473,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         tc_fence_after();
                         const uint32_t d_addr = d_tmem + buf * I8_D_COLS;
 #pragma unroll
-                        for (int hp = 0; hp < (SWPACK != 0 ? 1 : 2); ++hp) {
+                        for (int hp = 0; hp < (SWPACK != 0 ? (I8SegList<SWPACK>::count() + 3) / 4 : 2); ++hp) {
 #pragma unroll
                             for (int wg = 0; wg < 2; ++wg) {
                                 const int j0 = wg + 4 * hp, j1 = j0 + 2;
@@ -591,11 +649,17 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 constexpr int J = decltype(jc)::value;
                                 if constexpr (J < SL::count()) {
                                     if ((J & 1) == wg && J <= kmax) {
-                                        unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J),
-                                                                      a_base + (J >> 1) * 32);
+                                        if constexpr (SL::w(J) == SL::sw(J))
+                                            unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J),
+                                                                          a_base + ((J >> 1) & 1) * 32);
+                                        else
+                                            unpack_step<GS, SL::w(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::pos(J),
+                                                                      a_base + ((J >> 1) & 1) * 32);
                                     }
                                 }
                             };
+                            // a warpgroup hands over up to two tiles at a time: segments wg, wg + 2, then wg + 4, wg + 6
+                            constexpr int NHP = (SL::count() + 3) / 4;
                             if (wg <= kmax) {
                                 handoff_begin();
                                 do_seg(std::integral_constant<int, 0>{});
@@ -606,6 +670,16 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 handoff_end();
                             } else if (pend) {
                                 fold_prefetch(gc - 1);
+                            }
+                            if constexpr (NHP > 1) {
+                                if (wg + 4 <= kmax) {
+                                    handoff_begin();
+                                    do_seg(std::integral_constant<int, 4>{});
+                                    do_seg(std::integral_constant<int, 5>{});
+                                    do_seg(std::integral_constant<int, 6>{});
+                                    do_seg(std::integral_constant<int, 7>{});
+                                    handoff_end();
+                                }
                             }
                         } else {
                             if (wg > kmax && pend) fold_prefetch(gc - 1);
@@ -666,7 +740,8 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints).
 __global__ void __launch_bounds__(256)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
-               int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status) {
+               int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status,
+               I8SegMap sm) {
     extern __shared__ int32_t s_prep[];
     __shared__ int s_total;
     const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
@@ -760,9 +835,9 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
             const int len = min(len_e - start, I8_SLOTS);
             I8Unit u;
             u.e = e; u.slot0 = p0 + start; u.nslots = len; u.kmax = 0; u.nblk = 0;
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < 8; ++j) {          // per stored segment: the slots of the width classes that include it
                 u.blk[j] = 0;
-                u.npad[j] = j < D.K ? max(0, min(len, cpad[j] - start)) : 0;
+                u.npad[j] = j < sm.n_seg ? max(0, min(len, cpad[sm.seg_kk[j]] - start)) : 0;
                 if (u.npad[j] > 0) u.kmax = j;
             }
             for (int j = D.K - 1; j >= 0; --j) {          // real slots of class j: [cpad[j+1], cpad[j+1] + cnt[j])
@@ -940,6 +1015,14 @@ cudaError_t launch_wait_expiry(int which, int32_t* device_status, cudaStream_t s
     return cudaGetLastError();
 }
 
+// nibble j = width of step j (bits[j] - bits[j-1]) for lists of at most four widths, else 0
+static int i8_wpack(const MoeDims& D) {
+    int wpack = 0, prev = 0;
+    if (D.K <= 4)
+        for (int j = 0; j < D.K; ++j) { wpack |= (D.bits[j] - prev) << (4 * j); prev = D.bits[j]; }
+    return wpack;
+}
+
 cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                           const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
                           const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
@@ -955,8 +1038,15 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
 
     const int ffn_grid = 2 * device_sm_count();
     const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
+    // operands of the expert kernels: the width steps themselves when the list has a specialised kernel (the fields of
+    // a step are merged in registers), otherwise the stored segments one by one
+    const int wp = i8_wpack(D);
+    const bool by_step = D.g == 128 && (wp == 0x4112 || wp == 0x422 || wp == 0x1115);
+    I8SegMap sm;
+    sm.n_seg = by_step ? D.K : Lgu.n_seg;
+    for (int j = 0; j < 8; ++j) sm.seg_kk[j] = by_step ? j : Lgu.seg_kk[j];
     i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
-                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status);
+                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status, sm);
     i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
                                                     qx, B.xk_x, sigma_x, device_status);
 
@@ -995,9 +1085,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
                                                              kappa, qh, B.xk_h, sigma_h, device_status);
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
-        int wpack = 0;
-        if (p.L.n_seg <= 4)
-            for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
+        const int wpack = i8_wpack(D);
         auto launch = [&](auto kc) -> cudaError_t {
             constexpr auto kern = decltype(kc)::value;
             cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
@@ -1009,7 +1097,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         cudaError_t e;
         if (D.g == 128 && wpack == 0x4112) e = launch(I8_KERNEL(128, 0x4112));        // {2,3,4,8}
         else if (D.g == 128 && wpack == 0x422) e = launch(I8_KERNEL(128, 0x422));     // {2,4,8}
-        else if (D.g == 128 && wpack == 0x1115) e = launch(I8_KERNEL(128, 0x1115));   // {5,6,7,8}
+        else if (D.g == 128 && wpack == 0x1115) e = launch(I8_KERNEL(128, 0x1115));   // {5,6,7,8}: the 5-bit step stored as 4 + 1
         else if (D.g == 128) e = launch(I8_KERNEL(128, 0));
         else e = launch(I8_KERNEL(64, 0));
 #undef I8_KERNEL

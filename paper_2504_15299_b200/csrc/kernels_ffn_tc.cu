@@ -254,11 +254,16 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     }
     // per-width constants of the dequant loop, read from shared memory instead of the kernel parameters
     // (a dynamically indexed parameter read costs a constant-cache round trip per tile)
-    int4* seg_tab = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + 256);   // {sw, seg_off, 2^-(bits[kk]-bits[0]) bits, logical width | offset of the segment's scales << 4}
+    // per stored segment: {storage width | width index << 8 | last segment of its width << 16, byte offset,
+    // bits of 2^(position - (top - b1)), scale_mode 1: byte offset of the scale of the field's lowest bit}
+    int4* seg_tab = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + 256);
     if (threadIdx.x < 8) {
-        const int kk = threadIdx.x;
-        const int db = kk < p.D.K ? p.D.bits[kk] - p.D.bits[0] : 0;
-        seg_tab[kk] = make_int4(p.L.seg_sw[kk], p.L.seg_off[kk], (127 - db) << 23, p.L.seg_w[kk] | (p.L.seg_sc_off[kk] << 4));
+        const int j = threadIdx.x;
+        const int kk = p.L.seg_kk[j];
+        const int last = (j < p.L.n_seg && p.L.last_seg[kk] == j) ? 1 : 0;
+        const int e = p.L.seg_shift[j] - (p.L.top - p.L.b1);
+        const int sc_t0 = p.L.w_sc_off[kk] + ((p.L.top - p.L.b1 - 1 - p.L.seg_shift[j]) - p.L.w_lv0[kk]) * D2MOE_TILE_ROWS * 2;
+        seg_tab[j] = make_int4(p.L.seg_sw[j] | (kk << 8) | (last << 16), p.L.seg_off[j], (127 + e) << 23, sc_t0);
     }
     if (warp == WARP_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -492,50 +497,49 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     seg_step(std::integral_constant<int, 2>{});
                     seg_step(std::integral_constant<int, 3>{});
                 } else {
+                    const int smax = p.L.last_seg[kmax];         // stored segments 0..smax
                     if (p.L.scale_mode == 1) {
                         // free residual scales: W_hat = lo + s1 Q + sum over the steps of s_l (2 bit_l - 1)
                         float cneg = 0.0f;                       // - sum of the scales of the steps folded in so far, times 2^-S
 #pragma unroll 1
-                        for (int kk = 0; kk <= kmax; ++kk) {
-                            const int4 tb = seg_tab[kk];
-                            const int sw = tb.x;
+                        for (int sj = 0; sj <= smax; ++sj) {
+                            const int4 tb = seg_tab[sj];
+                            const int sw = tb.x & 255, kk = (tb.x >> 8) & 255;
                             const uint32_t seg = wb + (uint32_t)tb.y;
-                            if (kk == 0) {
-                                dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, h2dup(s1 * two_mS * 16777216.0f), h2dup(lo * two_mS));
+                            if (kk == 0) {                       // a field of the base code: s1 times its value at its position
+                                const __half2 m0 = h2dup(s1 * __int_as_float(tb.z) * two_mS * 16777216.0f);
+                                if (sj == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, h2dup(lo * two_mS));
+                                else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
                             } else {
-                                const int W = tb.w & 15;
-                                const uint32_t sc = wb + (uint32_t)(tb.w >> 4) + 2u * rr;       // this row's scales of the segment
+                                const uint32_t sc = wb + (uint32_t)tb.w + 2u * rr;       // this row's scale of the field's lowest bit
                                 __half2 mb[8];
 #pragma unroll
                                 for (int pos = 0; pos < 8; ++pos) {
-                                    const int t = pos % sw;               // bit of the field; its step: W - 1 - t (most significant first)
-                                    float m = 0.0f;
-                                    if (t < W) {
-                                        unsigned short raw;
-                                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc + (uint32_t)((W - 1 - t) * D2MOE_TILE_ROWS * 2)));
-                                        const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
-                                        m = 2.0f * sl * __int_as_float((127 + 24 - pos) << 23);
-                                        if (pos < sw) cneg -= sl;         // each step once
-                                    }
-                                    mb[pos] = h2dup(m);
+                                    const int t = pos % sw;               // bit of the field; its step's scale lies t planes before
+                                    unsigned short raw;
+                                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc - (uint32_t)(t * D2MOE_TILE_ROWS * 2)));
+                                    const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
+                                    mb[pos] = h2dup(2.0f * sl * __int_as_float((127 + 24 - pos) << 23));
+                                    if (pos < sw) cneg -= sl;             // each step once
                                 }
-                                dequant_bits_dispatch<GS>(sw, seg, rr, wg, acc, W, mb);
+                                dequant_bits_dispatch<GS>(sw, seg, rr, wg, acc, sw, mb);
                             }
-                            if ((present >> kk) & 1u) write_tile(cneg);
+                            if (((tb.x >> 16) & 1) && ((present >> kk) & 1u)) write_tile(cneg);
                         }
                     } else {
 #pragma unroll 1
-                    for (int kk = 0; kk <= kmax; ++kk) {
-                        const int4 tb = seg_tab[kk];
-                        const int sw = tb.x;
-                        // M_kk * 2^-S and the multiplier of a code at bit position 0, M_kk * 2^(24 - S)
-                        const float Mk = s1 * __int_as_float(tb.z) * two_mS;
-                        const __half2 m0 = h2dup(Mk * 16777216.0f);
-                        const uint32_t seg = wb + (uint32_t)tb.y;
-                        if (kk == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
-                        else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
-                        if ((present >> kk) & 1u) write_tile(0.5f * Mk);
-                    }
+                        for (int sj = 0; sj <= smax; ++sj) {
+                            const int4 tb = seg_tab[sj];
+                            const int sw = tb.x & 255, kk = (tb.x >> 8) & 255;
+                            // the field's multiplier: s1 2^(position - (top - b1)) 2^-S, and for a code at bit position 0 of its lane
+                            const float Ms = s1 * __int_as_float(tb.z) * two_mS;
+                            const __half2 m0 = h2dup(Ms * 16777216.0f);
+                            const uint32_t seg = wb + (uint32_t)tb.y;
+                            if (sj == 0) dequant_dispatch<GS, true>(sw, seg, rr, wg, acc, m0, u0);
+                            else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
+                            // the last field of a width's step sits at that width's unit: half a step completes the tile
+                            if (((tb.x >> 16) & 1) && ((present >> kk) & 1u)) write_tile(0.5f * Ms);
+                        }
                     }
                 }
                 mbar_arrive(W_EMPTY(s));
@@ -936,7 +940,8 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         int wpack = 0;
-        if (p.L.n_seg <= 4 && p.L.scale_mode == 0)       // (their segment offsets are compile-time: tied-scale layout)
+        // (compile-time segment offsets: tied-scale layout, every width step stored as one segment)
+        if (p.L.n_seg <= 4 && p.L.scale_mode == 0 && p.L.n_seg == p.L.n_widths)
             for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
         auto launch = [&](auto kc) -> cudaError_t {
             constexpr auto kern = decltype(kc)::value;

@@ -20,9 +20,9 @@ struct I8Unit {
     int e;         // expert (routed, then shared)
     int slot0;     // first slot (multiple of 8); the quantised activations of slot s are rows 2s, 2s+1
     int nslots;    // slots in this unit (multiple of 8, <= 32)
-    int kmax;      // highest width index present
+    int kmax;      // last stored segment any of its tokens reads
     int nblk;      // blocks of 4 slots that hold at least one real token
-    int npad[8];   // slots covered by the product of segment j (multiple of 8, 0 = absent)
+    int npad[8];   // slots covered by the product of stored segment j (multiple of 8, 0 = absent)
     int blk[8];    // the real blocks: first slot / 4, relative to slot0
 };
 

@@ -198,8 +198,9 @@ __device__ __forceinline__ __half2 h2dup(float v) { return __float2half2_rn(v); 
 __device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 __device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
-// Compile-time description of a width list of at most four segments: nibble j of WPACK is the logical
-// width of segment j (stored 1, 2, 4 or 8 bits wide).  WPACK == 0 selects the run-time path.
+// Compile-time description of a width list of at most four widths: nibble j of WPACK is the width of step j
+// (bits[j] - bits[j-1]; sw: the width of the field it is stored in when that is a single field).  WPACK == 0
+// selects the run-time path.
 template <int WPACK>
 struct WidthList {
     __host__ __device__ static constexpr int w(int j) { return (WPACK >> (4 * j)) & 15; }
@@ -207,7 +208,8 @@ struct WidthList {
     __host__ __device__ static constexpr int count() { int k = 0; while (k < 8 && w(k) != 0) ++k; return k; }
     __host__ __device__ static constexpr int top() { int b = 0; for (int i = 0; i < count(); ++i) b += w(i); return b; }
     __host__ __device__ static constexpr int pos(int j) { int b = 0; for (int i = 0; i <= j; ++i) b += w(i); return top() - b; }
-    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * sw(i) / 8; return o; }
+    // a step of w bits is stored as power-of-two fields that add up to exactly w bits per code
+    __host__ __device__ static constexpr int seg_off(int gs, int j) { int o = D2MOE_TILE_ROWS * 4; for (int i = 0; i < j; ++i) o += D2MOE_TILE_ROWS * gs * w(i) / 8; return o; }
 };
 
 // exponent S of the common factor 2^-S from the header of a packed matrix

@@ -71,6 +71,10 @@ def test_packed_bytes_is_the_top_width_only(lib):
     assert a == b == c
     total, code, meta = a
     assert code == rows * cols and meta == rows * (cols // 64) * 4 and total == 256 + code + meta
+    # so do lists whose steps are not powers of two: 5 = 4 + 1, 3 = 2 + 1, 7 = 4 + 2 + 1 bits, eight one-bit steps
+    for bits in ((5, 6, 7, 8), (3, 8), (1, 8), (1, 2, 3, 4, 5, 6, 7, 8), (7, 8), (6, 8)):
+        assert binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, bits), rows, cols) == a, bits
+    assert binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (3, 5)), rows, cols)[1] == rows * cols * 5 // 8
     # a 4-bit top width stores half of that
     assert binding.packed_bytes(binding.Config(256, 512, 4, 2, 64, (2, 3, 4)), rows, cols)[1] == rows * cols // 2
     # rows are padded to the 64-row tile
