@@ -104,8 +104,15 @@ def sum_pinned(a: np.ndarray) -> np.ndarray:
     return acc[..., 0]
 
 
-def quantize(W: np.ndarray, bits: Sequence[int], group_size: int, scale_mode: int = 0) -> MWQTensor:
+def quantize(W: np.ndarray, bits: Sequence[int], group_size: int, scale_mode: int = 0,
+             col_energy: Optional[np.ndarray] = None, return_what: bool = False):
     """MWQ of W [rows, cols] with groups of ``group_size`` along the input (column) axis.
+
+    ``col_energy`` (scale_mode 1 only): per input column i the second moment d_i of the calibration
+    activations.  Eq. 5 with the cross-column terms of X X^T dropped is a weighted least-squares fit, whose
+    minimiser for Q = sign(R) is s = sum_i d_i |R_i| / sum_i d_i over the group (both sums in the pinned
+    order); with equal energies it is the plain mean.  ``return_what``: also return the fp32 reconstruction
+    at the top width as the quantizer itself accumulated it (used by the block compensation).
 
     Step 1 is the per-group asymmetric b1-bit quantization of Eq. 2; steps 2.. are the binary
     residual quantization of Eq. 4, one bit per step up to the top width, with tied scales
@@ -136,9 +143,18 @@ def quantize(W: np.ndarray, bits: Sequence[int], group_size: int, scale_mode: in
     R = (Wg - What).astype(F32)
     code = Q.astype(np.int32)
     s_extra = np.zeros((rows, cols // g, top - b1), dtype=F32) if scale_mode == 1 else None
+    if col_energy is not None:
+        assert scale_mode == 1
+        dg = np.ascontiguousarray(col_energy, dtype=F32).reshape(1, cols // g, g)
+        den = sum_pinned(dg)                                   # [1, groups]
     for j in range(1, top - b1 + 1):
         if scale_mode == 0:
             s_j = (s1_b * F32(2.0 ** -(j + 1))).astype(F32)   # exact: power-of-two multiple
+        elif col_energy is not None:
+            # Eq. 5 with per-column activation energies: weighted mean of |R|
+            mean_abs = (sum_pinned((np.abs(R) * dg).astype(F32)) / den).astype(F32)
+            s_extra[:, :, j - 1] = mean_abs.astype(np.float16).astype(F32)
+            s_j = s_extra[:, :, j - 1][:, :, None]
         else:
             # Eq. 5 without calibration data: argmin_s ||R - s sign(R)||^2 = mean |R| over the group
             mean_abs = (sum_pinned(np.abs(R)) / F32(g)).astype(F32)
@@ -149,7 +165,49 @@ def quantize(W: np.ndarray, bits: Sequence[int], group_size: int, scale_mode: in
         R = (Wg - What).astype(F32)
         code = code * 2 + bit.astype(np.int32)
     assert code.min() >= 0 and code.max() < (1 << top)
-    return MWQTensor(code.reshape(rows, cols).astype(np.uint8), s1, lo, tuple(bits), g, s_extra)
+    q = MWQTensor(code.reshape(rows, cols).astype(np.uint8), s1, lo, tuple(bits), g, s_extra)
+    if return_what:
+        return q, What.reshape(rows, cols)
+    return q
+
+
+def quantize_calibrated(W: np.ndarray, bits: Sequence[int], group_size: int, hc: Optional[np.ndarray],
+                        col_energy: Optional[np.ndarray] = None) -> MWQTensor:
+    """Calibration-aware MWQ (Eq. 3 / Eq. 5 and Algorithm 1) with free per-step scales.
+
+    ``hc``: the upper-triangular Cholesky factor H^c of (2 X X^T + lambda I)^-1 that Algorithm 1 starts from,
+    fp32 [cols, cols].  Reading of Algorithm 1 (its printed loop nest is garbled: the level loop never reaches
+    K, W is changed inside it, E is divided by an index that is not a block): blocks are the quantization
+    groups (gamma = g), taken left to right; a block is quantized at once through all its steps (Eq. 2, then
+    Eq. 4 with the scales of Eq. 5) - "only block-level compensation ... eliminating column-level error
+    corrections" (Section 3.3.1) -; its error at the top width, column j divided by H^c[j, j], is then taken
+    out of all later columns: W[:, later] -= E H^c[block, later].  All of it fp32, one rounding per operation,
+    the update as g successive rank-one corrections in ascending column order (so that it is reproducible bit
+    for bit).  PARITY UNPINNED as far as that reading goes; what is pinned: with a diagonal H^c nothing is
+    propagated and the result is ``quantize(..., scale_mode=1)``; the first block never changes; on correlated
+    activations the compensated weights reproduce W X better than the uncompensated ones.
+    """
+    check_bits(bits)
+    W = np.array(W, dtype=F32, copy=True)
+    rows, cols = W.shape
+    g = group_size
+    assert cols % g == 0
+    parts = []
+    for b in range(0, cols, g):
+        ce = None if col_energy is None else np.asarray(col_energy, dtype=F32)[b:b + g]
+        q, what = quantize(W[:, b:b + g], bits, g, scale_mode=1, col_energy=ce, return_what=True)
+        parts.append(q)
+        if hc is not None and b + g < cols:
+            hcf = np.asarray(hc, dtype=F32)
+            diag = hcf[np.arange(b, b + g), np.arange(b, b + g)]
+            E = ((W[:, b:b + g] - what).astype(F32) / diag[None, :]).astype(F32)
+            for j in range(g):
+                W[:, b + g:] = (W[:, b + g:] - (E[:, j:j + 1] * hcf[b + j, b + g:][None, :]).astype(F32)).astype(F32)
+    code = np.concatenate([q.code for q in parts], axis=1)
+    s1 = np.concatenate([q.s1 for q in parts], axis=1)
+    lo = np.concatenate([q.lo for q in parts], axis=1)
+    s_extra = np.concatenate([q.s_extra for q in parts], axis=1)
+    return MWQTensor(code, s1, lo, tuple(bits), g, s_extra)
 
 
 def slice_code(q: MWQTensor, b: int) -> np.ndarray:

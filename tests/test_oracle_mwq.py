@@ -333,3 +333,64 @@ def test_free_scales_approach_the_tied_ones_on_uniform_residuals():
     for j in range(1, 4):
         ratio = q.s_extra[:, :, j - 1] / (q.s1 * 2.0 ** -(j + 1))
         assert np.all(np.abs(ratio - 1.0) < 0.15), (j, ratio.min(), ratio.max())
+
+
+# ---------------------------------------------------------------- calibration-aware MWQ (Eq. 5 with activation energies, Algorithm 1)
+def calib(cols, n=512, seed=0, corr=0.6):
+    """Correlated synthetic calibration activations X [cols, n] and the factor Algorithm 1 starts from."""
+    import torch
+    r = np.random.default_rng(seed)
+    base = r.standard_normal((cols, n))
+    mix = np.eye(cols) + corr * np.roll(np.eye(cols), 1, axis=1) + 0.3 * corr * np.roll(np.eye(cols), 7, axis=1)
+    X = (mix @ base) * (0.5 + r.random((cols, 1)) * 2.0)
+    H = 2.0 * X @ X.T / n + 1e-2 * np.eye(cols)
+    Hinv = np.linalg.inv(H)
+    hc = torch.linalg.cholesky(torch.from_numpy(Hinv), upper=True).numpy().astype(F32)
+    return X, hc, (X * X).mean(axis=1).astype(F32)
+
+
+def test_weighted_scale_is_the_weighted_least_squares_scale():
+    W = gaussian(5, 128, seed=31)
+    d = (np.random.default_rng(32).random(128) * 3 + 0.1).astype(F32)
+    q = mwq.quantize(W, (2, 8), 32, scale_mode=1, col_energy=d)
+    Wg = W.reshape(5, 4, 32).astype(np.float64)
+    dg = d.reshape(1, 4, 32).astype(np.float64)
+    code = q.code.reshape(5, 4, 32).astype(np.int64)
+    What = q.lo.astype(np.float64)[:, :, None] + (code >> 6) * q.s1.astype(np.float64)[:, :, None]
+    for j in range(1, 7):
+        R = Wg - What
+        sign = np.where(R >= 0, 1.0, -1.0)
+        s = q.s_extra[:, :, j - 1].astype(np.float64)
+        err = lambda sc: (dg * (R - sc[:, :, None] * sign) ** 2).sum(axis=2)
+        slack = (dg.sum(axis=2)) * (2.0 ** -11 * s) ** 2
+        for f in np.linspace(0.0, 3.0, 61):
+            assert np.all(err(s) <= err(s * f) + slack)
+        assert np.allclose(s, (dg * np.abs(R)).sum(axis=2) / dg.sum(axis=2), rtol=2.0 ** -10)
+        What = What + s[:, :, None] * sign
+    # equal energies: the plain mean of scale_mode 1, whatever their common value
+    a = mwq.quantize(W, (2, 8), 32, scale_mode=1)
+    b = mwq.quantize(W, (2, 8), 32, scale_mode=1, col_energy=np.full(128, 4.0, dtype=F32))
+    assert np.array_equal(a.code, b.code) and np.array_equal(a.s_extra, b.s_extra)
+
+
+def test_block_compensation_special_cases_and_effect():
+    W = gaussian(48, 256, seed=33)
+    bits, g = (2, 3, 4, 8), 64
+    plain = mwq.quantize(W, bits, g, scale_mode=1)
+    # a diagonal factor propagates nothing: the calibration-free result
+    diag = np.diag(np.linspace(0.5, 2.0, 256)).astype(F32)
+    q = mwq.quantize_calibrated(W, bits, g, diag)
+    assert np.array_equal(q.code, plain.code) and np.array_equal(q.s_extra, plain.s_extra) and np.array_equal(q.s1, plain.s1)
+    assert np.array_equal(mwq.quantize_calibrated(W, bits, g, None).code, plain.code)
+    # correlated activations: the first block is untouched, later blocks change, and W X is reproduced better at every width
+    X, hc, energy = calib(256, seed=34)
+    qc = mwq.quantize_calibrated(W, bits, g, hc)
+    assert np.array_equal(qc.code[:, :g], plain.code[:, :g]) and not np.array_equal(qc.code[:, g:], plain.code[:, g:])
+    ref = W.astype(np.float64) @ X
+    for b in (4, 8):
+        e_plain = np.linalg.norm(mwq.dequantize(plain, b) @ X - ref)
+        e_comp = np.linalg.norm(mwq.dequantize(qc, b) @ X - ref)
+        assert e_comp < e_plain, (b, e_comp, e_plain)
+    # and with the energies in the scale fit as well it still runs through the same machinery
+    qe = mwq.quantize_calibrated(W, bits, g, hc, energy)
+    assert qe.code.shape == W.shape and np.array_equal(qe.code[:, :g] >> 6, plain.code[:, :g] >> 6)
