@@ -104,6 +104,25 @@ d2moe_status d2moe_pack_mwq(const d2moe_config* cfg, const float* W, int64_t row
                             void* packed, size_t packed_bytes, void* stream);
 
 /*
+ * Calibration-aware MWQ (Section 3.3.1: Eq. 5 with activation statistics, Algorithm 1), scale_mode 1 only.
+ *   W           device fp32 [rows, cols]; OVERWRITTEN (it is the working copy Algorithm 1 updates)
+ *   hc          device fp32 [cols, cols] row-major, the upper-triangular Cholesky factor H^c of
+ *               (2 X X^T + lambda I)^-1 that Algorithm 1 starts from (the caller factorises; NULL: no
+ *               error compensation)
+ *   col_energy  device fp32 [cols], second moment of every input column of the calibration activations
+ *               (NULL: equal energies): Eq. 5 with the cross-column terms of X X^T dropped, i.e. every
+ *               step's scale is the energy-weighted mean of |residual| over the group
+ * Blocks are the quantization groups, left to right: a group is quantized through all its steps, its error at
+ * the top width, column j divided by H^c[j, j], is taken out of all later columns (W[:, later] -= E H^c[block,
+ * later]); block-level compensation only, as the paper states.  The printed loop nest of Algorithm 1 is garbled;
+ * this reading is the library's.  With hc diagonal or NULL and col_energy NULL the result equals d2moe_pack_mwq.
+ * Packed layout, readers and kernels are those of scale_mode 1.
+ */
+d2moe_status d2moe_pack_mwq_calibrated(const d2moe_config* cfg, float* W, int64_t rows, int64_t cols,
+                                       const float* hc, const float* col_energy, void* packed,
+                                       size_t packed_bytes, void* stream);
+
+/*
  * Test hook: canonical codes of a packed matrix at width `bits` (bits[0] <= bits <= top width, need
  * not be a listed width): codes[r*cols + c] = top-width code >> (top - bits), one byte per weight.
  * scale / offset (either may be NULL): device fp32 [rows, cols/group_size], the stored s1 and lo.

@@ -59,7 +59,7 @@ _lib = None
 EXPORTS = ["d2moe_status_string", "d2moe_check_config", "d2moe_packed_bytes", "d2moe_pack_mwq",
            "d2moe_unpack_codes", "d2moe_workspace_bytes", "d2moe_route", "d2moe_moe_forward",
            "d2moe_stack_layer", "d2moe_moe_forward_events", "d2moe_forward_launch_count",
-           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry", "d2moe_unpack_scales", "d2moe_plan_load_order", "d2moe_plan_simulate", "d2moe_plan_budget_step"]
+           "d2moe_route_static_scratch", "d2moe_selftest_wait_expiry", "d2moe_unpack_scales", "d2moe_plan_load_order", "d2moe_plan_simulate", "d2moe_plan_budget_step", "d2moe_pack_mwq_calibrated"]
 
 
 def lib() -> ctypes.CDLL:
@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.d2moe_packed_bytes.argtypes = [cfgp, i64, i64, ctypes.POINTER(sz), ctypes.POINTER(sz), ctypes.POINTER(sz)]
     L.d2moe_pack_mwq.argtypes = [cfgp, vp, i64, i64, vp, sz, vp]
     L.d2moe_unpack_codes.argtypes = [cfgp, vp, i64, i64, ctypes.c_int, vp, vp, vp, vp]
+    L.d2moe_pack_mwq_calibrated.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, sz, vp]
     L.d2moe_unpack_scales.argtypes = [cfgp, vp, i64, i64, vp, vp]
     i32p, dp = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double)
     L.d2moe_plan_load_order.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, ctypes.c_int32, ctypes.POINTER(_PlanItem),
@@ -182,6 +183,19 @@ def pack_mwq(cfg: Config, W: torch.Tensor, out: Optional[torch.Tensor] = None, s
         out = torch.empty(total, dtype=torch.uint8, device=W.device)
     _check(lib().d2moe_pack_mwq(ctypes.byref(cfg.c()), _ptr(W.contiguous()), rows, cols, _ptr(out),
                                 out.numel(), _stream(stream)), "d2moe_pack_mwq")
+    return out
+
+
+def pack_mwq_calibrated(cfg: Config, W: torch.Tensor, hc: Optional[torch.Tensor] = None,
+                        col_energy: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Calibration-aware MWQ of a device fp32 matrix (a copy of W is made: the library overwrites its input)."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.dim() == 2
+    rows, cols = W.shape
+    total, _, _ = packed_bytes(cfg, rows, cols)
+    out = torch.empty(total, dtype=torch.uint8, device=W.device)
+    work = W.contiguous().clone()
+    _check(lib().d2moe_pack_mwq_calibrated(ctypes.byref(cfg.c()), _ptr(work), rows, cols, _ptr(hc), _ptr(col_energy),
+                                           _ptr(out), out.numel(), _stream(stream)), "d2moe_pack_mwq_calibrated")
     return out
 
 

@@ -91,6 +91,22 @@ extern "C" d2moe_status d2moe_pack_mwq(const d2moe_config* c, const float* W, in
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
 }
 
+extern "C" d2moe_status d2moe_pack_mwq_calibrated(const d2moe_config* c, float* W, int64_t rows, int64_t cols,
+                                                  const float* hc, const float* col_energy, void* packed,
+                                                  size_t packed_bytes, void* stream) {
+    size_t need = 0;
+    d2moe_status s = d2moe_packed_bytes(c, rows, cols, &need, nullptr, nullptr);
+    if (s != D2MOE_OK) return s;
+    if (c->scale_mode != 1) return D2MOE_ERR_CONFIG;         // the scale fit of Eq. 5 needs the free scales
+    if (!W || !packed) return D2MOE_ERR_NULL;
+    if (packed_bytes < need) return D2MOE_ERR_WORKSPACE;
+    if (((uintptr_t)packed & 255) != 0) return D2MOE_ERR_SHAPE;
+    PackLayout L;
+    d2moe_make_layout(L, c->bits, c->n_bits, c->group_size, rows, cols, c->scale_mode);
+    cudaError_t e = launch_pack_calibrated(L, c->bits, c->n_bits, W, hc, col_energy, (uint8_t*)packed, (cudaStream_t)stream);
+    return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
+}
+
 extern "C" d2moe_status d2moe_unpack_codes(const d2moe_config* c, const void* packed, int64_t rows,
                                            int64_t cols, int bits, uint8_t* codes, float* scale,
                                            float* offset, void* stream) {

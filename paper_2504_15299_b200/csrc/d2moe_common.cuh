@@ -180,6 +180,8 @@ void d2moe_carve_workspace(const d2moe_config* cfg, long long max_tokens, Worksp
 // kernels_pack.cu
 cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const float* W, uint8_t* packed,
                         cudaStream_t st);
+cudaError_t launch_pack_calibrated(const PackLayout& L, const int* bits, int n_bits, float* W, const float* hc,
+                                   const float* col_energy, uint8_t* packed, cudaStream_t st);
 cudaError_t launch_unpack(const PackLayout& L, const uint8_t* packed, int bits, uint8_t* codes,
                           float* scale, float* offset, cudaStream_t st);
 cudaError_t launch_unpack_scales(const PackLayout& L, const uint8_t* packed, float* s_extra, cudaStream_t st);

@@ -21,11 +21,15 @@ __global__ void pack_header_kernel(PackHeader* h, PackLayout L, int n_bits,
 // group's (s1, lo) and the top-width code of every element, in exactly the fp32 operation order of
 // the definition (one IEEE rounding per operation, no contraction).  Phase B: the block assembles
 // the segment words and writes them with coalesced stores.
+// Calibrated packing (g_first >= 0 selects one group per launch): col_energy (optional) weights the scale fit of
+// Eq. 5; err_out (optional, = W itself) receives, in place of the group's weights, their error at the top width
+// divided by hc_diag[column] - the E of Algorithm 1 that the caller then takes out of the later columns.
 __global__ void __launch_bounds__(PACK_THREADS)
-pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ packed) {
+pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ packed, int g_first,
+            const float* __restrict__ col_energy, float* err_out, const float* __restrict__ hc_diag) {
     extern __shared__ uint8_t smem[];
     uint8_t* codes = smem;                                  // [64][g]
-    const int G = blockIdx.x, rt = blockIdx.y;
+    const int G = (g_first >= 0 ? g_first : 0) + blockIdx.x, rt = blockIdx.y;
     const int g = L.g;
     uint8_t* blk = packed + d2moe_block_offset(L, rt, G);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,14 +95,26 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
                     cd[e] = (int)q;
                 }
             }
+            // Eq. 5 with per-column activation energies: the weighted mean of |R| (denominator: the group's energy sum)
+            float dw[8], den = (float)g;
+            if (col_energy) {
+                float dpart = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    dw[e] = e < n_el ? col_energy[(long long)G * g + lane + 32 * e] : 0.0f;
+                    if (e < n_el) dpart = __fadd_rn(dpart, dw[e]);
+                }
+                for (int off = 16; off; off >>= 1) dpart = __fadd_rn(dpart, __shfl_xor_sync(0xffffffffu, dpart, off));
+                den = dpart;
+            }
             for (int j = 1; j <= L.top - L.b1; ++j) {
                 // mean |R| in the pinned order: this lane's elements ascending, then the butterfly
                 float part = 0.0f;
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
-                    if (e < n_el) part = __fadd_rn(part, fabsf(rs[e]));
+                    if (e < n_el) part = __fadd_rn(part, col_energy ? __fmul_rn(fabsf(rs[e]), dw[e]) : fabsf(rs[e]));
                 for (int off = 16; off; off >>= 1) part = __fadd_rn(part, __shfl_xor_sync(0xffffffffu, part, off));
-                const __half sj_h = __float2half_rn(__fdiv_rn(part, (float)g));
+                const __half sj_h = __float2half_rn(__fdiv_rn(part, den));
                 const float sj = __half2float(sj_h);
                 if (lane == 0) *reinterpret_cast<__half*>(blk + d2moe_level_offset(L, j - 1, r)) = sj_h;
 #pragma unroll
@@ -114,6 +130,15 @@ pack_kernel(PackLayout L, const float* __restrict__ W, uint8_t* __restrict__ pac
 #pragma unroll
             for (int e = 0; e < 8; ++e)
                 if (e < n_el) codes[r * g + lane + 32 * e] = (uint8_t)cd[e];
+            if (err_out) {                                  // E = (W - W_hat) / H^c[j, j], in place of the group's weights
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if (e < n_el) {
+                        const long long col = (long long)G * g + lane + 32 * e;
+                        err_out[row * (long long)L.cols + col] = __fdiv_rn(__fsub_rn(wv[e], wh[e]), hc_diag[col * (L.cols + 1)]);
+                    }
+                }
+            }
         }
         if (lane == 0) {
             __half2 m = __halves2half2(s1_h, lo_h);          // low half = s1, high half = lo
@@ -193,7 +218,50 @@ __global__ void unpack_scales_kernel(PackLayout L, const uint8_t* __restrict__ p
     }
 }
 
+// Algorithm 1's propagation of a block's error: W[r, c] -= sum_j E[r, j] H^c[b + j, c] for every later column c,
+// as g successive corrections in ascending j, each one fp32 multiply and one fp32 subtract (the oracle's order).
+// E sits in W's own columns [b, b + g).  One thread per (row, column); the block's E rows are staged in shared memory.
+__global__ void __launch_bounds__(256)
+compensate_kernel(float* W, long long rows, int cols, int b, int g, const float* __restrict__ hc) {
+    extern __shared__ float s_e[];                          // [16 rows][g]
+    const int c = b + g + blockIdx.x * 16 + (threadIdx.x & 15);
+    const long long r0 = (long long)blockIdx.y * 16;
+    for (int i = threadIdx.x; i < 16 * g; i += 256) {
+        const long long r = r0 + i / g;
+        s_e[i] = r < rows ? W[r * cols + b + (i % g)] : 0.0f;
+    }
+    __syncthreads();
+    const long long r = r0 + (threadIdx.x >> 4);
+    if (r >= rows || c >= cols) return;
+    float acc = W[r * cols + c];
+    const float* e = s_e + (threadIdx.x >> 4) * g;
+    for (int j = 0; j < g; ++j) acc = __fsub_rn(acc, __fmul_rn(e[j], hc[(long long)(b + j) * cols + c]));
+    W[r * cols + c] = acc;
+}
+
 }  // namespace
+
+cudaError_t launch_pack_calibrated(const PackLayout& L, const int* bits, int n_bits, float* W, const float* hc,
+                                   const float* col_energy, uint8_t* packed, cudaStream_t st) {
+    cudaError_t err = cudaMemsetAsync(packed, 0, D2MOE_HEADER_BYTES, st);
+    if (err != cudaSuccess) return err;
+    int b[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int i = 0; i < n_bits; ++i) b[i] = bits[i];
+    pack_header_kernel<<<1, 32, 0, st>>>(reinterpret_cast<PackHeader*>(packed), L, n_bits,
+                                         b[0], b[1], b[2], b[3], b[4], b[5], b[6], b[7]);
+    const size_t smem = (size_t)D2MOE_TILE_ROWS * L.g;
+    for (int G = 0; G < L.n_groups; ++G) {
+        const bool prop = hc != nullptr && G + 1 < L.n_groups;
+        dim3 grid(1, L.n_rt);
+        pack_kernel<<<grid, PACK_THREADS, smem, st>>>(L, W, packed, G, col_energy, prop ? W : nullptr, hc);
+        if (prop) {
+            const int later = L.cols - (G + 1) * L.g;
+            dim3 cg((later + 15) / 16, (unsigned)((L.rows + 15) / 16));
+            compensate_kernel<<<cg, 256, (size_t)16 * L.g * 4, st>>>(W, L.rows, L.cols, G * L.g, L.g, hc);
+        }
+    }
+    return cudaGetLastError();
+}
 
 cudaError_t launch_unpack_scales(const PackLayout& L, const uint8_t* packed, float* s_extra, cudaStream_t st) {
     const long long n = (long long)L.rows * L.n_groups * (L.top - L.b1);
@@ -213,7 +281,7 @@ cudaError_t launch_pack(const PackLayout& L, const int* bits, int n_bits, const 
                                          b[0], b[1], b[2], b[3], b[4], b[5], b[6], b[7]);
     dim3 grid(L.n_groups, L.n_rt);
     size_t smem = (size_t)D2MOE_TILE_ROWS * L.g;
-    pack_kernel<<<grid, PACK_THREADS, smem, st>>>(L, W, packed);
+    pack_kernel<<<grid, PACK_THREADS, smem, st>>>(L, W, packed, -1, nullptr, nullptr, nullptr);
     return cudaGetLastError();
 }
 

@@ -587,3 +587,29 @@ def test_pack_free_scales_bit_exact(B, bits, g, rows, cols):
 def test_free_scales_layer_against_oracle(B, case):
     cross, err = small_layer_case(B, scale_mode=1, **case)
     assert cross < TOL and err < TOL, (cross, err)
+
+
+# ------------------------------------------------------------------ calibration-aware MWQ (Eq. 5 with energies, Algorithm 1)
+@pytest.mark.parametrize("bits,g,rows,cols", [((2, 3, 4, 8), 128, 200, 512), ((2, 4, 8), 64, 64, 256), ((3, 5), 32, 130, 128)])
+def test_pack_calibrated_bit_exact(B, bits, g, rows, cols):
+    """Codes, base scales and every per-step scale of the calibrated packing against the oracle, bit for bit: with the
+    Cholesky factor of a correlated synthetic activation set (error propagated block by block), with per-column
+    energies in the scale fit, with both, and with neither (= the calibration-free packing)."""
+    mwq, _, _ = oracle_mods()
+    cfg = B.Config(cols, cols, 2, 1, g, bits, scale_mode=1)
+    W = synth.normal(13, 5, (rows, cols), 0.02, "cuda")
+    X = synth.normal(13, 6, (cols, 384), 1.0, "cpu").double()
+    X = X + 0.6 * torch.roll(X, 1, 0) + 0.2 * torch.roll(X, 5, 0)
+    X = X * (0.5 + 2.0 * synth.normal(13, 7, (cols, 1), 1.0, "cpu").abs().double())
+    H = 2.0 * X @ X.T / X.shape[1] + 1e-2 * torch.eye(cols, dtype=torch.float64)
+    hc = torch.linalg.cholesky(torch.linalg.inv(H), upper=True).float().contiguous()
+    energy = (X * X).mean(dim=1).float().contiguous()
+    for use_hc, use_e in ((True, False), (False, True), (True, True), (False, False)):
+        blob = B.pack_mwq_calibrated(cfg, W, hc.cuda() if use_hc else None, energy.cuda() if use_e else None)
+        q = mwq.quantize_calibrated(np_f32(W), bits, g, hc.numpy() if use_hc else None, energy.numpy() if use_e else None)
+        codes, s1, lo = B.unpack_codes(cfg, blob, rows, cols, bits[-1])
+        assert np.array_equal(codes.cpu().numpy(), q.code), (use_hc, use_e)
+        assert np.array_equal(np_f32(s1), q.s1) and np.array_equal(np_f32(lo), q.lo)
+        assert np.array_equal(np_f32(B.unpack_scales(cfg, blob, rows, cols)), q.s_extra)
+        if not use_hc and not use_e:
+            assert torch.equal(blob[256:], B.pack_mwq(cfg, W)[256:])
