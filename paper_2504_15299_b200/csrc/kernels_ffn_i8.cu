@@ -49,8 +49,8 @@
 
 namespace {
 
-constexpr int I8_THREADS = 320;
-constexpr int I8_WARP_PROD = 8, I8_WARP_MMA = 9;
+constexpr int I8_THREADS = 448;
+constexpr int I8_WARP_PROD = 12, I8_WARP_MMA = 13;
 constexpr int I8_TMEM_COLS = 256;
 constexpr int I8_D_COLS = 64;                 // one accumulator buffer: 32 slots x (high, low)
 constexpr int I8_SLOTS = 32;                  // token slots per unit
@@ -241,7 +241,7 @@ template <int WPACK> using I8SegList = WidthList<WPACK>;
 // 32: first slot, 33: tile, 34: split), so that the phase starts without a trip to global memory.
 static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int r, int n_mine, uint32_t blks,
                                                  float (&acc)[4][4], uint8_t* smem) {
-    const float* rec = reinterpret_cast<const float*>(smem + p.smem_rec_off) + (threadIdx.x >> 5) * 40;
+    const float* rec = reinterpret_cast<const float*>(smem + p.smem_rec_off) + ((threadIdx.x >> 5) - 4) * 40;
     float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
     // the warpgroup's exchange barrier (128 arrivals): two phases per work item, so the parities are always 0, 1;
     // a bounded wait, like every other wait of the kernel
@@ -334,7 +334,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 256); }
+        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 384); }
         // an activation stage is released by the MMA issuer (its products have read the tile) and by
         // the eight folding warps (they have read the sums)
         for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 9); }
@@ -342,7 +342,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
         // a queue entry is released by the issuer warp and the eight unpack / fold warps
-        for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 9); }
+        for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 13); }
         for (int wg = 0; wg < 2; ++wg) mbar_init(bar0 + 8u * (uint32_t)(I8_N_BARS - 2 + wg), 128);
         *abort_flag = 0;
         *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
@@ -512,16 +512,14 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // all products have completed before TMEM is released
         if (gc > 0) mbar_wait(D_FULL((gc - 1) & 1), ((gc - 1) >> 1) & 1, abort_flag, p.status, true);
         if (gc > 1) mbar_wait(D_FULL((gc - 2) & 1), ((gc - 2) >> 1) & 1, abort_flag, p.status, true);
-    } else if (warp < 8) {
-        // -------- two warpgroups: unpack (segments wg, wg+2, ... of every group), fold, write out --------
-        const int wg = warp >> 2;
+    } else if (warp < 4) {
+        // -------- unpack warpgroup: fills both operand slots of every group (slot 0: segments 0, 2, (4, 6); slot 1:
+        // segments 1, 3, (5, 7)), one hand-off per slot --------
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
         const int blk = r >> 6, rr = r & 63;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
-        const uint32_t a_base = a_tmem + wg * 64 + lane_addr;          // my two operand tiles: +0, +32
-        const uint32_t d_base = d_tmem + lane_addr;
-        uint32_t gc = 0, hs = 0;                   // groups folded / operand hand-offs so far
-        uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
+        uint32_t hs[2] = {0, 0};                   // hand-offs so far, per slot
+        uint32_t ws = 0, wph = 0;
         uint32_t w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
         for (uint32_t qi = 0;; ++qi) {
             const uint32_t q = qi & (I8_NSQ - 1);
@@ -531,10 +529,113 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             if (lane == 0) mbar_arrive(SQ_EMPTY(q));
             if (item < 0) break;
             const I8Item ii = i8_item(p, item);
+            const int kmax = p.units[ii.unit].kmax;
+            for (int G = ii.g0; G < ii.g1; G += GPS) {
+                const int ng = min(GPS, ii.g1 - G);
+                mbar_wait_blk(W_FULL(ws), wph);
+#pragma unroll
+                for (int sub = 0; sub < GPS; ++sub) {
+                    if (sub < ng) {
+                        const uint32_t wb = w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes;
+                        auto handoff_begin = [&](int sl) {
+                            mbar_wait_blk(A_EMPTY(sl, 0), (hs[sl] & 1) ^ 1);
+                            tc_fence_after();
+                        };
+                        auto handoff_end = [&](int sl) {
+                            tc_wait_st();
+                            tc_fence_before();
+                            mbar_arrive(A_FULL(sl, 0));
+                            ++hs[sl];
+                        };
+                        if constexpr (SWPACK != 0) {
+                            using SL = I8SegList<SWPACK>;
+                            auto do_seg = [&](auto jc) {
+                                constexpr int J = decltype(jc)::value;
+                                if constexpr (J < SL::count()) {
+                                    if (J <= kmax) {
+                                        const uint32_t taddr = a_tmem + (J & 1) * 64 + lane_addr + ((J >> 1) & 1) * 32;
+                                        if constexpr (SL::w(J) == SL::sw(J))
+                                            unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J), taddr);
+                                        else
+                                            unpack_step<GS, SL::w(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::pos(J), taddr);
+                                    }
+                                }
+                            };
+                            constexpr int NHP = (SL::count() + 3) / 4;
+                            {                                        // slot 0: segments 0, 2
+                                handoff_begin(0);
+                                do_seg(std::integral_constant<int, 0>{});
+                                do_seg(std::integral_constant<int, 2>{});
+                                handoff_end(0);
+                            }
+                            if (1 <= kmax) {                         // slot 1: segments 1, 3
+                                handoff_begin(1);
+                                do_seg(std::integral_constant<int, 1>{});
+                                do_seg(std::integral_constant<int, 3>{});
+                                handoff_end(1);
+                            }
+                            if constexpr (NHP > 1) {
+                                if (4 <= kmax) {
+                                    handoff_begin(0);
+                                    do_seg(std::integral_constant<int, 4>{});
+                                    do_seg(std::integral_constant<int, 6>{});
+                                    handoff_end(0);
+                                }
+                                if (5 <= kmax) {
+                                    handoff_begin(1);
+                                    do_seg(std::integral_constant<int, 5>{});
+                                    do_seg(std::integral_constant<int, 7>{});
+                                    handoff_end(1);
+                                }
+                            }
+                        } else {
+#pragma unroll 1
+                            for (int j0 = 0; j0 <= kmax; j0 += 4) {
+#pragma unroll 1
+                                for (int sl = 0; sl < 2; ++sl) {
+                                    const int j = j0 + sl;
+                                    if (j > kmax) break;
+                                    const uint32_t taddr = a_tmem + sl * 64 + lane_addr;
+                                    handoff_begin(sl);
+                                    unpack_dispatch<GS>(p.L.seg_sw[j], wb + (uint32_t)p.L.seg_off[j], rr, p.L.seg_w[j], p.L.seg_shift[j], taddr);
+                                    if (j + 2 <= kmax)
+                                        unpack_dispatch<GS>(p.L.seg_sw[j + 2], wb + (uint32_t)p.L.seg_off[j + 2], rr, p.L.seg_w[j + 2],
+                                                            p.L.seg_shift[j + 2], taddr + 32);
+                                    handoff_end(sl);
+                                }
+                            }
+                        }
+                    }
+                }
+                mbar_arrive(W_EMPTY(ws));
+                w_addr += w_slot_bytes;
+                if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
+            }
+        }
+    } else if (warp < 12) {
+        // -------- two fold warpgroups: every group's accumulator into fp32 sums, each for half of the token blocks;
+        // output phase --------
+        const int wg = (warp >> 2) - 1;            // 0, 1
+        const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
+        const int blk = r >> 6, rr = r & 63;
+        const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
+        const uint32_t d_base = d_tmem + lane_addr;
+        uint32_t gc = 0;                           // groups folded so far
+        uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
+        uint32_t w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
+        const float s1_factor = __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
+        for (uint32_t qi = 0;; ++qi) {
+            const uint32_t q = qi & (I8_NSQ - 1);
+            mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
+            const int item = sq_item[q];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(SQ_EMPTY(q));
+            if (item < 0) break;
+            const I8Item ii = i8_item(p, item);
             const I8Unit* u = p.units + ii.unit;
-            const int kmax = u->kmax, nblk = u->nblk;
+            const int nblk = u->nblk;
             {
-                float* rec = reinterpret_cast<float*>(smem + p.smem_rec_off) + warp * 40;     // this warp's record of the item
+                float* rec = reinterpret_cast<float*>(smem + p.smem_rec_off) + (warp - 4) * 40;     // this warp's record of the item
                 const int slot0 = u->slot0;
                 asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
                              ::"r"(smem_u32(rec + lane)), "l"(p.sigma + slot0 + lane) : "memory");
@@ -550,165 +651,71 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             uint32_t myblks = 0;                                 // byte i: first slot / 4 of my block i
 #pragma unroll
             for (int i = 0; i < 4; ++i) myblks |= (uint32_t)u->blk[min((wg == 0 ? 0 : h0) + i, 7)] << (8 * i);
-            uint32_t blk_r[4];                                   // the same, one register each (hot loop)
+            uint32_t blk_r[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) blk_r[i] = (myblks >> (8 * i)) & 255u;
-#define MYBLK(i) blk_r[i]
             float acc[4][4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int s = 0; s < 4; ++s) acc[i][s] = 0.0f;
 
-            // Fold of group g (accumulator buffer g & 1) into acc, in two steps so that the tensor-memory loads are
-            // in flight while the warp does other work: fold_prefetch waits for the group's products and issues
-            // the loads of the first two blocks (it runs between the two segments the warp unpacks for the next
-            // group); fold_compute issues the loads of the other two blocks, folds the first two while those
-            // are in flight, then the rest.  fbs / fbph: ring position and phase of the group's activation sums,
-            // sub: group inside the stage, rel: last group of the stage (the stage is released afterwards).
-            uint32_t fv0[2][8], fv1[2][8];
-            auto fold_prefetch = [&](uint32_t g) {
-                const int buf = g & 1;
-                mbar_wait_blk(D_FULL(buf), (g >> 1) & 1);
-                tc_fence_after();
-#pragma unroll
-                for (int i = 0; i < 2; ++i)
-                    if (i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(i), fv0[i]);
-            };
-            auto fold_compute = [&](uint32_t g, uint32_t fbs, uint32_t fbph, int sub, bool rel, uint32_t meta) {
-                const int buf = g & 1;
-                const __half2 mh = as_h2(meta);
-                const float s1p = __low2float(mh) * __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
-                const float lo = __high2float(mh);
-                mbar_wait_blk(B_FULL(fbs), fbph);
-                const uint32_t xk_addr = xkbuf + (fbs * 2 + sub) * I8_XK_BYTES;
-                auto fold_block = [&](int b, const uint32_t (&v)[8]) {
-                    float xk[8];
-                    const uint32_t a = xk_addr + 32u * MYBLK(b);
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
-                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
-                    // the four slots of a block have one width: s1' kappa + lo once per block
-                    const float cx = fmaf(s1p, xk[1], lo);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) {
-                        const int di = (int)v[2 * s] * 128 + (int)v[2 * s + 1];
-                        acc[b][s] = fmaf(s1p, (float)di, acc[b][s]);
-                        acc[b][s] = fmaf(cx, xk[2 * s], acc[b][s]);
-                    }
-                };
-                tc_wait_ld();                                  // the first two blocks have landed
-                if (n_mine > 2) {
-#pragma unroll
-                    for (int i = 0; i < 2; ++i)
-                        if (2 + i < n_mine) tc_ld8(d_base + buf * I8_D_COLS + 8 * MYBLK(2 + i), fv1[i]);
-                } else {
-                    tc_fence_before();
-                    mbar_arrive(D_EMPTY(buf));                 // nothing more to read from this buffer
-                }
-                if (0 < n_mine) fold_block(0, fv0[0]);
-                if (1 < n_mine) fold_block(1, fv0[1]);
-                if (n_mine > 2) {
-                    tc_wait_ld();
-                    tc_fence_before();
-                    mbar_arrive(D_EMPTY(buf));
-                    fold_block(2, fv1[0]);
-                    if (3 < n_mine) fold_block(3, fv1[1]);
-                }
-                if (rel) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(B_EMPTY(fbs));
-                }
-            };
-
-            bool pend = false;
-            uint32_t pend_bs = 0, pend_bph = 0, pend_meta = 0;
-            int pend_sub = 0;
-            bool pend_rel = true;
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
+                // the scales of this stage's groups, then the stage is released as far as this warpgroup goes
                 mbar_wait_blk(W_FULL(ws), wph);
+                uint32_t meta[GPS];
 #pragma unroll
-                for (int sub = 0; sub < GPS; ++sub) {
-                    if (sub < ng) {
-                        const uint32_t wb = w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes;
-                        uint32_t meta;
-                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
-                        auto handoff_begin = [&]() {
-                            mbar_wait_blk(A_EMPTY(wg, 0), (hs & 1) ^ 1);
-                            tc_fence_after();
-                        };
-                        auto handoff_end = [&]() {
-                            tc_wait_st();
-                            tc_fence_before();
-                            mbar_arrive(A_FULL(wg, 0));
-                            ++hs;
-                        };
-                        if constexpr (SWPACK != 0) {
-                            using SL = I8SegList<SWPACK>;
-                            auto do_seg = [&](auto jc) {
-                                constexpr int J = decltype(jc)::value;
-                                if constexpr (J < SL::count()) {
-                                    if ((J & 1) == wg && J <= kmax) {
-                                        if constexpr (SL::w(J) == SL::sw(J))
-                                            unpack_segment<GS, SL::sw(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::w(J), SL::pos(J),
-                                                                          a_base + ((J >> 1) & 1) * 32);
-                                        else
-                                            unpack_step<GS, SL::w(J)>(wb + (uint32_t)SL::seg_off(GS, J), rr, SL::pos(J),
-                                                                      a_base + ((J >> 1) & 1) * 32);
-                                    }
-                                }
-                            };
-                            // a warpgroup hands over up to two tiles at a time: segments wg, wg + 2, then wg + 4, wg + 6
-                            constexpr int NHP = (SL::count() + 3) / 4;
-                            if (wg <= kmax) {
-                                handoff_begin();
-                                do_seg(std::integral_constant<int, 0>{});
-                                do_seg(std::integral_constant<int, 1>{});
-                                if (pend) fold_prefetch(gc - 1);     // in flight during the second segment
-                                do_seg(std::integral_constant<int, 2>{});
-                                do_seg(std::integral_constant<int, 3>{});
-                                handoff_end();
-                            } else if (pend) {
-                                fold_prefetch(gc - 1);
-                            }
-                            if constexpr (NHP > 1) {
-                                if (wg + 4 <= kmax) {
-                                    handoff_begin();
-                                    do_seg(std::integral_constant<int, 4>{});
-                                    do_seg(std::integral_constant<int, 5>{});
-                                    do_seg(std::integral_constant<int, 6>{});
-                                    do_seg(std::integral_constant<int, 7>{});
-                                    handoff_end();
-                                }
-                            }
-                        } else {
-                            if (wg > kmax && pend) fold_prefetch(gc - 1);
-#pragma unroll 1
-                            for (int j = wg; j <= kmax; j += 4) {
-                                handoff_begin();
-                                unpack_dispatch<GS>(p.L.seg_sw[j], wb + (uint32_t)p.L.seg_off[j], rr, p.L.seg_w[j], p.L.seg_shift[j], a_base);
-                                if (j + 2 <= kmax)
-                                    unpack_dispatch<GS>(p.L.seg_sw[j + 2], wb + (uint32_t)p.L.seg_off[j + 2], rr, p.L.seg_w[j + 2],
-                                                        p.L.seg_shift[j + 2], a_base + 32);
-                                if (pend && j + 4 > kmax) fold_prefetch(gc - 1);       // before the last hand-off of the group
-                                handoff_end();
-                            }
-                        }
-                        if (pend) fold_compute(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
-                        pend = true;
-                        pend_meta = meta;
-                        pend_bs = bs; pend_bph = bph; pend_sub = sub; pend_rel = sub == ng - 1;
-                        ++gc;
-                    }
-                }
+                for (int sub = 0; sub < GPS; ++sub)
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta[sub])
+                                 : "r"(w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes + 4u * rr));
                 mbar_arrive(W_EMPTY(ws));
                 w_addr += w_slot_bytes;
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
+                mbar_wait_blk(B_FULL(bs), bph);
+#pragma unroll
+                for (int sub = 0; sub < GPS; ++sub) {
+                    if (sub < ng) {
+                        const int buf = gc & 1;
+                        const __half2 mh = as_h2(meta[sub]);
+                        const float s1p = __low2float(mh) * s1_factor;
+                        const float lo = __high2float(mh);
+                        const uint32_t xk_addr = xkbuf + (bs * 2 + sub) * I8_XK_BYTES;
+                        const uint32_t d_addr = d_base + buf * I8_D_COLS;
+                        mbar_wait_blk(D_FULL(buf), (gc >> 1) & 1);
+                        tc_fence_after();
+                        auto fold_block = [&](int b, const uint32_t (&v)[8]) {
+                            float xk[8];
+                            const uint32_t a = xk_addr + 32u * blk_r[b];
+                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[0]), "=f"(xk[1]), "=f"(xk[2]), "=f"(xk[3]) : "r"(a));
+                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(xk[4]), "=f"(xk[5]), "=f"(xk[6]), "=f"(xk[7]) : "r"(a + 16u));
+                            const float cx = fmaf(s1p, xk[1], lo);
+#pragma unroll
+                            for (int s = 0; s < 4; ++s) {
+                                const int di = (int)v[2 * s] * 128 + (int)v[2 * s + 1];
+                                acc[b][s] = fmaf(s1p, (float)di, acc[b][s]);
+                                acc[b][s] = fmaf(cx, xk[2 * s], acc[b][s]);
+                            }
+                        };
+                        // two rounds of two blocks, one set of loaded values at a time (registers)
+#pragma unroll
+                        for (int rd = 0; rd < 2; ++rd) {
+                            uint32_t v[2][8];
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                if (2 * rd + i < n_mine) tc_ld8(d_addr + 8 * blk_r[2 * rd + i], v[i]);
+                            tc_wait_ld();
+                            if (rd == 1) { tc_fence_before(); mbar_arrive(D_EMPTY(buf)); }
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                if (2 * rd + i < n_mine) fold_block(2 * rd + i, v[i]);
+                        }
+                        ++gc;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(B_EMPTY(bs));
                 if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
-            }
-            if (pend) {
-                fold_prefetch(gc - 1);
-                fold_compute(gc - 1, pend_bs, pend_bph, GPS == 1 ? 0 : pend_sub, GPS == 1 ? true : pend_rel, pend_meta);
             }
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
@@ -716,7 +723,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int q = 0; q < 4; ++q) out[i][q] = acc[i][q];
+                for (int q4 = 0; q4 < 4; ++q4) out[i][q4] = acc[i][q4];
             i8_write_out(p, wg, r, n_mine, myblks, out, smem);
         }
     }
