@@ -5,6 +5,11 @@
 
 #include <string.h>
 
+bool d2moe_pdl_enabled() {
+    static const bool on = [] { const char* e = getenv("D2MOE_NO_PDL"); return !(e && e[0] == '1'); }();
+    return on;
+}
+
 namespace {
 
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
@@ -237,6 +242,7 @@ extern "C" d2moe_status d2moe_route(const d2moe_config* c, int64_t T, const void
     }
     uint8_t* w = (uint8_t*)workspace;
     RouteBufs R{topk_idx, topk_w, bit_idx, perm, inv_perm, group_off};
+    launch_chain_begin();
     cudaError_t e = launch_route(D, (const __nv_bfloat16*)x, (const __nv_bfloat16*)gate_w, logits,
                                  (const __nv_bfloat16*)bit_w, forced, R, (float*)(w + ws.off_logits),
                                  (int32_t*)(w + ws.off_keys), (int32_t*)(w + ws.off_hist), device_status, st);
@@ -274,9 +280,11 @@ static d2moe_status validate_forward(const d2moe_config* c, int64_t T, const voi
 static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x, const void* const* expert_w,
                                  const d2moe_route_in* in, const d2moe_route_out* pre,
                                  const void* residual, void* y, int32_t* device_status, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t st, void* const* ev = nullptr) {
+                                 size_t workspace_bytes, cudaStream_t st, void* const* ev = nullptr,
+                                 bool continue_chain = false) {
     d2moe_status s = validate_forward(c, T, x, expert_w, in, pre, y, workspace, workspace_bytes);
     if (s != D2MOE_OK || T == 0) return s;
+    if (!continue_chain) launch_chain_begin();
     const int n_exp = c->n_experts + c->n_shared;
     Workspace ws;
     d2moe_carve_workspace(c, T, &ws);
@@ -395,7 +403,8 @@ extern "C" d2moe_status d2moe_stack_layer(const d2moe_config* c, int64_t T, void
     if (s != D2MOE_OK || T == 0) return s;
     if (!(eps >= 0.0f)) return D2MOE_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
+    launch_chain_begin();
     cudaError_t e = launch_rmsnorm((int)T, c->d_model, eps, (const __nv_bfloat16*)x, (__nv_bfloat16*)xn, st);
     if (e != cudaSuccess) return D2MOE_ERR_CUDA;
-    return forward_impl(c, T, xn, expert_w, in, nullptr, x, x, device_status, workspace, workspace_bytes, st);
+    return forward_impl(c, T, xn, expert_w, in, nullptr, x, x, device_status, workspace, workspace_bytes, st, nullptr, true);
 }

@@ -17,6 +17,40 @@
 #define D2MOE_MAX_EXPERTS 320       // routed + shared
 
 // ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch for the kernels of one library call.
+//
+// The kernels of a call form a chain in one stream (route, group, unit build, quantise, expert
+// kernels, combine).  Every kernel after the first is launched with the programmatic-serialisation
+// attribute: its blocks may be scheduled while the kernel before it is still draining, run their
+// set-up, and block in pdl_enter() / pdl_wait() until that kernel has completed and its writes are
+// visible.  Every kernel of the chain executes the wait in every block before it reads or writes
+// global memory, so completion is transitive along the chain.  The first kernel of a call is an
+// ordinary launch.  D2MOE_NO_PDL=1 in the environment turns the attribute off (ordinary launches).
+// ------------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); }
+#endif
+
+bool d2moe_pdl_enabled();                 // d2moe_api.cu: reads the environment once
+inline thread_local bool t_launch_chained = false;
+inline void launch_chain_begin() { t_launch_chained = false; }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = (t_launch_chained && d2moe_pdl_enabled()) ? 1 : 0;
+    t_launch_chained = true;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Packed layout of one [rows, cols] matrix.
 //
 //   blob   = header (256 B) | block(rt = 0, G = 0) | block(0, 1) | ... | block(n_rt-1, n_groups-1)

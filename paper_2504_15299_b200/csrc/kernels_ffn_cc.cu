@@ -95,6 +95,7 @@ __device__ float row_dot(const PackLayout& L, const uint8_t* __restrict__ packed
 __global__ void __launch_bounds__(256)
 gateup_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, const __nv_bfloat16* __restrict__ x, RouteBufs R,
                  float* __restrict__ hbuf, int32_t* device_status) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
     const int a = blockIdx.x;                       // assignments on the x dimension: no 65535 limit
@@ -114,6 +115,7 @@ gateup_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, const __nv_bfloat16* __r
 __global__ void __launch_bounds__(256)
 down_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, RouteBufs R, const float* __restrict__ hbuf,
                float* __restrict__ obuf, int32_t* device_status) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
     const int a = blockIdx.x;
@@ -133,6 +135,7 @@ down_cc_kernel(MoeDims D, PackLayout L, ExpertPtrs P, RouteBufs R, const float* 
 __global__ void combine_kernel(MoeDims D, RouteBufs R, const float* __restrict__ obuf, int n_split,
                                size_t split_stride, const int32_t* __restrict__ row_map,
                                const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ y) {
+    pdl_enter();
     const int t = blockIdx.x;                       // tokens on the x dimension: no 65535 limit
     const int c = blockIdx.y * blockDim.x + threadIdx.x;
     if (c >= D.d) return;
@@ -156,6 +159,7 @@ __global__ void combine_kernel(MoeDims D, RouteBufs R, const float* __restrict__
 __global__ void combine4_kernel(MoeDims D, RouteBufs R, const float* __restrict__ obuf, int n_split,
                                 size_t split_stride, const int32_t* __restrict__ row_map,
                                 const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ y) {
+    pdl_enter();
     const int t = blockIdx.x;
     const int c = 4 * (blockIdx.y * blockDim.x + threadIdx.x);
     if (c >= D.d) return;
@@ -194,6 +198,7 @@ __global__ void combine4_kernel(MoeDims D, RouteBufs R, const float* __restrict_
 // evaluation; one block per token.
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(int d, double eps, const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xn) {
+    pdl_enter();
     __shared__ double red[8];
     const int t = blockIdx.x;
     double ss = 0.0;
@@ -220,7 +225,7 @@ cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, con
                                     int32_t* device_status, cudaStream_t st) {
     if (D.A_tot == 0) return cudaSuccess;
     dim3 g1(D.A_tot, (D.F + 7) / 8);
-    gateup_cc_kernel<<<g1, 256, 0, st>>>(D, Lgu, P, x, R, hbuf, device_status);
+    launch_chained(gateup_cc_kernel, dim3(g1), dim3(256), 0, st, D, Lgu, P, x, R, hbuf, device_status);
     return cudaGetLastError();
 }
 
@@ -229,7 +234,7 @@ cudaError_t launch_down_cuda_core(const MoeDims& D, const PackLayout& Ld, const 
                                   int32_t* device_status, cudaStream_t st) {
     if (D.A_tot == 0) return cudaSuccess;
     dim3 g2(D.A_tot, (D.d + 7) / 8);
-    down_cc_kernel<<<g2, 256, 0, st>>>(D, Ld, P, R, hbuf, obuf, device_status);
+    launch_chained(down_cc_kernel, dim3(g2), dim3(256), 0, st, D, Ld, P, R, hbuf, obuf, device_status);
     return cudaGetLastError();
 }
 
@@ -241,16 +246,16 @@ cudaError_t launch_combine(const MoeDims& D, const RouteBufs& R, const float* ob
                      ((uintptr_t)residual & 7) == 0;
     if (vec) {
         dim3 grid(D.T, (D.d / 4 + 127) / 128);
-        combine4_kernel<<<grid, 128, 0, st>>>(D, R, obuf, n_split, split_stride, row_map, residual, y);
+        launch_chained(combine4_kernel, dim3(grid), dim3(128), 0, st, D, R, obuf, n_split, split_stride, row_map, residual, y);
     } else {
         dim3 grid(D.T, (D.d + 255) / 256);
-        combine_kernel<<<grid, 256, 0, st>>>(D, R, obuf, n_split, split_stride, row_map, residual, y);
+        launch_chained(combine_kernel, dim3(grid), dim3(256), 0, st, D, R, obuf, n_split, split_stride, row_map, residual, y);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_rmsnorm(int T, int d, float eps, const __nv_bfloat16* x, __nv_bfloat16* xn, cudaStream_t st) {
     if (T == 0) return cudaSuccess;
-    rmsnorm_kernel<<<T, 256, 0, st>>>(d, (double)eps, x, xn);
+    launch_chained(rmsnorm_kernel, dim3(T), dim3(256), 0, st, d, (double)eps, x, xn);
     return cudaGetLastError();
 }

@@ -361,6 +361,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     const uint32_t d_tmem = tmem_base;                         // buffer b: columns [64 b, 64 b + 64)
     const uint32_t a_tmem = tmem_base + 2 * I8_D_COLS;         // warpgroup wg, slot sl: + (wg*2 + sl)*32
 
+    // set-up done (barriers, TMEM): from here on the kernel reads what the kernels before it wrote
+    pdl_wait();
     const int n_units = *p.n_units;
     const int total_items = n_units * p.n_row_tiles * p.n_split;
     const int nsw = p.nsw;
@@ -749,6 +751,7 @@ __global__ void __launch_bounds__(256)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
                int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status,
                I8SegMap sm) {
+    pdl_enter();
     extern __shared__ int32_t s_prep[];
     __shared__ int s_total;
     const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
@@ -886,64 +889,81 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
 // 2 slot + 1 of q, in the byte order of the operand cells (elements k, k+2, k+1, k+3), and writes
 // per group the integer sum X of the row's xq, and kappa of the slot.  GATHER: the row of slot s is
 // x[src_token[s]] (bf16); otherwise it is row s of an fp32 buffer.  Padding slots become zeros.
+// One block per slot at a time; a thread keeps its cells (four elements each; cell c = threadIdx.x + k blockDim.x,
+// k < I8_QCPT) in registers between the maximum and the rounding, so a row of up to 16 blockDim.x elements is read
+// once (a longer row goes round by round and is read twice).  blockDim.x is a multiple of 32: the 32 (or 16) cells of
+// a group sit in one warp.
+constexpr int I8_QCPT = 4;
 template <bool GATHER>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, const int32_t* __restrict__ src_token,
                 const int32_t* __restrict__ pad_off, int n_off, const float* __restrict__ kappa,
                 int8_t* __restrict__ q, float* __restrict__ xk, float* __restrict__ sigma, int32_t* status) {
-    __shared__ float s_red[8];
+    pdl_enter();
+    __shared__ uint32_t s_red[32];
     const int total = pad_off[n_off];
     const int n_cells = n / 4, cpg = g / 4;                 // cells per group: 16 or 32
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int per_round = I8_QCPT * blockDim.x;
+    const bool single = n_cells <= per_round;             // the whole row fits the block's registers
     for (int slot = blockIdx.x; slot < total; slot += gridDim.x) {
         const int t = src_token[slot];
-        uint32_t* qh = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot) * n);
-        uint32_t* ql = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot + 1) * n);
-        auto load4 = [&](int c, float (&v)[4]) {
-            if (GATHER) {
-                const uint2 raw = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(src) + (size_t)t * n)[c];
-                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
-            } else {
-                const float4 f = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + (size_t)slot * n)[c];
-                v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+        float v[I8_QCPT][4];
+        // cells [base, base + I8_QCPT blockDim.x) of the row into v; returns the bits of their largest magnitude
+        // (they order like unsigned integers, a NaN or an infinity above every finite value)
+        auto load_round = [&](int base) -> uint32_t {
+            uint32_t m = 0;
+#pragma unroll
+            for (int k = 0; k < I8_QCPT; ++k) {
+                const int c = base + threadIdx.x + k * blockDim.x;
+                v[k][0] = v[k][1] = v[k][2] = v[k][3] = 0.0f;
+                if (c < n_cells) {
+                    if (GATHER) {
+                        const uint2 raw = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(src) + (size_t)t * n)[c];
+                        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                        v[k][0] = a.x; v[k][1] = a.y; v[k][2] = b.x; v[k][3] = b.y;
+                    } else {
+                        const float4 f = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + (size_t)slot * n)[c];
+                        v[k][0] = f.x; v[k][1] = f.y; v[k][2] = f.z; v[k][3] = f.w;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) m = max(m, __float_as_uint(fabsf(v[k][i])));
+                }
             }
+            return m;
         };
-        float amax = 0.0f;
-        int bad = 0;                               // a NaN or an infinity in the row (fmaxf would drop a NaN)
-        if (t >= 0) {
-            for (int c = threadIdx.x; c < n_cells; c += 256) {
-                float v[4];
-                load4(c, v);
-                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[0]), fabsf(v[1]))), fmaxf(fabsf(v[2]), fabsf(v[3])));
-                bad |= !(fabsf(v[0]) < 3.0e38f) | !(fabsf(v[1]) < 3.0e38f) | !(fabsf(v[2]) < 3.0e38f) | !(fabsf(v[3]) < 3.0e38f);
-            }
-        }
-        for (int off = 16; off; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
-        bad = __syncthreads_or(bad);
-        if (lane == 0) s_red[warp] = amax;
+        uint32_t mbits = 0;
+        if (t >= 0)
+            for (int base = 0; base < n_cells; base += per_round) mbits = max(mbits, load_round(base));
+        mbits = __reduce_max_sync(0xffffffffu, mbits);
+        if (lane == 0) s_red[warp] = mbits;
         __syncthreads();
-        amax = s_red[0];
-        for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_red[i]);
+        mbits = lane < n_warps ? s_red[lane] : 0u;
+        mbits = __reduce_max_sync(0xffffffffu, mbits);
+        __syncthreads();                           // s_red is free for the next slot
+        const float amax = __uint_as_float(mbits);
+        const bool bad = !(amax < 3.0e38f);        // a NaN or an infinity in the row
         const bool live = t >= 0 && amax > 0.0f && !bad;
         // a row with a NaN or an infinity cannot be quantised: its outputs are zero and the call is flagged
         if (bad && threadIdx.x == 0 && status) atomicOr(status, D2MOE_DEV_NONFINITE);
         const float scale = live ? I8_XMAX / amax : 0.0f;
         const float kap = kappa[slot];
         if (threadIdx.x == 0) sigma[slot] = live ? amax / I8_XMAX : 0.0f;
-        const int n_iter = (n_cells + 255) / 256;
-        for (int itr = 0; itr < n_iter; ++itr) {
-            const int c = itr * 256 + threadIdx.x;
+        uint32_t* qh = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot) * n);
+        uint32_t* ql = reinterpret_cast<uint32_t*>(q + (size_t)(2 * slot + 1) * n);
+        for (int base = 0; base < n_cells; base += per_round) {
+        if (!single && live) load_round(base);
+#pragma unroll
+        for (int k = 0; k < I8_QCPT; ++k) {
+            const int c = base + threadIdx.x + k * blockDim.x;
             int sum = 0;
             if (c < n_cells) {
                 uint32_t wh = 0, wl = 0;
                 if (live) {
-                    float v[4];
-                    load4(c, v);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        int xq = __float2int_rn(v[i] * scale);
+                        int xq = __float2int_rn(v[k][i] * scale);
                         xq = max(-16191, min(16191, xq));
                         const int lo8 = ((xq + 64) & 127) - 64;
                         const int hi = (xq - lo8) >> 7;
@@ -962,6 +982,7 @@ i8_quant_kernel(int n, int g, long long R_alloc, const void* __restrict__ src, c
                 o.x = (float)sum; o.y = kap;
                 reinterpret_cast<float2*>(xk)[(size_t)G * R_alloc + slot] = o;
             }
+        }
         }
     }
 }
@@ -1052,9 +1073,11 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     I8SegMap sm;
     sm.n_seg = by_step ? D.K : Lgu.n_seg;
     for (int j = 0; j < 8; ++j) sm.seg_kk[j] = by_step ? j : Lgu.seg_kk[j];
-    i8_prep_kernel<<<1, 256, prep_smem, st>>>(D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
+    launch_chained(i8_prep_kernel, dim3(1), dim3(256), prep_smem, st, D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
                                       pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status, sm);
-    i8_quant_kernel<true><<<q_blocks, 256, 0, st>>>(D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
+    // threads per slot: a quarter of the row's cells, in whole warps
+    auto q_threads = [](int n) { const int t = ((n / 4 + I8_QCPT - 1) / I8_QCPT + 31) & ~31; return t < 1024 ? t : 1024; };
+    launch_chained(i8_quant_kernel<true>, dim3(q_blocks), dim3(q_threads(D.d)), 0, st, D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,
                                                     qx, B.xk_x, sigma_x, device_status);
 
     TmaMaps maps_x, maps_h;
@@ -1088,8 +1111,8 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         p.smem_bar_off = (p.smem_rec_off + rec_bytes + 511) & ~511;   // 512-byte aligned from the 1024-byte aligned base
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         if (mode == 1)
-            i8_quant_kernel<false><<<q_blocks, 256, 0, st>>>(D.F, D.g, pl.R_alloc, B.h32, B.src_token, B.pad_off, n_exp,
-                                                             kappa, qh, B.xk_h, sigma_h, device_status);
+            launch_chained(i8_quant_kernel<false>, dim3(q_blocks), dim3(q_threads(D.F)), 0, st, D.F, D.g, pl.R_alloc, B.h32,
+                           B.src_token, B.pad_off, n_exp, kappa, qh, B.xk_h, sigma_h, device_status);
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         const int wpack = i8_wpack(D);
@@ -1097,7 +1120,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
             constexpr auto kern = decltype(kc)::value;
             cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
             if (err != cudaSuccess) return err;
-            kern<<<ffn_grid, I8_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            launch_chained(kern, dim3(ffn_grid), dim3(I8_THREADS), smem_bytes, st, p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
 #define I8_KERNEL(GS_, WP_) std::integral_constant<decltype(&ffn_i8_kernel<GS_, WP_>), &ffn_i8_kernel<GS_, WP_>>{}

@@ -277,6 +277,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     const uint32_t d_tmem = tmem_base;                       // columns [0, n_cap)
     const uint32_t a_tmem = tmem_base + D_COLS;              // A_SLOTS tiles, 64 columns apart
 
+    // set-up done (barriers, TMEM): from here on the kernel reads what the kernels before it wrote
+    pdl_wait();
     const int n_units = *p.n_units;
     const int total_items = n_units * p.n_row_tiles * p.n_split;
     const int nsw = p.nsw;
@@ -648,6 +650,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(MoeDims D, RouteBufs R, int n_cap, TcUnit* units, int* n_units, int32_t* pad_off,
                int32_t* row_map, int32_t* src_token, int max_units, int ffn_grid, int32_t* status) {
+    pdl_enter();
     __shared__ int s_total_rows, s_n_units;
     __shared__ int s_cost[1024];
     const int n_keys = D.E * D.K + D.n_shared;
@@ -795,6 +798,7 @@ __global__ void __launch_bounds__(128)
 tc_gather_kernel(int d, const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ src_token,
                  const int32_t* __restrict__ pad_off, int n_keys, __half* __restrict__ xp16,
                  float* __restrict__ row_scale, long long R_alloc, int32_t* status) {
+    pdl_enter();
     __shared__ float s_red[4];
     const int total_rows = pad_off[n_keys];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -907,9 +911,9 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
     auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
     const int n_keys = D.E * D.K + D.n_shared;
     const int sms = device_sm_count();
-    tc_prep_kernel<<<1, 256, 0, st>>>(D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms,
+    launch_chained(tc_prep_kernel, dim3(1), dim3(256), 0, st, D, R, pl.n_cap, B.units, B.n_units, B.pad_off, B.row_map, B.src_token, pl.max_units, sms,
                                       device_status);
-    tc_gather_kernel<<<1184, 128, 0, st>>>(D.d, x, B.src_token, B.pad_off, n_keys, B.xp16, B.slot_f, pl.R_alloc, device_status);
+    launch_chained(tc_gather_kernel, dim3(1184), dim3(128), 0, st, D.d, x, B.src_token, B.pad_off, n_keys, B.xp16, B.slot_f, pl.R_alloc, device_status);
 
     TmaMaps maps_x, maps_h;
     if (!make_maps(&maps_x, B.xp16, pl.R_alloc, D.d) || !make_maps(&maps_h, B.h16, pl.R_alloc, D.F))
@@ -947,7 +951,7 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
             constexpr auto kern = decltype(kc)::value;
             cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
             if (err != cudaSuccess) return err;
-            kern<<<sms, TC_THREADS, smem_bytes, st>>>(p, mode == 0 ? maps_x : maps_h);
+            launch_chained(kern, dim3(sms), dim3(TC_THREADS), smem_bytes, st, p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
 #define TC_KERNEL(GS_, WP_) std::integral_constant<decltype(&ffn_tc_kernel<GS_, WP_>), &ffn_tc_kernel<GS_, WP_>>{}

@@ -77,6 +77,7 @@ route_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16
              const float* __restrict__ logits_in, const __nv_bfloat16* __restrict__ bit_w,
              const int8_t* __restrict__ forced, RouteBufs R, int32_t* __restrict__ keys,
              int32_t* __restrict__ device_status) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= D.T) return;
@@ -136,6 +137,7 @@ route_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16
 
 // One warp per key: count the assignments that carry it.
 __global__ void count_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ hist) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (key >= n_keys) return;
@@ -150,6 +152,7 @@ __global__ void count_kernel(int A, int n_keys, const int32_t* __restrict__ keys
 
 // Exclusive prefix sum of the histogram by one warp.
 __global__ void scan_kernel(int n_keys, const int32_t* __restrict__ hist, int32_t* __restrict__ group_off) {
+    pdl_enter();
     const int lane = threadIdx.x;
     int carry = 0;
     for (int base = 0; base < n_keys; base += 32) {
@@ -170,6 +173,7 @@ __global__ void scan_kernel(int n_keys, const int32_t* __restrict__ hist, int32_
 __global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ keys,
                                const int32_t* __restrict__ group_off, int32_t* __restrict__ perm,
                                int32_t* __restrict__ inv_perm) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (key >= n_keys) return;
@@ -197,6 +201,7 @@ __global__ void scatter_kernel(int A, int n_keys, const int32_t* __restrict__ ke
 __global__ void __launch_bounds__(1024)
 group_block_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
                  int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+    pdl_enter();
     extern __shared__ int32_t s_grp[];
     int32_t* s_keys = s_grp;
     int32_t* s_off = s_grp + ((A + 31) & ~31);
@@ -274,6 +279,7 @@ __device__ __forceinline__ void stage_row(__nv_bfloat16* dst, const __nv_bfloat1
 __global__ void __launch_bounds__(256)
 gate_logits_kernel(int T, int E, int d, const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gate_w,
                    float* __restrict__ logits, int TB, int EB) {
+    pdl_enter();
     extern __shared__ __align__(16) uint8_t rsm[];
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(rsm);
     __nv_bfloat16* ws = xs + (size_t)TB * d;
@@ -298,6 +304,7 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
                    const float* __restrict__ logits_in, const __nv_bfloat16* __restrict__ bit_w,
                    const int8_t* __restrict__ forced, RouteBufs R, int32_t* __restrict__ keys,
                    int32_t* __restrict__ device_status, int EB) {
+    pdl_enter();
     extern __shared__ __align__(16) uint8_t rsm[];
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(rsm);
     __nv_bfloat16* ws = xs + D.d;
@@ -409,7 +416,7 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
             cudaError_t e = ensure_dynamic_smem<&gate_logits_kernel>((int)lsm);
             if (e != cudaSuccess) return e;
             dim3 grid((D.T + TB - 1) / TB, (D.E + EBL - 1) / EBL);
-            gate_logits_kernel<<<grid, 256, lsm, st>>>(D.T, D.E, D.d, x, gate_w, logits_ws, TB, EBL);
+            launch_chained(gate_logits_kernel, dim3(grid), dim3(256), lsm, st, D.T, D.E, D.d, x, gate_w, logits_ws, TB, EBL);
             logits_in = logits_ws;
             gate_w = nullptr;
         }
@@ -418,9 +425,9 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
         if (e != cudaSuccess) return e;
         // logits and widths both supplied: no dot products, one warp per token does the selection
         const int threads = (logits_in && forced) ? 32 : 256;
-        route_block_kernel<<<D.T, threads, smem, st>>>(D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status, EB);
+        launch_chained(route_block_kernel, dim3(D.T), dim3(threads), smem, st, D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status, EB);
     } else
-    route_kernel<<<(D.T + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+    launch_chained(route_kernel, dim3((D.T + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, st, 
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
     // few assignments and keys: histogram, scan and scatter in one single-block launch (beyond about a
     // thousand warp walks the three grid-wide kernels are faster: 39 vs 10 us at 192 keys x 1536 assignments)
@@ -431,12 +438,12 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
         cudaError_t e = ensure_dynamic_smem<&group_block_kernel>((int)gsm);
         if (e != cudaSuccess) return e;
         const int blocks = small ? 1 : (n_keys < 16 ? n_keys : 16);
-        group_block_kernel<<<blocks, 1024, gsm, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+        launch_chained(group_block_kernel, dim3(blocks), dim3(1024), gsm, st, D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
         return cudaGetLastError();
     }
-    count_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, hist_ws);
-    scan_kernel<<<1, 32, 0, st>>>(n_keys, hist_ws, R.group_off);
-    scatter_kernel<<<(n_keys + 3) / 4, 128, 0, st>>>(D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+    launch_chained(count_kernel, dim3((n_keys + 3) / 4), dim3(128), 0, st, D.A, n_keys, keys_ws, hist_ws);
+    launch_chained(scan_kernel, dim3(1), dim3(32), 0, st, n_keys, hist_ws, R.group_off);
+    launch_chained(scatter_kernel, dim3((n_keys + 3) / 4), dim3(128), 0, st, D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
     return cudaGetLastError();
 }
 
@@ -509,6 +516,7 @@ extern "C" d2moe_status d2moe_route_static_scratch(const d2moe_config* c, int64_
     int32_t* keys = reinterpret_cast<int32_t*>(scratch);
     int32_t* hist = keys + D2MOE_STATIC_MAX_ASSIGNMENTS;
     RouteBufs R{topk_idx, topk_w, bit_idx, perm, inv_perm, group_off};
+    launch_chain_begin();
     cudaError_t e = launch_route(D, (const __nv_bfloat16*)x, (const __nv_bfloat16*)gate_w, logits,
                                  (const __nv_bfloat16*)bit_w, forced, R, nullptr, keys, hist, device_status, st);
     return e == cudaSuccess ? D2MOE_OK : D2MOE_ERR_CUDA;
