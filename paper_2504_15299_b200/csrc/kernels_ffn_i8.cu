@@ -25,13 +25,14 @@
 //     (the plane reuse of Section 3.4), through a ring of bulk async copies; a unit whose widest
 //     token is narrower than the top width reads only the prefix it needs.
 //   * The accumulator is double buffered per group: while the products of group G+1 run, the
-//     dequant threads fold group G into fp32 registers.
+//     fold warps add group G to their fp32 registers.
 //
-// CTA = 320 threads, 2 CTAs per SM (96 registers per thread).  Warps 0-3 and 4-7 are two warpgroups
-// (thread = weight row = TMEM lane): warpgroup w unpacks the segments w, w+2 of every group into its
-// two 32-column operand tiles in TMEM, hands both to the issuer at once and folds half of the unit's
-// token blocks; warp 8 streams packed blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and
-// the per-group activation sums, warp 9 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns +
+// CTA = 448 threads, 2 CTAs per SM (72 registers per thread); thread = weight row = TMEM lane in every
+// warpgroup.  Warps 0-3 unpack: per group they fill operand slot 0 (segments 0 and 2 of the group, two
+// 32-column tiles in TMEM) and hand it to the issuer, then slot 1 (segments 1 and 3).  Warps 4-7 and 8-11
+// fold: each warpgroup takes half of the unit's token blocks and, at the end of a work item, half of the
+// output phase.  Warp 12 streams packed blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and
+// the per-group activation sums, warp 13 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns +
 // 4 x 32 operand columns.
 //
 // Work distribution: a work item is one unit x one tile of 128 weight rows x a range of groups.  The
@@ -259,26 +260,26 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int 
         }
     }
     if (p.mode == 0) {
-        if (blk == 1) {
+        // rows r < 64 of the tile hold the gate projection, rows r >= 64 the up projection of the same 64 hidden
+        // units: the two halves exchange through shared memory so that each finishes half of the blocks
+        // (the gate half blocks 0 and 1 with the other's up values, the up half blocks 2 and 3 with the other's gate values)
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (i < n_mine)
+        for (int i = 0; i < 4; ++i)
+            if (i < n_mine && (blk == 1) == (i < 2))
 #pragma unroll
-                    for (int s = 0; s < 4; ++s) epi[rr * I8_EPI_STRIDE + 4 * i + s] = acc[i][s];
-        }
+                for (int s = 0; s < 4; ++s) epi[rr * I8_EPI_STRIDE + 4 * i + s] = acc[i][s];
         mbar_arrive(ebar);
         mbar_wait_blk(ebar, 0);
-        if (blk == 0) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (i < n_mine) {
-                    float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
+        for (int i = 0; i < 4; ++i) {
+            if (i < n_mine && (blk == 0) == (i < 2)) {
+                float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
 #pragma unroll
-                    for (int s = 0; s < 4; ++s) {
-                        const float g = acc[i][s];
-                        const float up = epi[rr * I8_EPI_STRIDE + 4 * i + s];
-                        dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
-                    }
+                for (int s = 0; s < 4; ++s) {
+                    const float other = epi[rr * I8_EPI_STRIDE + 4 * i + s];
+                    const float g = blk == 0 ? acc[i][s] : other;
+                    const float up = blk == 0 ? other : acc[i][s];
+                    dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
                 }
             }
         }
@@ -341,7 +342,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         for (int wg = 0; wg < 2; ++wg)
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
-        // a queue entry is released by the issuer warp and the eight unpack / fold warps
+        // a queue entry is released by the issuer warp, the four unpack warps and the eight fold warps
         for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 13); }
         for (int wg = 0; wg < 2; ++wg) mbar_init(bar0 + 8u * (uint32_t)(I8_N_BARS - 2 + wg), 128);
         *abort_flag = 0;
@@ -856,8 +857,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
                     if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
             }
             units[nu] = u;                        // every window starts with a real token: never empty
-            // work per group and warp: a warpgroup unpacks every other segment and folds half of the blocks
-            cost[nu] = 80 * ((u.kmax + 2) / 2) + 25 * ((u.nblk + 1) / 2);
+            // work per group: one warpgroup unpacks every operand, each of the other two folds half of the blocks
+            cost[nu] = 80 * (u.kmax + 1) + 25 * ((u.nblk + 1) / 2);
         }
     }
     __syncthreads();
@@ -1100,7 +1101,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         const int epi_bytes = 2 * 64 * I8_EPI_STRIDE * 4;
         const int bar_bytes = 512;
         const int budget = 112 * 1024;
-        const int rec_bytes = 8 * 40 * 4;                             // per unpack / fold warp: the record of its work item
+        const int rec_bytes = 8 * 40 * 4;                             // per fold warp: the record of its work item
         int nsw = (budget - b_bytes - epi_bytes - rec_bytes - 128 - bar_bytes - 1024) / w_slot;
         if (nsw > I8_MAX_NSW) nsw = I8_MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
