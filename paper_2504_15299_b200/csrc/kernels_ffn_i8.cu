@@ -335,13 +335,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 384); }
+        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 12); }
         // an activation stage is released by the MMA issuer (its products have read the tile) and by
         // the eight folding warps (they have read the sums)
         for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 9); }
         for (int wg = 0; wg < 2; ++wg)
-            for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 128); mbar_init(A_EMPTY(wg, sl), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 256); }
+            for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 4); mbar_init(A_EMPTY(wg, sl), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 8); }
         // a queue entry is released by the issuer warp, the four unpack warps and the eight fold warps
         for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 13); }
         for (int wg = 0; wg < 2; ++wg) mbar_init(bar0 + 8u * (uint32_t)(I8_N_BARS - 2 + wg), 128);
@@ -547,7 +547,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         auto handoff_end = [&](int sl) {
                             tc_wait_st();
                             tc_fence_before();
-                            mbar_arrive(A_FULL(sl, 0));
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(A_FULL(sl, 0));
                             ++hs[sl];
                         };
                         if constexpr (SWPACK != 0) {
@@ -610,7 +611,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                         }
                     }
                 }
-                mbar_arrive(W_EMPTY(ws));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(W_EMPTY(ws));
                 w_addr += w_slot_bytes;
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
             }
@@ -672,7 +674,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 for (int sub = 0; sub < GPS; ++sub)
                     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta[sub])
                                  : "r"(w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes + 4u * rr));
-                mbar_arrive(W_EMPTY(ws));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(W_EMPTY(ws));
                 w_addr += w_slot_bytes;
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
                 mbar_wait_blk(B_FULL(bs), bph);
@@ -708,7 +711,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                             for (int i = 0; i < 2; ++i)
                                 if (2 * rd + i < n_mine) tc_ld8(d_addr + 8 * blk_r[2 * rd + i], v[i]);
                             tc_wait_ld();
-                            if (rd == 1) { tc_fence_before(); mbar_arrive(D_EMPTY(buf)); }
+                            if (rd == 1) { tc_fence_before(); __syncwarp(); if (lane == 0) mbar_arrive(D_EMPTY(buf)); }
 #pragma unroll
                             for (int i = 0; i < 2; ++i)
                                 if (2 * rd + i < n_mine) fold_block(2 * rd + i, v[i]);
