@@ -494,10 +494,52 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                             }
                         }
                     };
-                    seg_step(std::integral_constant<int, 0>{});
-                    seg_step(std::integral_constant<int, 1>{});
-                    seg_step(std::integral_constant<int, 2>{});
-                    seg_step(std::integral_constant<int, 3>{});
+                    // free residual scales: W_hat = lo + s1 Q + sum over the steps of s_l (2 bit_l - 1); a step's w one-bit
+                    // levels each bring their own scale (stored in front of the step's codes)
+                    float cneg = 0.0f;                           // - sum of the scales folded in so far, times 2^-S
+                    auto seg_step_free = [&](auto jc) {
+                        constexpr int J = decltype(jc)::value;
+                        if constexpr (J < WL::count()) {
+                            if (J <= kmax) {
+                                const uint32_t seg = wb + (uint32_t)p.L.seg_off[J];
+                                if constexpr (J == 0) {
+                                    dequant_segment<GS, WL::sw(0), true>(seg, rr, wg, acc, h2dup(s1 * two_mS * 16777216.0f),
+                                                                         h2dup(lo * two_mS));
+                                } else {
+                                    constexpr int SW = WL::sw(J);
+                                    // this row's scale of the field's lowest bit; bit t of the field: t planes before
+                                    const uint32_t sc = wb + (uint32_t)(p.L.w_sc_off[J] + ((p.L.top - p.L.b1 - 1 - p.L.seg_shift[J]) - p.L.w_lv0[J]) * D2MOE_TILE_ROWS * 2)
+                                                      + 2u * rr;
+                                    float sl2[SW];
+#pragma unroll
+                                    for (int t = 0; t < SW; ++t) {
+                                        unsigned short raw;
+                                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc - (uint32_t)(t * D2MOE_TILE_ROWS * 2)));
+                                        const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
+                                        cneg -= sl;
+                                        sl2[t] = 2.0f * sl;
+                                    }
+                                    __half2 mb[8];
+#pragma unroll
+                                    for (int pos = 0; pos < 8; ++pos)
+                                        mb[pos] = h2dup(sl2[pos % SW] * __int_as_float((127 + 24 - pos) << 23));
+                                    dequant_segment_bits<GS, SW>(seg, rr, wg, acc, SW, mb);
+                                }
+                                if ((present >> J) & 1u) write_tile(cneg);
+                            }
+                        }
+                    };
+                    if (p.L.scale_mode == 1) {
+                        seg_step_free(std::integral_constant<int, 0>{});
+                        seg_step_free(std::integral_constant<int, 1>{});
+                        seg_step_free(std::integral_constant<int, 2>{});
+                        seg_step_free(std::integral_constant<int, 3>{});
+                    } else {
+                        seg_step(std::integral_constant<int, 0>{});
+                        seg_step(std::integral_constant<int, 1>{});
+                        seg_step(std::integral_constant<int, 2>{});
+                        seg_step(std::integral_constant<int, 3>{});
+                    }
                 } else {
                     const int smax = p.L.last_seg[kmax];         // stored segments 0..smax
                     if (p.L.scale_mode == 1) {
@@ -514,16 +556,24 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                                 else dequant_dispatch<GS, false>(sw, seg, rr, wg, acc, m0, u0);
                             } else {
                                 const uint32_t sc = wb + (uint32_t)tb.w + 2u * rr;       // this row's scale of the field's lowest bit
+                                // bit t of the field belongs to the step whose scale lies t planes before; the byte lane
+                                // holds 8 / sw fields, so position pos carries the scale of bit pos % sw
+                                float sl2[8];
+#pragma unroll
+                                for (int t = 0; t < 8; ++t) {
+                                    sl2[t] = 0.0f;
+                                    if (t < sw) {
+                                        unsigned short raw;
+                                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc - (uint32_t)(t * D2MOE_TILE_ROWS * 2)));
+                                        const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
+                                        cneg -= sl;                       // each step once
+                                        sl2[t] = 2.0f * sl;
+                                    }
+                                }
                                 __half2 mb[8];
 #pragma unroll
-                                for (int pos = 0; pos < 8; ++pos) {
-                                    const int t = pos % sw;               // bit of the field; its step's scale lies t planes before
-                                    unsigned short raw;
-                                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(sc - (uint32_t)(t * D2MOE_TILE_ROWS * 2)));
-                                    const float sl = __half2float(__ushort_as_half(raw)) * two_mS;
-                                    mb[pos] = h2dup(2.0f * sl * __int_as_float((127 + 24 - pos) << 23));
-                                    if (pos < sw) cneg -= sl;             // each step once
-                                }
+                                for (int pos = 0; pos < 8; ++pos)
+                                    mb[pos] = h2dup(sl2[pos & (sw - 1)] * __int_as_float((127 + 24 - pos) << 23));
                                 dequant_bits_dispatch<GS>(sw, seg, rr, wg, acc, sw, mb);
                             }
                             if (((tb.x >> 16) & 1) && ((present >> kk) & 1u)) write_tile(cneg);
@@ -944,8 +994,8 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         int wpack = 0;
-        // (compile-time segment offsets: tied-scale layout, every width step stored as one segment)
-        if (p.L.n_seg <= 4 && p.L.scale_mode == 0 && p.L.n_seg == p.L.n_widths)
+        // (every width step stored as one segment; the tied-scale layout has compile-time segment offsets)
+        if (p.L.n_seg <= 4 && p.L.n_seg == p.L.n_widths)
             for (int j = 0; j < p.L.n_seg; ++j) wpack |= p.L.seg_w[j] << (4 * j);
         auto launch = [&](auto kc) -> cudaError_t {
             constexpr auto kern = decltype(kc)::value;
