@@ -295,7 +295,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     if (warp == WARP_WPROD) {
         // ---------------- weight producer ----------------
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, wph = 0;
+            int ws = 0;
             int item = blockIdx.x;
             for (uint32_t qi = 0;; ++qi) {
                 const uint32_t q = qi & (NSQ - 1);
@@ -314,8 +315,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 if (p.mode == 0) { m0 = p.P.w[3 * e + 0]; m1 = p.P.w[3 * e + 1]; rt0 = rt1 = ii.tile; }
                 else { m0 = m1 = p.P.w[3 * e + 2]; rt0 = 2 * ii.tile; rt1 = 2 * ii.tile + 1; }
                 for (int G = ii.g0; G < ii.g1; ++G, ++it) {
-                    const int s = it % nsw;
-                    mbar_wait(W_EMPTY(s), ((it / nsw) & 1) ^ 1, abort_flag, p.status);
+                    const int s = ws;                                  // ring slot and parity advance by addition
+                    mbar_wait(W_EMPTY(s), wph ^ 1u, abort_flag, p.status);
+                    if (++ws == nsw) { ws = 0; wph ^= 1u; }
                     mbar_expect_tx(W_FULL(s), 2 * bytes);
                     const uint32_t dst = wbuf + s * w_slot_bytes;
                     bulk_g2s(dst, m0 + d2moe_block_offset(p.L, rt0, G), bytes, W_FULL(s));
@@ -436,6 +438,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (128 * 9);
         uint32_t it = 0, at = 0, ic = 0, eph = 0;       // eph: parity of the warpgroup's next exchange barrier phase
+        uint32_t wph = 0;                               // weight ring: slot and parity advance by addition
+        int ws = 0;
         __half2 acc[GS / 4];
         for (uint32_t qi = 0;; ++qi, ++ic) {
             const int item = pop(qi, true);
@@ -451,8 +455,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 
 #pragma unroll 1
             for (int G = ii.g0; G < ii.g1; ++G, ++it) {
-                const int s = it % nsw;
-                mbar_wait(W_FULL(s), (it / nsw) & 1, abort_flag, p.status);
+                const int s = ws;
+                mbar_wait(W_FULL(s), wph, abort_flag, p.status);
+                if (++ws == nsw) { ws = 0; wph ^= 1u; }
                 const uint32_t wb = wbuf + s * w_slot_bytes + blk * p.L.block_bytes;
                 uint32_t meta;
                 asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta) : "r"(wb + 4u * rr));
