@@ -65,6 +65,19 @@ struct TcParams {
     int smem_w_off, smem_epi_off, smem_bar_off;
 };
 
+// Packed half-precision arithmetic on raw 32-bit registers (a pair of halves each): the running tile lives in plain
+// registers, so nothing is moved between a bit pattern and a half2 value.
+__device__ __forceinline__ uint32_t hfma2_bits(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t hadd2_bits(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Dequantization of one K-half of one segment of one row into the running tile.
 //   seg     shared-memory address of the segment inside the block (this row's chunks are at
@@ -75,7 +88,7 @@ struct TcParams {
 //   FIRST   segment 0: the addend is u0 = (lo - s1/2) * 2^-S instead of acc
 // ------------------------------------------------------------------------------------------------
 template <int GS, int SW, bool FIRST>
-__device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], __half2 m0, __half2 u0) {
+__device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, uint32_t (&acc)[GS / 4], __half2 m0, __half2 u0) {
     constexpr int ROW_BYTES = GS * SW / 8;
     constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
     constexpr int HB = ROW_BYTES / 2;            // bytes of this half
@@ -109,9 +122,8 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, 
 #pragma unroll
             for (int e = 0; e < PER; ++e) {
                 const uint32_t src = (e & 1) ? hi8 : lo8;       // pair e of the word: bytes (0,2) or (1,3), bit SW*(e/2)
-                const __half2 code = as_h2(src & (FIELD << ((e >> 1) * SW)));
                 const int i = (l * WPL + q) * PER + e;
-                acc[i] = __hfma2(code, mult[e >> 1], FIRST ? u0 : acc[i]);
+                acc[i] = hfma2_bits(src & (FIELD << ((e >> 1) * SW)), as_u32(mult[e >> 1]), FIRST ? as_u32(u0) : acc[i]);
             }
         }
     }
@@ -122,7 +134,7 @@ __device__ __forceinline__ void dequant_segment(uint32_t seg, int rr, int half, 
 // W_hat = ... + s_l (2 bit_l - 1) is added when the tile is written).  mb[pos]: multiplier of a bit at position pos
 // of its byte lane, 2 s_l 2^(24 - S - pos) for the step that bit belongs to (0 for the unused bits of the field).
 template <int GS, int SW>
-__device__ __forceinline__ void dequant_segment_bits(uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], int W,
+__device__ __forceinline__ void dequant_segment_bits(uint32_t seg, int rr, int half, uint32_t (&acc)[GS / 4], int W,
                                                      const __half2 (&mb)[8]) {
     constexpr int ROW_BYTES = GS * SW / 8;
     constexpr int CS = ROW_BYTES < 16 ? ROW_BYTES : 16;
@@ -155,7 +167,7 @@ __device__ __forceinline__ void dequant_segment_bits(uint32_t seg, int rr, int h
                 for (int t = 0; t < SW; ++t) {
                     if (t < W) {
                         const int pos = (e >> 1) * SW + t;
-                        acc[i] = __hfma2(as_h2(src & (0x00010001u << pos)), mb[pos], acc[i]);
+                        acc[i] = hfma2_bits(src & (0x00010001u << pos), as_u32(mb[pos]), acc[i]);
                     }
                 }
             }
@@ -164,7 +176,7 @@ __device__ __forceinline__ void dequant_segment_bits(uint32_t seg, int rr, int h
 }
 
 template <int GS>
-__device__ __forceinline__ void dequant_bits_dispatch(int sw, uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], int W,
+__device__ __forceinline__ void dequant_bits_dispatch(int sw, uint32_t seg, int rr, int half, uint32_t (&acc)[GS / 4], int W,
                                                       const __half2 (&mb)[8]) {
     switch (sw) {
         case 1: dequant_segment_bits<GS, 1>(seg, rr, half, acc, W, mb); break;
@@ -175,7 +187,7 @@ __device__ __forceinline__ void dequant_bits_dispatch(int sw, uint32_t seg, int 
 }
 
 template <int GS, bool FIRST>
-__device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, int half, __half2 (&acc)[GS / 4], __half2 m0, __half2 u0) {
+__device__ __forceinline__ void dequant_dispatch(int sw, uint32_t seg, int rr, int half, uint32_t (&acc)[GS / 4], __half2 m0, __half2 u0) {
     switch (sw) {
         case 1: dequant_segment<GS, 1, FIRST>(seg, rr, half, acc, m0, u0); break;
         case 2: dequant_segment<GS, 2, FIRST>(seg, rr, half, acc, m0, u0); break;
@@ -434,13 +446,15 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         // ---------------- dequant + epilogue warps: warpgroup wg owns K-half wg of every tile ----------------
         const int wg = warp >> 2;
         const int r = threadIdx.x & 127;         // row of the tile = TMEM lane
-        const int blk = r >> 6, rr = r & 63;
+        // lanes 2i and 2i + 1 hold row i of the tile's first and second packed block (mode 0: the gate and the up row of
+        // one hidden unit, which the epilogue pairs with a shuffle)
+        const int blk = r & 1, rr = r >> 1;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (128 * 9);
         uint32_t it = 0, at = 0, ic = 0, eph = 0;       // eph: parity of the warpgroup's next exchange barrier phase
         uint32_t wph = 0;                               // weight ring: slot and parity advance by addition
         int ws = 0;
-        __half2 acc[GS / 4];
+        uint32_t acc[GS / 4];                           // the running tile: packed half pairs
         for (uint32_t qi = 0;; ++qi, ++ic) {
             const int item = pop(qi, true);
             if (item < 0) break;
@@ -474,10 +488,13 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     const uint32_t dst = a_tmem + slot * 64 + wg * (TILE_COLS / 2) + lane_addr;
 #pragma unroll
                     for (int c = 0; c < GS / 64; ++c) {
-                        uint32_t v[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = as_u32(__hadd2(acc[c * 16 + j], half_m));
-                        tc_st16(dst + c * 16, v);
+                        for (int h8 = 0; h8 < 2; ++h8) {
+                            uint32_t v[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] = hadd2_bits(acc[c * 16 + h8 * 8 + j], as_u32(half_m));
+                            tc_st8(dst + c * 16 + h8 * 8, v);
+                        }
                     }
                     tc_wait_st();
                     tc_fence_before();
@@ -639,22 +656,19 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                         hq[0] = b0.x; hq[1] = b0.y; hq[2] = b0.z; hq[3] = b0.w; hq[4] = b1.x; hq[5] = b1.y; hq[6] = b1.z; hq[7] = b1.w;
                     }
                     tc_wait_ld();
-                    // exchange: the gate thread publishes tokens 8..15, the up thread tokens 0..7
-                    const int give = blk == 0 ? 8 : 0;
+                    // exchange with the neighbouring lane (the other row of the hidden unit): the gate thread hands
+                    // over tokens 8..15, the up thread tokens 0..7, already times their own matrix's 2^S
+                    float other_v[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) epi[(blk * 64 + rr) * 9 + j] = __uint_as_float(v[give + j]) * two_S;
-                    // a bounded wait like every other one (after a timeout the warps of a warpgroup may leave
-                    // the queue at different items: no bar.sync inside the roles)
-                    mbar_arrive(EPI_BAR(wg));
-                    mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
-                    eph ^= 1u;
+                    for (int j = 0; j < 8; ++j)
+                        other_v[j] = __shfl_xor_sync(0xffffffffu, __uint_as_float(blk == 0 ? v[8 + j] : v[j]) * two_S, 1);
                     __half* dst = p.hbuf + (grow + keep) * p.D.F + (long long)ii.tile * 64 + rr;
                     bool over = false;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         if (keep + j < nreal) {
-                            const float mine = __uint_as_float(v[keep + j]) * two_S * xs[j];
-                            const float other = epi[((1 - blk) * 64 + rr) * 9 + j] * xs[j];
+                            const float mine = __uint_as_float(blk == 0 ? v[j] : v[8 + j]) * two_S * xs[j];
+                            const float other = other_v[j] * xs[j];
                             const float g = blk == 0 ? mine : other, up = blk == 0 ? other : mine;
                             float h = __fdividef(g, 1.0f + __expf(-g)) * up * hq[j];
                             // beyond fp16 even at the token's own scale (or not a number): stored as zero, call flagged
@@ -663,9 +677,6 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                         }
                     }
                     if (over && p.status) atomicOr(p.status, D2MOE_DEV_NONFINITE);
-                    mbar_arrive(EPI_BAR(wg));
-                    mbar_wait(EPI_BAR(wg), eph, abort_flag, p.status);
-                    eph ^= 1u;
                 } else {
                     float hs[16];                                // undoes the factor h was stored with
                     {
@@ -677,7 +688,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                         }
                     }
                     tc_wait_ld();
-                    float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + r;
+                    float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + blk * 64 + rr;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j < nreal) dst[(long long)j * p.D.d] = __uint_as_float(v[j]) * two_S * hs[j];
