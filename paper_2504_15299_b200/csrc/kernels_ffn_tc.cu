@@ -22,8 +22,9 @@
 // pack time) so that the multipliers stay inside fp16 range; the epilogue multiplies by 2^S.
 //
 // Warp roles (352 threads, 1 CTA per SM, all 512 TMEM columns): warps 0-3 and 4-7 are two dequant
-// warpgroups, each owning one K-half of every tile (thread = weight row = TMEM lane) and taking
-// alternate 16-column chunks of the epilogue; warp 8 streams packed blocks (cp.async.bulk), warp 9
+// warpgroups, each owning one K-half of every tile (thread = weight row = TMEM lane; lanes 2i and 2i + 1
+// hold row i of the tile's two packed blocks, for gate/up the two rows of one hidden unit, which the
+// epilogue pairs with a shuffle) and taking alternate 16-column chunks of the epilogue; warp 8 streams packed blocks (cp.async.bulk), warp 9
 // streams activation tiles (TMA, 128B swizzle, boxes of up to 256 rows), warp 10 issues the MMAs (the
 // whole warp runs the loop, one elected lane issues).  A unit holds up to 320 tokens, so that one
 // dequantization of a weight tile is amortised over enough tensor work to leave the kernel bound by
@@ -62,7 +63,7 @@ struct TcParams {
     const float* row_scale;   // [3][R]: per padded row the power-of-two factors of the activation scaling (see tc_gather_kernel)
     long long R_alloc;
     int32_t* status;
-    int smem_w_off, smem_epi_off, smem_bar_off;
+    int smem_w_off, smem_bar_off;
 };
 
 // Packed half-precision arithmetic on raw 32-bit registers (a pair of halves each): the running tile lives in plain
@@ -222,7 +223,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     constexpr int TILE_COLS = GS / 2;            // TMEM columns of one operand tile
     extern __shared__ uint8_t smem_raw[];
     // shared layout (from a 1024-byte boundary, which the 128B-swizzled operand tiles need):
-    // [activation ring: NSB x n_cap*GS*2] [weight ring: nsw x 2 blocks] [epilogue x2] [barriers]
+    // [activation ring: NSB x n_cap*GS*2] [weight ring: nsw x 2 blocks] [barriers]
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t b_slot_bytes = (uint32_t)p.n_cap * GS * 2;
@@ -247,7 +248,6 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
     static_assert(8 * (2 * MAX_NSW + 2 * NSB + 2 * A_SLOTS + 2) + 8 <= 160, "barrier block");
     auto SQ_FULL = [&](uint32_t i) { return bar0 + 160u + 8u * i; };
     auto SQ_EMPTY = [&](uint32_t i) { return bar0 + 192u + 8u * i; };
-    auto EPI_BAR = [&](int wg) { return bar0 + 224u + 8u * (uint32_t)wg; };     // SwiGLU exchange of a warpgroup (128 arrivals)
     volatile int* sq_item = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 240);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -259,7 +259,6 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         mbar_init(D_FULL, 1);
         mbar_init(D_EMPTY, 256);
         for (int i = 0; i < NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 10); }
-        for (int wg = 0; wg < 2; ++wg) mbar_init(EPI_BAR(wg), 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -450,8 +449,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
         // one hidden unit, which the epilogue pairs with a shuffle)
         const int blk = r & 1, rr = r >> 1;
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
-        float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (128 * 9);
-        uint32_t it = 0, at = 0, ic = 0, eph = 0;       // eph: parity of the warpgroup's next exchange barrier phase
+        uint32_t it = 0, at = 0, ic = 0;
         uint32_t wph = 0;                               // weight ring: slot and parity advance by addition
         int ws = 0;
         uint32_t acc[GS / 4];                           // the running tile: packed half pairs
@@ -996,16 +994,14 @@ cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const Pac
         p.hbuf = B.h16; p.obuf = B.o32; p.row_scale = B.slot_f; p.R_alloc = pl.R_alloc; p.status = device_status;
         const int b_bytes = NSB * pl.n_cap * D.g * 2;
         const int w_slot = 2 * p.L.block_bytes;
-        const int epi_bytes = 2 * 128 * 9 * 4;            // per warpgroup: 128 rows x 8 exchanged values (+1 pad)
         const int bar_bytes = 512;
         const int budget = 224 * 1024;
-        int nsw = (budget - b_bytes - epi_bytes - bar_bytes - 1024) / w_slot;
+        int nsw = (budget - b_bytes - bar_bytes - 1024) / w_slot;
         if (nsw > MAX_NSW) nsw = MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
         p.nsw = nsw;
         p.smem_w_off = b_bytes;
-        p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
-        p.smem_bar_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        p.smem_bar_off = (b_bytes + nsw * w_slot + 127) & ~127;
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;   // + slack for the 1024-byte alignment
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
