@@ -60,11 +60,10 @@ constexpr int I8_MAX_NSW = 8;                 // weight ring depth (upper bound)
 constexpr int I8_B_TILE = 2 * I8_SLOTS * 128; // 64 rows x 128 bytes (128 input columns)
 constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa) per slot, one group
 constexpr int I8_B_STAGE = I8_B_TILE + 2 * I8_XK_BYTES;
-constexpr int I8_EPI_STRIDE = 17;
 constexpr int I8_NSQ = 4;                     // entries of the work queue between the producer and the other warps
 // barriers: weight ring (full, empty), activation ring (full, empty), 4 + 4 hand-offs, 2 + 2 accumulators,
 // work queue (full, empty), 2 exchange barriers of the output phase
-constexpr int I8_N_BARS = 2 * I8_MAX_NSW + 2 * I8_NSB + 12 + 2 * I8_NSQ + 2;
+constexpr int I8_N_BARS = 2 * I8_MAX_NSW + 2 * I8_NSB + 12 + 2 * I8_NSQ;
 constexpr float I8_XMAX = 16191.0f;           // |xq| <= 126 * 128 + 63
 
 struct I8Params {
@@ -82,7 +81,7 @@ struct I8Params {
     float* obuf;              // [n_split][R_alloc, d]
     long long R_alloc;
     int32_t* status;
-    int smem_w_off, smem_epi_off, smem_rec_off, smem_bar_off;
+    int smem_w_off, smem_rec_off, smem_bar_off;
 };
 
 struct I8Item { int unit, tile, split, g0, g1; };
@@ -243,15 +242,11 @@ template <int WPACK> using I8SegList = WidthList<WPACK>;
 static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int r, int n_mine, uint32_t blks,
                                                  float (&acc)[4][4], uint8_t* smem) {
     const float* rec = reinterpret_cast<const float*>(smem + p.smem_rec_off) + ((threadIdx.x >> 5) - 4) * 40;
-    float* epi = reinterpret_cast<float*>(smem + p.smem_epi_off) + wg * (64 * I8_EPI_STRIDE);
-    // the warpgroup's exchange barrier (128 arrivals): two phases per work item, so the parities are always 0, 1;
-    // a bounded wait, like every other wait of the kernel
-    const uint32_t ebar = smem_u32(smem + p.smem_bar_off) + 8u * (uint32_t)(I8_N_BARS - 2 + wg);
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncwarp();
     const int slot0 = reinterpret_cast<const int*>(rec)[32];
     const int io_tile = reinterpret_cast<const int*>(rec)[33], io_split = reinterpret_cast<const int*>(rec)[34];
-    const int blk = r >> 6, rr = r & 63;
+    const int blk = r & 1, rr = r >> 1;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (i < n_mine) {
@@ -260,37 +255,32 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int 
         }
     }
     if (p.mode == 0) {
-        // rows r < 64 of the tile hold the gate projection, rows r >= 64 the up projection of the same 64 hidden
-        // units: the two halves exchange through shared memory so that each finishes half of the blocks
-        // (the gate half blocks 0 and 1 with the other's up values, the up half blocks 2 and 3 with the other's gate values)
+        // lanes 2i and 2i + 1 hold the gate and the up row of hidden unit i of the tile: the two exchange by
+        // shuffle so that each finishes half of the blocks (the gate lane blocks 0 and 1 with the other's up
+        // values, the up lane blocks 2 and 3 with the other's gate values)
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (i < n_mine && (blk == 1) == (i < 2))
+        for (int i = 0; i < 2; ++i) {
+            float other[4];
 #pragma unroll
-                for (int s = 0; s < 4; ++s) epi[rr * I8_EPI_STRIDE + 4 * i + s] = acc[i][s];
-        mbar_arrive(ebar);
-        mbar_wait_blk(ebar, 0);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i < n_mine && (blk == 0) == (i < 2)) {
-                float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
+            for (int s = 0; s < 4; ++s)
+                other[s] = __shfl_xor_sync(0xffffffffu, blk == 0 ? acc[i + 2][s] : acc[i][s], 1);
+            const int ib = blk == 0 ? i : i + 2;                 // the block this lane finishes
+            if (ib < n_mine) {
+                float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * ib)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
 #pragma unroll
                 for (int s = 0; s < 4; ++s) {
-                    const float other = epi[rr * I8_EPI_STRIDE + 4 * i + s];
-                    const float g = blk == 0 ? acc[i][s] : other;
-                    const float up = blk == 0 ? other : acc[i][s];
+                    const float g = blk == 0 ? acc[i][s] : other[s];
+                    const float up = blk == 0 ? other[s] : acc[i + 2][s];
                     dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
                 }
             }
         }
-        mbar_arrive(ebar);
-        mbar_wait_blk(ebar, 1);
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (i < n_mine) {
                 float* dst = p.obuf + (long long)io_split * p.R_alloc * p.D.d
-                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io_tile * 128 + r;
+                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io_tile * 128 + blk * 64 + rr;
 #pragma unroll
                 for (int s = 0; s < 4; ++s) dst[(long long)s * p.D.d] = acc[i][s];
             }
@@ -305,7 +295,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     constexpr int KSTEPS = GS / 32;            // MMAs (K = 32) per segment and group
     extern __shared__ uint8_t smem_raw[];
     // shared layout from a 1024-byte boundary:
-    // [activation tiles: I8_NSB x 8 KiB] [activation sums: I8_NSB x 512 B] [weight ring: nsw x GPS x 2 blocks] [epilogue x2] [barriers]
+    // [activation tiles: I8_NSB x 8 KiB] [activation sums: I8_NSB x 512 B] [weight ring: nsw x GPS x 2 blocks] [work-item records] [barriers]
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t w_slot_bytes = (uint32_t)(GPS * 2) * (uint32_t)p.L.block_bytes;
@@ -344,7 +334,6 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 8); }
         // a queue entry is released by the issuer warp, the four unpack warps and the eight fold warps
         for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 13); }
-        for (int wg = 0; wg < 2; ++wg) mbar_init(bar0 + 8u * (uint32_t)(I8_N_BARS - 2 + wg), 128);
         *abort_flag = 0;
         *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -519,7 +508,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // -------- unpack warpgroup: fills both operand slots of every group (slot 0: segments 0, 2, (4, 6); slot 1:
         // segments 1, 3, (5, 7)), one hand-off per slot --------
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
-        const int blk = r >> 6, rr = r & 63;
+        const int blk = r & 1, rr = r >> 1;         // lanes 2i, 2i + 1: row i of the tile's two packed blocks
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         uint32_t hs[2] = {0, 0};                   // hand-offs so far, per slot
         uint32_t ws = 0, wph = 0;
@@ -622,7 +611,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         // output phase --------
         const int wg = (warp >> 2) - 1;            // 0, 1
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
-        const int blk = r >> 6, rr = r & 63;
+        const int blk = r & 1, rr = r >> 1;         // lanes 2i, 2i + 1: row i of the tile's two packed blocks
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         const uint32_t d_base = d_tmem + lane_addr;
         uint32_t gc = 0;                           // groups folded so far
@@ -1101,17 +1090,15 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         const int gps = 128 / D.g;
         const int b_bytes = I8_NSB * I8_B_STAGE;
         const int w_slot = gps * 2 * p.L.block_bytes;
-        const int epi_bytes = 2 * 64 * I8_EPI_STRIDE * 4;
         const int bar_bytes = 512;
         const int budget = 112 * 1024;
         const int rec_bytes = 8 * 40 * 4;                             // per fold warp: the record of its work item
-        int nsw = (budget - b_bytes - epi_bytes - rec_bytes - 128 - bar_bytes - 1024) / w_slot;
+        int nsw = (budget - b_bytes - rec_bytes - 128 - bar_bytes - 1024) / w_slot;
         if (nsw > I8_MAX_NSW) nsw = I8_MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
         p.nsw = nsw;
         p.smem_w_off = b_bytes;
-        p.smem_epi_off = (b_bytes + nsw * w_slot + 127) & ~127;
-        p.smem_rec_off = (p.smem_epi_off + epi_bytes + 127) & ~127;
+        p.smem_rec_off = (b_bytes + nsw * w_slot + 127) & ~127;
         p.smem_bar_off = (p.smem_rec_off + rec_bytes + 511) & ~511;   // 512-byte aligned from the 1024-byte aligned base
         const int smem_bytes = p.smem_bar_off + bar_bytes + 1024;
         if (mode == 1)
