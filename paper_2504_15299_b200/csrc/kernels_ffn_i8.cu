@@ -62,7 +62,7 @@ constexpr int I8_XK_BYTES = I8_SLOTS * 8;     // (X, kappa) per slot, one group
 constexpr int I8_B_STAGE = I8_B_TILE + 2 * I8_XK_BYTES;
 constexpr int I8_NSQ = 4;                     // entries of the work queue between the producer and the other warps
 // barriers: weight ring (full, empty), activation ring (full, empty), 4 + 4 hand-offs, 2 + 2 accumulators,
-// work queue (full, empty), 2 exchange barriers of the output phase
+// work queue (full, empty)
 constexpr int I8_N_BARS = 2 * I8_MAX_NSW + 2 * I8_NSB + 12 + 2 * I8_NSQ;
 constexpr float I8_XMAX = 16191.0f;           // |xq| <= 126 * 128 + 63
 
