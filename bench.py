@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, each from one ncu capture of
 # the same workload through this script (the summaries of those captures are committed beside the numbers
 # they come from); key = workload:tokens:stage:path
-NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1043027576, "mixtral_decode:T64:down:auto": 535613024,
-               "mixtral_prefill:T2048:gate_up:auto": 1674879592, "mixtral_prefill:T2048:down:auto": 1022797248,
-               "finegrained:T256:gate_up:auto": 460187648, "finegrained:T256:down:auto": 234222848}
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1042331288, "mixtral_decode:T64:down:auto": 536724944,
+               "mixtral_prefill:T2048:gate_up:auto": 1649562264, "mixtral_prefill:T2048:down:auto": 1008650536,
+               "finegrained:T256:gate_up:auto": 463707392, "finegrained:T256:down:auto": 233998336}
 
 
 def measured_peaks():
