@@ -8,7 +8,10 @@
  *     memory.  The caller owns every buffer; the library allocates nothing and keeps no state
  *     between calls (unless an entry point's comment says otherwise).
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and the
- *     call returns without synchronising.
+ *     call returns without synchronising.  The kernels of one call are launched as programmatic
+ *     dependents of one another (each waits on the device for the one before it; the first kernel
+ *     of a call is an ordinary launch); the environment variable D2MOE_NO_PDL=1, read once, makes
+ *     every launch an ordinary one.
  *   - The return value reports what the host can see before and at launch: null pointers, bad
  *     configuration or shapes, short buffers, a failed launch.  Nothing is launched when an
  *     argument check fails.  Anomalies only the device can see (non-finite router logits, a bounded

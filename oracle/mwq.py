@@ -179,8 +179,8 @@ def quantize_calibrated(W: np.ndarray, bits: Sequence[int], group_size: int, hc:
     fp32 [cols, cols].  Reading of Algorithm 1 (its printed loop nest is garbled: the level loop never reaches
     K, W is changed inside it, E is divided by an index that is not a block): blocks are the quantization
     groups (gamma = g), taken left to right; a block is quantized at once through all its steps (Eq. 2, then
-    Eq. 4 with the scales of Eq. 5) - "only block-level compensation ... eliminating column-level error
-    corrections" (Section 3.3.1) -; its error at the top width, column j divided by H^c[j, j], is then taken
+    Eq. 4 with the scales of Eq. 5) - Section 3.3.1 says that errors are compensated per block, not per
+    column -; its error at the top width, column j divided by H^c[j, j], is then taken
     out of all later columns: W[:, later] -= E H^c[block, later].  All of it fp32, one rounding per operation,
     the update as g successive rank-one corrections in ascending column order (so that it is reproducible bit
     for bit).  PARITY UNPINNED as far as that reading goes; what is pinned: with a diagonal H^c nothing is

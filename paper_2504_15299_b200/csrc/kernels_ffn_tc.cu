@@ -352,6 +352,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 const ItemInfo ii = decode_item(p, item);
                 const TcUnit* u = p.units + ii.unit;
                 const int ncols = u->ncols;                       // multiple of 16, <= n_cap
+                const int row0 = u->row0;                         // read once: the copies below are issued back to back
                 const uint32_t bytes = (uint32_t)ncols * 128u * HALVES;
                 for (int G = ii.g0; G < ii.g1; ++G, ++it) {
                     const int s = it % NSB;
@@ -366,7 +367,7 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
 #pragma unroll
                             for (int h = 0; h < HALVES; ++h)
                                 tma_load_2d(dst + h * (uint32_t)p.n_cap * 128u + (uint32_t)r * 128u, &maps.m[mi],
-                                            G * GS + h * 64, u->row0 + r, B_FULL(s));
+                                            G * GS + h * 64, row0 + r, B_FULL(s));
                             r += box;
                         }
                     }
@@ -464,6 +465,8 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             const float two_mS = exp2f((float)-S);
             unsigned present = 0;
             for (int kk = 0; kk <= kmax; ++kk) present |= (u->cnt[kk] > 0 ? 1u : 0u) << kk;
+            const long long row0 = u->row0;                      // read here: the epilogue must not wait for it
+            const int ncols = u->ncols;
 
 #pragma unroll 1
             for (int G = ii.g0; G < ii.g1; ++G, ++it) {
@@ -629,8 +632,27 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             mbar_wait(D_FULL, ic & 1, abort_flag, p.status);
             tc_fence_after();
             const float two_S = exp2f((float)S);
-            const int ncols = u->ncols;
+            // the tokens' scale factors of a chunk (mode 0: xs of the eight tokens this thread finishes, then hq of the
+            // same; mode 1: hs of all sixteen) are fetched one chunk ahead
+            const int keep = blk == 0 ? 0 : 8;
+            auto load_scales = [&](int c0, float4 (&sc)[4]) {
+                const long long grow = row0 + c0;
+                if (p.mode == 0) {
+                    const float4* a = reinterpret_cast<const float4*>(p.row_scale + grow + keep);
+                    const float4* b = reinterpret_cast<const float4*>(p.row_scale + p.R_alloc + grow + keep);
+                    sc[0] = a[0]; sc[1] = a[1]; sc[2] = b[0]; sc[3] = b[1];
+                } else {
+                    const float4* a = reinterpret_cast<const float4*>(p.row_scale + 2 * p.R_alloc + grow);
+                    sc[0] = a[0]; sc[1] = a[1]; sc[2] = a[2]; sc[3] = a[3];
+                }
+            };
+            float4 sc_next[4];
+            if (wg * 16 < ncols) load_scales(wg * 16, sc_next);
             for (int c0 = wg * 16; c0 < ncols; c0 += 32) {
+                float4 sc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) sc[q] = sc_next[q];
+                if (c0 + 32 < ncols) load_scales(c0 + 32, sc_next);
                 int nreal = 0;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
@@ -640,16 +662,13 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 if (nreal == 0) continue;            // padding columns only (uniform across the warpgroup)
                 uint32_t v[16];
                 tc_ld16(d_tmem + lane_addr + c0, v);
-                const long long grow = u->row0 + c0;
+                const long long grow = row0 + c0;
                 if (p.mode == 0) {
                     // the tokens this thread finishes, and their scales: xs undoes the scaling of the activation
                     // row, hq is the factor h is stored with (both powers of two; 32-byte aligned: grow % 16 == 0)
-                    const int keep = blk == 0 ? 0 : 8;
                     float xs[8], hq[8];
                     {
-                        const float4* a = reinterpret_cast<const float4*>(p.row_scale + grow + keep);
-                        const float4* b = reinterpret_cast<const float4*>(p.row_scale + p.R_alloc + grow + keep);
-                        const float4 a0 = a[0], a1 = a[1], b0 = b[0], b1 = b[1];
+                        const float4 a0 = sc[0], a1 = sc[1], b0 = sc[2], b1 = sc[3];
                         xs[0] = a0.x; xs[1] = a0.y; xs[2] = a0.z; xs[3] = a0.w; xs[4] = a1.x; xs[5] = a1.y; xs[6] = a1.z; xs[7] = a1.w;
                         hq[0] = b0.x; hq[1] = b0.y; hq[2] = b0.z; hq[3] = b0.w; hq[4] = b1.x; hq[5] = b1.y; hq[6] = b1.z; hq[7] = b1.w;
                     }
@@ -678,10 +697,9 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                 } else {
                     float hs[16];                                // undoes the factor h was stored with
                     {
-                        const float4* a = reinterpret_cast<const float4*>(p.row_scale + 2 * p.R_alloc + grow);
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            const float4 t4 = a[q];
+                            const float4 t4 = sc[q];
                             hs[4 * q] = t4.x; hs[4 * q + 1] = t4.y; hs[4 * q + 2] = t4.z; hs[4 * q + 3] = t4.w;
                         }
                     }
