@@ -101,3 +101,43 @@ def test_guard_zones_survive_and_reruns_are_bit_identical(B, name, T):
     assert bool(torch.isfinite(y.float()).all().item())
     for g in guards + r_bufs + [ws, yg]:
         assert g.intact()
+
+
+_CHAIN_SCRIPT = r"""
+import hashlib, sys, torch
+from paper_2504_15299_b200 import binding as B, synth
+out = []
+for name, T in (("tiny", 24), ("mixtral_decode", 8)):
+    wl = synth.WORKLOADS[name]
+    cfg = B.Config.from_workload(wl)
+    blobs = []
+    for e in range(wl.n_experts + wl.n_shared):
+        for m in range(3):
+            blobs.append(B.pack_mwq(cfg, synth.expert_matrix(wl, e, m, device="cuda")))
+    x = synth.tokens_bf16(wl, T, "cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = B.moe_forward(cfg, x, blobs, gate_w=synth.gate_weight_bf16(wl, "cuda"),
+                      forced_bit_idx=synth.forced_bit_idx(wl, T, "cuda"), device_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    out.append(hashlib.sha256(y.view(torch.int16).cpu().numpy().tobytes()).hexdigest())
+print("HASH", " ".join(out))
+"""
+
+
+def test_ordinary_launches_give_the_same_bits_as_the_dependent_launch_chain(B):
+    """The kernels of a call are programmatic dependent launches; D2MOE_NO_PDL=1 (read once per process, hence the
+    child processes) makes them ordinary launches.  Both must give the same output bits."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    hashes = []
+    for flag in ("0", "1"):
+        env = dict(os.environ, D2MOE_NO_PDL=flag, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+        r = subprocess.run([sys.executable, "-c", _CHAIN_SCRIPT], env=env, cwd=root, capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        line = [ln for ln in r.stdout.splitlines() if ln.startswith("HASH")]
+        assert line, r.stdout[-2000:]
+        hashes.append(line[-1])
+    assert hashes[0] == hashes[1]
