@@ -621,20 +621,30 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
             }
 
             // ---- epilogue: D (128 rows x ncols) -> global; the two warpgroups take alternate 16-column chunks ----
-            // While it runs the tensor pipe is idle, so it is kept short: the pieces' extents are read once,
-            // and SwiGLU is split between the two threads of a hidden unit (the gate row's thread finishes the
-            // first eight tokens of a chunk, the up row's thread the other eight).
+            // While it runs the tensor pipe is idle, so it is kept short: a warp finishes two chunks at a time (two
+            // independent chains of tensor-memory load, shuffle, SwiGLU and stores), their scale factors are fetched a
+            // pair ahead, and SwiGLU is split between the two threads of a hidden unit (the gate row's thread
+            // finishes the first eight tokens of a chunk, the up row's thread the other eight).  Padding columns
+            // (their activation rows and scale factors are never written) are neither stored nor checked.
             int pc0[8], pcn[8], prl[8];                          // per piece: first column, columns, real columns
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 pc0[kk] = u->col0[kk]; pcn[kk] = kk <= kmax ? u->cnt[kk] : 0; prl[kk] = u->real[kk];
             }
+            auto nreal_of = [&](int c0) -> int {               // real tokens among the 16 columns from c0
+                int nreal = 0;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const int rel = c0 - pc0[kk];
+                    if (pcn[kk] > 0 && rel >= 0 && rel < pcn[kk]) nreal = min(16, max(0, prl[kk] - rel));
+                }
+                return nreal;
+            };
             mbar_wait(D_FULL, ic & 1, abort_flag, p.status);
             tc_fence_after();
             const float two_S = exp2f((float)S);
-            // the tokens' scale factors of a chunk (mode 0: xs of the eight tokens this thread finishes, then hq of the
-            // same; mode 1: hs of all sixteen) are fetched one chunk ahead
             const int keep = blk == 0 ? 0 : 8;
+            // mode 0: xs of the eight tokens this thread finishes, then hq of the same; mode 1: hs of all sixteen
             auto load_scales = [&](int c0, float4 (&sc)[4]) {
                 const long long grow = row0 + c0;
                 if (p.mode == 0) {
@@ -646,33 +656,13 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     sc[0] = a[0]; sc[1] = a[1]; sc[2] = a[2]; sc[3] = a[3];
                 }
             };
-            float4 sc_next[4];
-            if (wg * 16 < ncols) load_scales(wg * 16, sc_next);
-            for (int c0 = wg * 16; c0 < ncols; c0 += 32) {
-                float4 sc[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) sc[q] = sc_next[q];
-                if (c0 + 32 < ncols) load_scales(c0 + 32, sc_next);
-                int nreal = 0;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const int rel = c0 - pc0[kk];
-                    if (pcn[kk] > 0 && rel >= 0 && rel < pcn[kk]) nreal = min(16, max(0, prl[kk] - rel));
-                }
-                if (nreal == 0) continue;            // padding columns only (uniform across the warpgroup)
-                uint32_t v[16];
-                tc_ld16(d_tmem + lane_addr + c0, v);
+            uint32_t overbits = 0;                               // largest |h| seen, as bits (a NaN above every number)
+            auto finish = [&](int c0, const uint32_t (&v)[16], const float4 (&sc)[4]) {
                 const long long grow = row0 + c0;
+                const int nreal = nreal_of(c0);
                 if (p.mode == 0) {
-                    // the tokens this thread finishes, and their scales: xs undoes the scaling of the activation
-                    // row, hq is the factor h is stored with (both powers of two; 32-byte aligned: grow % 16 == 0)
-                    float xs[8], hq[8];
-                    {
-                        const float4 a0 = sc[0], a1 = sc[1], b0 = sc[2], b1 = sc[3];
-                        xs[0] = a0.x; xs[1] = a0.y; xs[2] = a0.z; xs[3] = a0.w; xs[4] = a1.x; xs[5] = a1.y; xs[6] = a1.z; xs[7] = a1.w;
-                        hq[0] = b0.x; hq[1] = b0.y; hq[2] = b0.z; hq[3] = b0.w; hq[4] = b1.x; hq[5] = b1.y; hq[6] = b1.z; hq[7] = b1.w;
-                    }
-                    tc_wait_ld();
+                    const float xs[8] = {sc[0].x, sc[0].y, sc[0].z, sc[0].w, sc[1].x, sc[1].y, sc[1].z, sc[1].w};
+                    const float hq[8] = {sc[2].x, sc[2].y, sc[2].z, sc[2].w, sc[3].x, sc[3].y, sc[3].z, sc[3].w};
                     // exchange with the neighbouring lane (the other row of the hidden unit): the gate thread hands
                     // over tokens 8..15, the up thread tokens 0..7, already times their own matrix's 2^S
                     float other_v[8];
@@ -680,36 +670,47 @@ ffn_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ TmaMap
                     for (int j = 0; j < 8; ++j)
                         other_v[j] = __shfl_xor_sync(0xffffffffu, __uint_as_float(blk == 0 ? v[8 + j] : v[j]) * two_S, 1);
                     __half* dst = p.hbuf + (grow + keep) * p.D.F + (long long)ii.tile * 64 + rr;
-                    bool over = false;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
+                        const float mine = __uint_as_float(blk == 0 ? v[j] : v[8 + j]) * two_S * xs[j];
+                        const float other = other_v[j] * xs[j];
+                        const float g = blk == 0 ? mine : other, up = blk == 0 ? other : mine;
+                        float h = __fdividef(g, 1.0f + __expf(-g)) * up * hq[j];
                         if (keep + j < nreal) {
-                            const float mine = __uint_as_float(blk == 0 ? v[j] : v[8 + j]) * two_S * xs[j];
-                            const float other = other_v[j] * xs[j];
-                            const float g = blk == 0 ? mine : other, up = blk == 0 ? other : mine;
-                            float h = __fdividef(g, 1.0f + __expf(-g)) * up * hq[j];
-                            // beyond fp16 even at the token's own scale (or not a number): stored as zero, call flagged
-                            if (!(fabsf(h) <= 65504.0f)) { h = 0.0f; over = true; }
+                            const uint32_t hb = __float_as_uint(h) & 0x7fffffffu;
+                            overbits = max(overbits, hb);
+                            // beyond fp16 even at the token's own scale (or not a number): stored as zero, call flagged below
+                            if (hb > 0x477fe000u) h = 0.0f;                  // bits of 65504
                             dst[(long long)j * p.D.F] = __float2half_rn(h);
                         }
                     }
-                    if (over && p.status) atomicOr(p.status, D2MOE_DEV_NONFINITE);
                 } else {
-                    float hs[16];                                // undoes the factor h was stored with
-                    {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float4 t4 = sc[q];
-                            hs[4 * q] = t4.x; hs[4 * q + 1] = t4.y; hs[4 * q + 2] = t4.z; hs[4 * q + 3] = t4.w;
-                        }
-                    }
-                    tc_wait_ld();
+                    const float hs[16] = {sc[0].x, sc[0].y, sc[0].z, sc[0].w, sc[1].x, sc[1].y, sc[1].z, sc[1].w,
+                                          sc[2].x, sc[2].y, sc[2].z, sc[2].w, sc[3].x, sc[3].y, sc[3].z, sc[3].w};
                     float* dst = p.obuf + (long long)ii.split * p.R_alloc * p.D.d + grow * p.D.d + (long long)ii.tile * 128 + blk * 64 + rr;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j < nreal) dst[(long long)j * p.D.d] = __uint_as_float(v[j]) * two_S * hs[j];
                 }
+            };
+            float4 sa_next[4], sb_next[4];
+            if (wg * 16 < ncols) load_scales(wg * 16, sa_next);
+            if (wg * 16 + 32 < ncols) load_scales(wg * 16 + 32, sb_next);
+            for (int c0 = wg * 16; c0 < ncols; c0 += 64) {
+                const bool two = c0 + 32 < ncols;
+                uint32_t va[16], vb[16];
+                tc_ld16(d_tmem + lane_addr + c0, va);
+                if (two) tc_ld16(d_tmem + lane_addr + c0 + 32, vb);
+                float4 sa[4], sb[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { sa[q] = sa_next[q]; sb[q] = sb_next[q]; }
+                if (c0 + 64 < ncols) load_scales(c0 + 64, sa_next);
+                if (c0 + 96 < ncols) load_scales(c0 + 96, sb_next);
+                tc_wait_ld();
+                finish(c0, va, sa);
+                if (two) finish(c0 + 32, vb, sb);
             }
+            if (p.mode == 0 && overbits > 0x477fe000u && p.status) atomicOr(p.status, D2MOE_DEV_NONFINITE);
             tc_fence_before();
             mbar_arrive(D_EMPTY);
         }
