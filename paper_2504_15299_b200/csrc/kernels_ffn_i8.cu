@@ -314,10 +314,13 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     auto D_EMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 10 + b); };
     auto SQ_FULL = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 12 + i); };
     auto SQ_EMPTY = [&](int i) { return bar0 + 8u * (uint32_t)(2 * I8_MAX_NSW + 2 * I8_NSB + 12 + I8_NSQ + i); };
-    static_assert(8 * I8_N_BARS + 4 * I8_NSQ <= 488, "barrier block");
+    static_assert(8 * I8_N_BARS + 8 * I8_NSQ <= 488, "barrier block");
     // work queue entries (after the barriers): the producer takes work items from a global counter and
     // publishes them here, so that CTAs that drew cheap items take more of them
     volatile int* sq_item = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 8 * I8_N_BARS);
+    // ... and with every entry the item's last operand (kmax of its unit), which the unpack warps need before they can
+    // start: the producer reads the unit one item ahead, so they start without a trip to global memory
+    volatile int* sq_kmax = sq_item + I8_NSQ;
     // tail of the 512-byte barrier block: TMEM base (488), device-status pointer (496), abort flag (504)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 488);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 504);
@@ -364,17 +367,23 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             // ring positions advance by addition, nothing is recomputed per stage.
             uint32_t it = 0, ws = 0, wph = 1, bs = 0, bph = 1;         // ring positions, parity of the "empty" waits
             int item = blockIdx.x;
+            // the fields of the item's unit that this thread needs, read one item ahead
+            int u_e = 0, u_kmax = 0, u_nslots = 0, u_slot0 = 0;
+            if (item < total_items) {
+                const I8Unit* u0 = p.units + i8_item(p, item).unit;
+                u_e = u0->e; u_kmax = u0->kmax; u_nslots = u0->nslots; u_slot0 = u0->slot0;
+            }
             for (uint32_t qi = 0;; ++qi) {
                 const uint32_t q = qi & (I8_NSQ - 1);
                 mbar_wait_blk(SQ_EMPTY(q), ((qi / I8_NSQ) & 1u) ^ 1u);
                 if (item >= total_items) item = -1;                    // the end mark
                 sq_item[q] = item;
+                sq_kmax[q] = u_kmax;
                 mbar_arrive(SQ_FULL(q));
                 if (item < 0) break;
                 const int next = atomicAdd(p.next_item, 1);            // in flight while this item's stages are issued
                 const I8Item ii = i8_item(p, item);
-                const I8Unit* u = p.units + ii.unit;
-                const int e = u->e, kmax = u->kmax;
+                const int e = u_e, kmax = u_kmax;
                 // kmax: the unit's last width step (specialised kernels: a step is one operand) or its last stored segment
                 const uint32_t bytes = (uint32_t)(SWPACK != 0 ? d2moe_prefix_bytes(p.L, kmax) : p.L.seg_off[kmax + 1]);
                 const uint8_t *m0, *m1;
@@ -385,7 +394,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                     m0 = p.P.w[3 * e + 2] + d2moe_block_offset(p.L, 2 * ii.tile, ii.g0);
                     m1 = p.P.w[3 * e + 2] + d2moe_block_offset(p.L, 2 * ii.tile + 1, ii.g0);
                 }
-                const int nslots = u->nslots, slot0 = u->slot0;
+                const int nslots = u_nslots, slot0 = u_slot0;
                 const int mi = nslots <= 8 ? 0 : (nslots <= 16 ? 1 : 2);        // boxes of 16, 32, 64 rows
                 const uint32_t tile_bytes = (16u << mi) * 128u;
                 const uint32_t xk_bytes = (uint32_t)nslots * 8u;
@@ -393,6 +402,10 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 const float* xk_src = p.xk + ((long long)ii.g0 * p.R_alloc + slot0) * 2;
                 const long long xk_step = p.R_alloc * 2;
                 const CUtensorMap* map = &maps.m[mi];
+                if (next < total_items) {                              // the next item's unit: in flight during the stage loop
+                    const I8Unit* un = p.units + i8_item(p, next).unit;
+                    u_e = un->e; u_kmax = un->kmax; u_nslots = un->nslots; u_slot0 = un->slot0;
+                }
                 for (int G = ii.g0; G < ii.g1; G += GPS, ++it) {
                     const int ng = min(GPS, ii.g1 - G);
                     {
@@ -517,11 +530,11 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             const uint32_t q = qi & (I8_NSQ - 1);
             mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
             const int item = sq_item[q];
+            const int kmax = sq_kmax[q];
             __syncwarp();
             if (lane == 0) mbar_arrive(SQ_EMPTY(q));
             if (item < 0) break;
             const I8Item ii = i8_item(p, item);
-            const int kmax = p.units[ii.unit].kmax;
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
                 mbar_wait_blk(W_FULL(ws), wph);
