@@ -296,6 +296,7 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
     cudaError_t e;
     auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
     mark(0);
+    bool want_defer = false, group_deferred = false;
     if (pre) {
         R = RouteBufs{(int32_t*)pre->topk_idx, (float*)pre->topk_w, (int8_t*)pre->bit_idx,
                       (int32_t*)pre->perm, (int32_t*)pre->inv_perm, (int32_t*)pre->group_off};
@@ -303,10 +304,16 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
         R = RouteBufs{(int32_t*)(w + ws.off_topk_idx), (float*)(w + ws.off_topk_w), (int8_t*)(w + ws.off_bit_idx),
                       (int32_t*)(w + ws.off_perm), (int32_t*)(w + ws.off_inv_perm),
                       (int32_t*)(w + ws.off_group_off)};
+        // decode-sized loads on the 8-bit kernel: the grouping runs in front of that path's unit build, in one launch
+        if (use_tensor_path(c)) {
+            TcPlan pl0;
+            tc_plan(c, T, &pl0);
+            want_defer = pl0.decode != 0;
+        }
         e = launch_route(D, (const __nv_bfloat16*)x, (const __nv_bfloat16*)in->gate_w_bf16, in->logits,
                          (const __nv_bfloat16*)in->bit_w_bf16, in->forced_bit_idx, R,
                          (float*)(w + ws.off_logits), (int32_t*)(w + ws.off_keys),
-                         (int32_t*)(w + ws.off_hist), device_status, st);
+                         (int32_t*)(w + ws.off_hist), device_status, st, want_defer ? &group_deferred : nullptr);
         if (e != cudaSuccess) return D2MOE_ERR_CUDA;
     }
     ExpertPtrs P;
@@ -326,7 +333,8 @@ static d2moe_status forward_impl(const d2moe_config* c, int64_t T, const void* x
         B.xp16 = (__half*)(w + ws.off_xp16); B.h16 = (__half*)(w + ws.off_h); B.o32 = (float*)(w + ws.off_o);
         B.h32 = (float*)(w + ws.off_h32); B.xk_x = (float*)(w + ws.off_xk_x); B.xk_h = (float*)(w + ws.off_xk_h);
         B.slot_f = (float*)(w + ws.off_slot_f);
-        e = pl.decode ? launch_ffn_i8(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev)
+        e = pl.decode ? launch_ffn_i8(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev,
+                                      group_deferred ? (const int32_t*)(w + ws.off_keys) : nullptr)
                       : launch_ffn_tensor(c, D, Lgu, Ld, P, (const __nv_bfloat16*)x, R, pl, B, device_status, st, ev);
         if (e != cudaSuccess) return D2MOE_ERR_CUDA;
         mark(3);
@@ -382,6 +390,11 @@ extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int 
     const long long A = (long long)T * c->top_k, n_keys = (long long)c->n_experts * c->n_bits;
     const bool small = A <= 8192 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 1024;
     int route = routing_precomputed ? 0 : (small || d2moe_group_is_mid(A, n_keys) ? 2 : 4);
+    if (!routing_precomputed && small && use_tensor_path(c)) {          // grouping inside the decode path's unit build
+        TcPlan pl0;
+        tc_plan(c, T, &pl0);
+        if (pl0.decode) route -= 1;
+    }
     // more than 16 experts: the gate logits come from a tiled kernel of their own (when the caller supplies
     // logits instead of gate weights that launch does not happen: the count is then one too high)
     if (!routing_precomputed && c->n_experts > 16 && (size_t)c->d_model * 2 * 16 <= 200 * 1024) route += 1;

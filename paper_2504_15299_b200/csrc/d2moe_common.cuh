@@ -224,7 +224,11 @@ cudaError_t launch_unpack_scales(const PackLayout& L, const uint8_t* packed, flo
 cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
                          const float* logits_in, const __nv_bfloat16* bit_w, const int8_t* forced,
                          const RouteBufs& R, float* logits_ws, int32_t* keys_ws, int32_t* hist_ws,
-                         int32_t* device_status, cudaStream_t st);
+                         int32_t* device_status, cudaStream_t st, bool* defer_small_group = nullptr);
+// the single-block grouping rule of launch_route (decode-sized loads)
+static inline bool d2moe_group_is_small(long long A, long long n_keys) {
+    return A <= 8192 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 1024;
+}
 
 // kernels_ffn_cc.cu  (plain CUDA-core path)
 cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, const ExpertPtrs& P,

@@ -45,6 +45,7 @@
 #include "d2moe_common.cuh"
 #include "kernels_ffn_tc.cuh"
 #include "tc_common.cuh"
+#include "group_block.cuh"
 
 #include <type_traits>
 
@@ -753,12 +754,18 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // items from a counter, take the cheap ones last; sets both work counters (n_units[1], n_units[2]) to
 // the grid size of those kernels.
 // Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
                int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status,
-               I8SegMap sm) {
+               I8SegMap sm, const int32_t* group_keys) {
     pdl_enter();
     extern __shared__ int32_t s_prep[];
+    // decode-sized loads: the grouping of the assignments by (expert, width) first, in this launch (the routing
+    // kernels left it to this one); its results are read below after a barrier, by this same block
+    if (group_keys) {
+        group_block_body(D.A, D.E * D.K, group_keys, R.group_off, R.perm, R.inv_perm, s_prep, 0, 1);
+        __syncthreads();
+    }
     __shared__ int s_total;
     const int n_exp = D.E + D.n_shared, n_keys = D.E * D.K;
     int32_t* go = s_prep;                          // group_off
@@ -1059,7 +1066,8 @@ static int i8_wpack(const MoeDims& D) {
 
 cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                           const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
-                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev) {
+                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev,
+                          const int32_t* group_keys) {
     auto mark = [&](int i) { if (ev) cudaEventRecord((cudaEvent_t)ev[i], st); };
     const int n_exp = D.E + D.n_shared;
     I8Unit* units = reinterpret_cast<I8Unit*>(B.units);
@@ -1071,7 +1079,11 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
 
     const int ffn_grid = 2 * device_sm_count();
-    const size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
+    size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
+    if (group_keys) {                       // the grouping's staging area shares the buffer (at most 41 KB: decode-sized loads)
+        const size_t gsm = (size_t)(((D.A + 31) & ~31) + D.E * D.K + 1) * 4;
+        if (gsm > prep_smem) prep_smem = gsm;
+    }
     // operands of the expert kernels: the width steps themselves when the list has a specialised kernel (the fields of
     // a step are merged in registers), otherwise the stored segments one by one
     const int wp = i8_wpack(D);
@@ -1079,8 +1091,8 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     I8SegMap sm;
     sm.n_seg = by_step ? D.K : Lgu.n_seg;
     for (int j = 0; j < 8; ++j) sm.seg_kk[j] = by_step ? j : Lgu.seg_kk[j];
-    launch_chained(i8_prep_kernel, dim3(1), dim3(256), prep_smem, st, D, R, units, B.n_units, B.pad_off, B.row_map, B.src_token, kappa,
-                                      pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status, sm);
+    launch_chained(i8_prep_kernel, dim3(1), dim3(group_keys ? 512 : 256), prep_smem, st, D, R, units, B.n_units, B.pad_off, B.row_map,
+                   B.src_token, kappa, pl.max_units, Lgu.top, Lgu.b1, ffn_grid, device_status, sm, group_keys);
     // threads per slot: a quarter of the row's cells, in whole warps
     auto q_threads = [](int n) { const int t = ((n / 4 + I8_QCPT - 1) / I8_QCPT + 31) & ~31; return t < 1024 ? t : 1024; };
     launch_chained(i8_quant_kernel<true>, dim3(q_blocks), dim3(q_threads(D.d)), 0, st, D.d, D.g, pl.R_alloc, x, B.src_token, B.pad_off, n_exp, kappa,

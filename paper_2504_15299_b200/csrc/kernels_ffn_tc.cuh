@@ -57,6 +57,9 @@ void tc_plan(const d2moe_config* c, long long T, TcPlan* pl);
 cudaError_t launch_ffn_tensor(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                               const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
                               const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
+// group_keys: when not null, the sort keys of the assignments whose grouping (group_off, perm, inv_perm of R) is
+// still to be done: the unit build does it first, in the same launch
 cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLayout& Lgu, const PackLayout& Ld,
                           const ExpertPtrs& P, const __nv_bfloat16* x, const RouteBufs& R, const TcPlan& pl,
-                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev);
+                          const TcBuffers& B, int32_t* device_status, cudaStream_t st, void* const* ev,
+                          const int32_t* group_keys = nullptr);

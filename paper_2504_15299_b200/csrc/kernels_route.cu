@@ -2,6 +2,7 @@
 // grouping of assignments by (expert, width); its histogram is B_{j,k} of Section 3.4.3.
 #include "d2moe_common.cuh"
 #include "tc_common.cuh"
+#include "group_block.cuh"
 
 namespace {
 
@@ -203,58 +204,7 @@ group_block_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t*
                  int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
     pdl_enter();
     extern __shared__ int32_t s_grp[];
-    int32_t* s_keys = s_grp;
-    int32_t* s_off = s_grp + ((A + 31) & ~31);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int a = threadIdx.x; a < A; a += blockDim.x) s_keys[a] = keys[a];
-    __syncthreads();
-    for (int key = warp; key < n_keys; key += n_warps) {
-        int cnt = 0;
-        for (int base = 0; base < A; base += 32) {
-            const int a = base + lane;
-            cnt += __popc(__ballot_sync(0xffffffffu, a < A && s_keys[a] == key));
-        }
-        if (lane == 0) s_off[key] = cnt;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        int carry = 0;
-        for (int base = 0; base < n_keys; base += 32) {
-            const int i = base + lane;
-            const int v = i < n_keys ? s_off[i] : 0;
-            int incl = v;
-            for (int off = 1; off < 32; off <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += o;
-            }
-            if (i < n_keys) {
-                s_off[i] = carry + incl - v;
-                if (blockIdx.x == 0) group_off[i] = carry + incl - v;
-            }
-            carry += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (lane == 0) {
-            s_off[n_keys] = carry;
-            if (blockIdx.x == 0) group_off[n_keys] = carry;
-        }
-    }
-    __syncthreads();
-    // this block's keys, spread over its warps
-    for (int key = blockIdx.x + warp * gridDim.x; key < n_keys; key += n_warps * gridDim.x) {
-        int pos = s_off[key];
-        if (pos == s_off[key + 1]) continue;
-        for (int base = 0; base < A; base += 32) {
-            const int a = base + lane;
-            const bool m = a < A && s_keys[a] == key;
-            const unsigned bal = __ballot_sync(0xffffffffu, m);
-            if (m) {
-                const int p = pos + __popc(bal & ((1u << lane) - 1u));
-                perm[p] = a;
-                inv_perm[a] = p;
-            }
-            pos += __popc(bal);
-        }
-    }
+    group_block_body(A, n_keys, keys, group_off, perm, inv_perm, s_grp, blockIdx.x, gridDim.x);
 }
 
 // Same dot product with both vectors already in shared memory.
@@ -399,7 +349,7 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
 cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bfloat16* gate_w,
                          const float* logits_in, const __nv_bfloat16* bit_w, const int8_t* forced,
                          const RouteBufs& R, float* logits_ws, int32_t* keys_ws, int32_t* hist_ws,
-                         int32_t* device_status, cudaStream_t st) {
+                         int32_t* device_status, cudaStream_t st, bool* defer_small_group) {
     const int warps_per_block = 4;
     const int n_keys = D.E * D.K;
     // block-per-token kernel when the token row plus at least one weight row fit in shared memory
@@ -431,8 +381,9 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
         D, x, gate_w, logits_in, bit_w, forced, R, keys_ws, device_status);
     // few assignments and keys: histogram, scan and scatter in one single-block launch (beyond about a
     // thousand warp walks the three grid-wide kernels are faster: 39 vs 10 us at 192 keys x 1536 assignments)
-    const long long walks = (long long)n_keys * ((D.A + 31) / 32);
-    const bool small = D.A <= 8192 && n_keys <= 2048 && walks <= 1024;
+    const bool small = d2moe_group_is_small(D.A, n_keys);
+    // the caller runs the single-block grouping in front of its next kernel (one launch instead of two)
+    if (small && defer_small_group) { *defer_small_group = true; return cudaGetLastError(); }
     if (small || d2moe_group_is_mid(D.A, n_keys)) {
         const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
         cudaError_t e = ensure_dynamic_smem<&group_block_kernel>((int)gsm);
