@@ -322,6 +322,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     // ... and with every entry the item's last operand (kmax of its unit), which the unpack warps need before they can
     // start: the producer reads the unit one item ahead, so they start without a trip to global memory
     volatile int* sq_kmax = sq_item + I8_NSQ;
+    // ... and the slots each operand's product covers (npad of the unit), which the issuer needs (after the fold warps' records)
+    volatile int* sq_npad = reinterpret_cast<volatile int*>(smem + p.smem_rec_off + 8 * 40 * 4);
     // tail of the 512-byte barrier block: TMEM base (488), device-status pointer (496), abort flag (504)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 488);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(reinterpret_cast<uint8_t*>(bars) + 504);
@@ -369,10 +371,12 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             uint32_t it = 0, ws = 0, wph = 1, bs = 0, bph = 1;         // ring positions, parity of the "empty" waits
             int item = blockIdx.x;
             // the fields of the item's unit that this thread needs, read one item ahead
-            int u_e = 0, u_kmax = 0, u_nslots = 0, u_slot0 = 0;
+            int u_e = 0, u_kmax = 0, u_nslots = 0, u_slot0 = 0, u_npad[8] = {0, 0, 0, 0, 0, 0, 0, 0};
             if (item < total_items) {
                 const I8Unit* u0 = p.units + i8_item(p, item).unit;
                 u_e = u0->e; u_kmax = u0->kmax; u_nslots = u0->nslots; u_slot0 = u0->slot0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) u_npad[j] = u0->npad[j];
             }
             for (uint32_t qi = 0;; ++qi) {
                 const uint32_t q = qi & (I8_NSQ - 1);
@@ -380,6 +384,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 if (item >= total_items) item = -1;                    // the end mark
                 sq_item[q] = item;
                 sq_kmax[q] = u_kmax;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sq_npad[8 * q + j] = u_npad[j];
                 mbar_arrive(SQ_FULL(q));
                 if (item < 0) break;
                 const int next = atomicAdd(p.next_item, 1);            // in flight while this item's stages are issued
@@ -406,6 +412,8 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 if (next < total_items) {                              // the next item's unit: in flight during the stage loop
                     const I8Unit* un = p.units + i8_item(p, next).unit;
                     u_e = un->e; u_kmax = un->kmax; u_nslots = un->nslots; u_slot0 = un->slot0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) u_npad[j] = un->npad[j];
                 }
                 for (int G = ii.g0; G < ii.g1; G += GPS, ++it) {
                     const int ng = min(GPS, ii.g1 - G);
@@ -458,15 +466,14 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             const uint32_t q = qi & (I8_NSQ - 1);
             mbar_wait_blk(SQ_FULL(q), (qi / I8_NSQ) & 1u);
             const int item = sq_item[q];
-            __syncwarp();
+            const int kmax = sq_kmax[q];
+            uint32_t idesc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) idesc[j] = instr_desc_i8(2 * max(sq_npad[8 * q + j], 8));
+            __syncwarp();                                       // the entry is released after its last read
             if (lane == 0) mbar_arrive(SQ_EMPTY(q));
             if (item < 0) break;
             const I8Item ii = i8_item(p, item);
-            const I8Unit* u = p.units + ii.unit;
-            const int kmax = u->kmax;
-            uint32_t idesc[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) idesc[j] = instr_desc_i8(2 * max(u->npad[j], 8));
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
                 mbar_wait_blk(B_FULL(bs), bph);
@@ -1117,7 +1124,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         const int w_slot = gps * 2 * p.L.block_bytes;
         const int bar_bytes = 512;
         const int budget = 112 * 1024;
-        const int rec_bytes = 8 * 40 * 4;                             // per fold warp: the record of its work item
+        const int rec_bytes = 8 * 40 * 4 + I8_NSQ * 8 * 4;            // per fold warp: the record of its work item; per queue entry: npad
         int nsw = (budget - b_bytes - rec_bytes - 128 - bar_bytes - 1024) / w_slot;
         if (nsw > I8_MAX_NSW) nsw = I8_MAX_NSW;
         if (nsw < 2) return cudaErrorInvalidConfiguration;
