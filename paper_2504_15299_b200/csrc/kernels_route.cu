@@ -217,12 +217,16 @@ __device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const _
     return acc;
 }
 
+// Copies d elements (a multiple of 8; both ends 16-byte aligned) into shared memory with asynchronous 16-byte copies:
+// every copy of a block is in flight at once (one trip to memory instead of one per few registers).  The data may
+// be read after stage_wait() and a barrier.
 __device__ __forceinline__ void stage_row(__nv_bfloat16* dst, const __nv_bfloat16* __restrict__ src, int d) {
     const uint4* s = reinterpret_cast<const uint4*>(src);
-    uint4* t = reinterpret_cast<uint4*>(dst);
-#pragma unroll 4
-    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
+    const uint32_t t = smem_u32(dst);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(t + 16u * (uint32_t)i), "l"(s + i) : "memory");
 }
+__device__ __forceinline__ void stage_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Gate logits for many experts: a block stages TB token rows and EB weight rows once and forms the
 // TB x EB dot products (pinned order), so a weight row is read once per TB tokens instead of per token.
@@ -238,6 +242,7 @@ gate_logits_kernel(int T, int E, int d, const __nv_bfloat16* __restrict__ x, con
     const int nt = min(TB, T - t0), ne = min(EB, E - e0);
     stage_row(xs, x + (size_t)t0 * d, nt * d);                 // consecutive rows are contiguous: one copy loop each
     stage_row(ws, gate_w + (size_t)e0 * d, ne * d);
+    stage_wait();
     __syncthreads();
     for (int pr = warp; pr < nt * ne; pr += 8) {
         const int tt = pr / ne, ee = pr - tt * ne;
@@ -268,11 +273,13 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
     if (!(logits_in && forced)) stage_row(xs, x + (size_t)t * D.d, D.d);
     if (logits_in) {
         for (int e = threadIdx.x; e < E; e += blockDim.x) lg_s[e] = logits_in[(size_t)t * E + e];
+        stage_wait();
         __syncthreads();
     } else {
         for (int eb = 0; eb < E; eb += EB) {
             const int n = min(EB, E - eb);
             stage_row(ws, gate_w + (size_t)eb * D.d, n * D.d);       // the n rows are contiguous: one copy loop
+            stage_wait();
             __syncthreads();
             for (int r = warp; r < n; r += 8) {
                 const float v = dot_pinned_smem(xs, ws + (size_t)r * D.d, D.d, lane);
@@ -309,6 +316,7 @@ route_block_kernel(MoeDims D, const __nv_bfloat16* __restrict__ x, const __nv_bf
                 const int s = (rb + r) / D.K, c = (rb + r) - s * D.K;
                 stage_row(ws + (size_t)r * D.d, bit_w + ((size_t)sel_s[s] * D.K + c) * D.d, D.d);
             }
+            stage_wait();
             __syncthreads();
             for (int r = warp; r < n; r += 8) {
                 const float v = dot_pinned_smem(xs, ws + (size_t)r * D.d, D.d, lane);
