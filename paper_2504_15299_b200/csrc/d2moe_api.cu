@@ -389,8 +389,8 @@ extern "C" int d2moe_forward_launch_count(const d2moe_config* c, int64_t T, int 
     // route, then count + scan + scatter (one launch when the load is small: the rule of launch_route)
     const long long A = (long long)T * c->top_k, n_keys = (long long)c->n_experts * c->n_bits;
     const bool small = A <= 8192 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 1024;
-    int route = routing_precomputed ? 0 : (small || d2moe_group_is_mid(A, n_keys) ? 2 : 4);
-    if (!routing_precomputed && small && use_tensor_path(c)) {          // grouping inside the decode path's unit build
+    int route = routing_precomputed ? 0 : (small || d2moe_group_is_sortable(A, n_keys) || d2moe_group_is_mid(A, n_keys) ? 2 : 4);
+    if (!routing_precomputed && (small || d2moe_group_is_sortable(A, n_keys)) && use_tensor_path(c)) {   // grouping inside the decode path's unit build
         TcPlan pl0;
         tc_plan(c, T, &pl0);
         if (pl0.decode) route -= 1;

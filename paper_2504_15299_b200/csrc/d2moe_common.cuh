@@ -193,8 +193,9 @@ struct RouteBufs {
 };
 
 // Grouping of the assignments by (expert, width) key: the single-block kernel takes the smallest loads (its
-// rule is in launch_route), one launch of a few blocks the mid-sized ones (every block counts all keys: the
-// walks per warp must stay short), histogram + scan + scatter kernels the rest.
+// rule is in launch_route), a single-block counting sort loads of up to 4096 assignments on up to 512 keys, one
+// launch of a few blocks the other mid-sized ones (every block counts all keys: the walks per warp must stay
+// short), histogram + scan + scatter kernels the rest.  All give the same (unique) stable order.
 static inline bool d2moe_group_is_mid(long long A, long long n_keys) {
     return A <= 12288 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 6144;
 }
@@ -229,6 +230,11 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
 static inline bool d2moe_group_is_small(long long A, long long n_keys) {
     return A <= 8192 && n_keys <= 2048 && n_keys * ((A + 31) / 32) <= 1024;
 }
+// loads that one block groups by a counting sort (in front of the decode path's unit build)
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+static inline bool d2moe_group_is_sortable(long long A, long long n_keys) { return A <= 4096 && n_keys <= 512; }
 
 // kernels_ffn_cc.cu  (plain CUDA-core path)
 cudaError_t launch_gateup_cuda_core(const MoeDims& D, const PackLayout& Lgu, const ExpertPtrs& P,

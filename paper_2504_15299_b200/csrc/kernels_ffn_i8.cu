@@ -770,7 +770,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     // decode-sized loads: the grouping of the assignments by (expert, width) first, in this launch (the routing
     // kernels left it to this one); its results are read below after a barrier, by this same block
     if (group_keys) {
-        group_block_body(D.A, D.E * D.K, group_keys, R.group_off, R.perm, R.inv_perm, s_prep, 0, 1);
+        if (d2moe_group_is_sortable(D.A, D.E * D.K)) group_sort_body(D.A, D.E * D.K, group_keys, R.group_off, R.perm, R.inv_perm, s_prep);
+        else group_block_body(D.A, D.E * D.K, group_keys, R.group_off, R.perm, R.inv_perm, s_prep, 0, 1);
         __syncthreads();
     }
     __shared__ int s_total;
@@ -1087,9 +1088,14 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
 
     const int ffn_grid = 2 * device_sm_count();
     size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
-    if (group_keys) {                       // the grouping's staging area shares the buffer (at most 41 KB: decode-sized loads)
-        const size_t gsm = (size_t)(((D.A + 31) & ~31) + D.E * D.K + 1) * 4;
+    if (group_keys) {                       // the grouping's staging area shares the buffer
+        const size_t gsm = d2moe_group_is_sortable(D.A, D.E * D.K) ? group_sort_smem_ints(D.A, D.E * D.K, 512 / 32) * 4
+                                                                   : (size_t)(((D.A + 31) & ~31) + D.E * D.K + 1) * 4;
         if (gsm > prep_smem) prep_smem = gsm;
+    }
+    {
+        cudaError_t e = ensure_dynamic_smem<&i8_prep_kernel>((int)prep_smem);
+        if (e != cudaSuccess) return e;
     }
     // operands of the expert kernels: the width steps themselves when the list has a specialised kernel (the fields of
     // a step are merged in registers), otherwise the stored segments one by one

@@ -207,6 +207,15 @@ group_block_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t*
     group_block_body(A, n_keys, keys, group_off, perm, inv_perm, s_grp, blockIdx.x, gridDim.x);
 }
 
+// One block, counting sort: up to a few thousand assignments on up to 512 keys (see group_block.cuh).
+__global__ void __launch_bounds__(1024)
+group_sort_kernel(int A, int n_keys, const int32_t* __restrict__ keys, int32_t* __restrict__ group_off,
+                  int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+    pdl_enter();
+    extern __shared__ int32_t s_grp[];
+    group_sort_body(A, n_keys, keys, group_off, perm, inv_perm, s_grp);
+}
+
 // Same dot product with both vectors already in shared memory.
 __device__ __forceinline__ float dot_pinned_smem(const __nv_bfloat16* a, const __nv_bfloat16* b, int d, int lane) {
     float acc = 0.0f;
@@ -391,7 +400,15 @@ cudaError_t launch_route(const MoeDims& D, const __nv_bfloat16* x, const __nv_bf
     // thousand warp walks the three grid-wide kernels are faster: 39 vs 10 us at 192 keys x 1536 assignments)
     const bool small = d2moe_group_is_small(D.A, n_keys);
     // the caller runs the single-block grouping in front of its next kernel (one launch instead of two)
-    if (small && defer_small_group) { *defer_small_group = true; return cudaGetLastError(); }
+    if ((small || d2moe_group_is_sortable(D.A, n_keys)) && defer_small_group) { *defer_small_group = true; return cudaGetLastError(); }
+    if (!small && d2moe_group_is_sortable(D.A, n_keys)) {
+        const int threads = D.A >= 2048 ? 1024 : 512;
+        const size_t gsm = group_sort_smem_ints(D.A, n_keys, threads / 32) * 4;
+        cudaError_t e = ensure_dynamic_smem<&group_sort_kernel>((int)gsm);
+        if (e != cudaSuccess) return e;
+        launch_chained(group_sort_kernel, dim3(1), dim3(threads), gsm, st, D.A, n_keys, keys_ws, R.group_off, R.perm, R.inv_perm);
+        return cudaGetLastError();
+    }
     if (small || d2moe_group_is_mid(D.A, n_keys)) {
         const size_t gsm = (size_t)(((D.A + 31) & ~31) + n_keys + 1) * 4;
         cudaError_t e = ensure_dynamic_smem<&group_block_kernel>((int)gsm);
