@@ -760,7 +760,8 @@ __device__ __forceinline__ int round8(int n) { return (n + 7) & ~7; }
 // Then orders the units by decreasing work per group, so that the expert kernels, whose CTAs draw work
 // items from a counter, take the cheap ones last; sets both work counters (n_units[1], n_units[2]) to
 // the grid size of those kernels.
-// Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints).
+// Shared memory: group_off (E K + 1 ints), per expert its first unit (n_exp + 1 ints), per unit its cost (max_units ints),
+// the padded slot offsets (n_exp + 1 ints).
 __global__ void __launch_bounds__(512)
 i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad_off, int32_t* row_map,
                int32_t* src_token, float* kappa, int max_units, int top, int b1, int ffn_grid, int32_t* status,
@@ -779,6 +780,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     int32_t* go = s_prep;                          // group_off
     int32_t* unit_off = s_prep + n_keys + 1;
     int32_t* cost = unit_off + n_exp + 1;
+    int32_t* s_pad = cost + max_units;             // pad_off, kept here too (read back below without a trip to global memory)
     for (int i = threadIdx.x; i <= n_keys; i += blockDim.x) go[i] = R.group_off[i];
     __syncthreads();
     if (threadIdx.x < 32) {                       // padded slot offsets and first units (one warp scans)
@@ -799,12 +801,12 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
                 const int uo = __shfl_up_sync(0xffffffffu, uincl, off);
                 if (lane >= off) { incl += o; uincl += uo; }
             }
-            if (e < n_exp) { pad_off[e] = carry + incl - v; unit_off[e] = ucarry + uincl - nu; }
+            if (e < n_exp) { pad_off[e] = carry + incl - v; s_pad[e] = carry + incl - v; unit_off[e] = ucarry + uincl - nu; }
             carry += __shfl_sync(0xffffffffu, incl, 31);
             ucarry += __shfl_sync(0xffffffffu, uincl, 31);
         }
         if (lane == 0) {
-            pad_off[n_exp] = carry; s_total = carry; unit_off[n_exp] = ucarry;
+            pad_off[n_exp] = carry; s_pad[n_exp] = carry; s_total = carry; unit_off[n_exp] = ucarry;
             n_units[0] = min(ucarry, max_units);
             n_units[1] = ffn_grid; n_units[2] = ffn_grid;
         }
@@ -825,7 +827,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         }
         int start = 0;                            // classes of a larger width index come first
         for (int i = kk + 1; i < D.K; ++i) start += round8(go[e * D.K + i + 1] - go[e * D.K + i]);
-        const int slot = pad_off[e] + start + (pos - go[e * D.K + kk]);
+        const int slot = s_pad[e] + start + (pos - go[e * D.K + kk]);
         // pos must lie inside the group of (e, kk); otherwise the permutation does not belong to these indices
         if (pos < go[e * D.K + kk] || pos >= go[e * D.K + kk + 1] || slot < 0 || slot >= total) {
             row_map[a] = -1;
@@ -838,7 +840,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     }
     for (int i = threadIdx.x; i < D.n_shared * D.T; i += blockDim.x) {
         const int s = i / D.T, t = i - s * D.T;
-        const int slot = pad_off[D.E + s] + t;
+        const int slot = s_pad[D.E + s] + t;
         row_map[D.A + i] = slot;
         src_token[slot] = t;
         kappa[slot] = 0.5f - exp2f((float)(top - b1 - 1));
@@ -846,7 +848,8 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     // one thread per unit (an expert with many tokens, a shared one above all, has many units): the unit's
     // expert is the last one whose first unit is not beyond it
     const int n_all = min(unit_off[n_exp], max_units);
-    for (int nu = threadIdx.x; nu < n_all; nu += blockDim.x) {
+    I8Unit mine[4];                               // this thread's first four units stay in registers for the ordering below
+    for (int nu = threadIdx.x, mk = 0; nu < n_all; nu += blockDim.x, ++mk) {
         int lo_e = 0, hi_e = n_exp - 1;
         while (lo_e < hi_e) {
             const int mid = (lo_e + hi_e + 1) >> 1;
@@ -854,7 +857,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
         }
         while (lo_e + 1 < n_exp && unit_off[lo_e + 1] <= nu) ++lo_e;       // skip experts without units
         const int e = lo_e;
-        const int p0 = pad_off[e], len_e = pad_off[e + 1] - p0;
+        const int p0 = s_pad[e], len_e = s_pad[e + 1] - p0;
         int cnt[8], cpad[9];                      // cpad[j]: padded slots of the classes with index >= j
         cpad[D.K] = 0;
         for (int j = D.K - 1; j >= 0; --j) {
@@ -876,7 +879,14 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
                 for (int b = a0 / 4; 4 * b < a1; ++b)
                     if (u.nblk < 8) u.blk[u.nblk++] = b - start / 4;
             }
-            units[nu] = u;                        // every window starts with a real token: never empty
+            // every window starts with a real token: never empty.  With few units the list is ordered below and
+            // written then; otherwise it is written here, in the order it was built
+            if (n_all > 4 * (int)blockDim.x) units[nu] = u;
+            else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (mk == k) mine[k] = u;
+            }
             // work per group: one warpgroup unpacks every operand, each of the other two folds half of the blocks
             cost[nu] = 80 * (u.kmax + 1) + 25 * ((u.nblk + 1) / 2);
         }
@@ -884,14 +894,12 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
     __syncthreads();
     const int n = min(unit_off[n_exp], max_units);
     if (n <= 4 * (int)blockDim.x) {              // rank by (cost descending, index ascending), then permute
-        I8Unit mine[4];
         int rank[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int i = threadIdx.x + k * blockDim.x;
             rank[k] = -1;
             if (i < n) {
-                mine[k] = units[i];
                 const int c = cost[i];
                 int rk = 0;
                 for (int j = 0; j < n; ++j) rk += (cost[j] > c || (cost[j] == c && j < i)) ? 1 : 0;
@@ -1087,7 +1095,7 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
     const int q_blocks = (int)(pl.R_alloc < 1184 ? pl.R_alloc : 1184);
 
     const int ffn_grid = 2 * device_sm_count();
-    size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units) * 4;
+    size_t prep_smem = (size_t)(D.E * D.K + 1 + n_exp + 1 + pl.max_units + n_exp + 1) * 4;
     if (group_keys) {                       // the grouping's staging area shares the buffer
         const size_t gsm = d2moe_group_is_sortable(D.A, D.E * D.K) ? group_sort_smem_ints(D.A, D.E * D.K, 512 / 32) * 4
                                                                    : (size_t)(((D.A + 31) & ~31) + D.E * D.K + 1) * 4;
