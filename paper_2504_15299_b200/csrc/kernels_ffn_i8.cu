@@ -27,13 +27,14 @@
 //   * The accumulator is double buffered per group: while the products of group G+1 run, the
 //     fold warps add group G to their fp32 registers.
 //
-// CTA = 448 threads, 2 CTAs per SM (72 registers per thread); thread = weight row = TMEM lane in every
-// warpgroup.  Warps 0-3 unpack: per group they fill operand slot 0 (segments 0 and 2 of the group, two
-// 32-column tiles in TMEM) and hand it to the issuer, then slot 1 (segments 1 and 3).  Warps 4-7 and 8-11
-// fold: each warpgroup takes half of the unit's token blocks and, at the end of a work item, half of the
-// output phase.  Warp 12 streams packed blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and
-// the per-group activation sums, warp 13 issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns +
-// 4 x 32 operand columns.
+// Two instantiations per width list, 2 CTAs per SM either way; thread = weight row = TMEM lane in every warpgroup.
+// Warps 0-3 unpack: per group they fill operand slot 0 (segments 0 and 2 of the group, two 32-column tiles in TMEM)
+// and hand it to the issuer, then slot 1 (segments 1 and 3).  Then the fold warps: two warpgroups (CTA = 448
+// threads, 72 registers), each taking half of the unit's token blocks, when the units are full; one warpgroup
+// (CTA = 320 threads, 96 registers) that takes all blocks when a unit holds few tokens (fewer waiting warps: 4-5 %
+// faster up to about 12 tokens per expert, slower beyond).  The fold warps also run the output phase of a work item.
+// Then one warp that streams packed blocks (cp.async.bulk), activation tiles (TMA, 128B swizzle) and the per-group
+// activation sums, and one that issues the MMAs.  TMEM per CTA: 2 x 64 accumulator columns + 4 x 32 operand columns.
 //
 // Work distribution: a work item is one unit x one tile of 128 weight rows x a range of groups.  The
 // producer thread takes item numbers from a global counter (which starts at the grid size: item i < grid
@@ -51,8 +52,10 @@
 
 namespace {
 
-constexpr int I8_THREADS = 448;
-constexpr int I8_WARP_PROD = 12, I8_WARP_MMA = 13;
+// Warps: 0-3 unpack, then NF fold warpgroups (1 or 2), the producer warp, the issuer warp.  Two fold warpgroups
+// (each half of the unit's token blocks, 72 registers) win when the units are full; one (all blocks, 96 registers,
+// fewer waiting warps) when a unit holds few tokens.
+__host__ __device__ constexpr int i8_threads(int nf) { return 32 * (4 + 4 * nf + 2); }
 constexpr int I8_TMEM_COLS = 256;
 constexpr int I8_D_COLS = 64;                 // one accumulator buffer: 32 slots x (high, low)
 constexpr int I8_SLOTS = 32;                  // token slots per unit
@@ -236,52 +239,56 @@ __device__ __forceinline__ void unpack_dispatch(int sw, uint32_t seg, int rr, in
 template <int WPACK> using I8SegList = WidthList<WPACK>;
 
 // Output phase of one work item for one thread: scales the folded sums by the tokens' activation
-// scales, applies SwiGLU across the gate / up halves of the tile (mode 0) and writes the result.
-// blks: byte i = first slot / 4 of the thread's block i.  rec: the warp's record of the work item in shared
-// memory (words 0..31: activation scale of the unit's slots, copied asynchronously when the item began;
-// 32: first slot, 33: tile, 34: split), so that the phase starts without a trip to global memory.
-static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int r, int n_mine, uint32_t blks,
-                                                 float (&acc)[4][4], uint8_t* smem) {
+// scales, applies SwiGLU across the gate / up rows of a hidden unit (mode 0) and writes the result.
+// blks_lo / blks_hi: byte i = first slot / 4 of block i (blocks 0..3, 4..7).  rec: the warp's record of the work
+// item in shared memory (words 0..31: activation scale of the unit's slots, copied asynchronously when the item
+// began; 32: first slot, 33: tile, 34: split), so that the phase starts without a trip to global memory.
+template <int NB>
+static __device__ __noinline__ void i8_write_out(const I8Params& p, int r, int n_mine, uint32_t blks_lo, uint32_t blks_hi,
+                                                 float (&acc)[NB][4], uint8_t* smem) {
     const float* rec = reinterpret_cast<const float*>(smem + p.smem_rec_off) + ((threadIdx.x >> 5) - 4) * 40;
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncwarp();
     const int slot0 = reinterpret_cast<const int*>(rec)[32];
     const int io_tile = reinterpret_cast<const int*>(rec)[33], io_split = reinterpret_cast<const int*>(rec)[34];
     const int blk = r & 1, rr = r >> 1;
+    auto blk_of = [&](int i) -> uint32_t { return ((i < 4 ? blks_lo : blks_hi) >> (8 * (i & 3))) & 255u; };
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NB; ++i) {
         if (i < n_mine) {
-            const float4 sg = *reinterpret_cast<const float4*>(rec + 4 * ((blks >> (8 * i)) & 255u));
+            const float4 sg = *reinterpret_cast<const float4*>(rec + 4 * blk_of(i));
             acc[i][0] *= sg.x; acc[i][1] *= sg.y; acc[i][2] *= sg.z; acc[i][3] *= sg.w;
         }
     }
     if (p.mode == 0) {
         // lanes 2i and 2i + 1 hold the gate and the up row of hidden unit i of the tile: the two exchange by
-        // shuffle so that each finishes half of the blocks (the gate lane blocks 0 and 1 with the other's up
-        // values, the up lane blocks 2 and 3 with the other's gate values)
+        // shuffle so that each finishes half of the blocks (the gate lane the even blocks with the other's up
+        // values, the up lane the odd blocks with the other's gate values)
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            float other[4];
+        for (int i = 0; i < NB / 2; ++i) {
+            if (2 * i < n_mine) {                                // uniform across the warp
+                float other[4];
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
-                other[s] = __shfl_xor_sync(0xffffffffu, blk == 0 ? acc[i + 2][s] : acc[i][s], 1);
-            const int ib = blk == 0 ? i : i + 2;                 // the block this lane finishes
-            if (ib < n_mine) {
-                float* dst = p.hbuf + (long long)(slot0 + 4 * ((blks >> (8 * ib)) & 255u)) * p.D.F + (long long)io_tile * 64 + rr;
+                for (int s = 0; s < 4; ++s)
+                    other[s] = __shfl_xor_sync(0xffffffffu, blk == 0 ? acc[2 * i + 1][s] : acc[2 * i][s], 1);
+                const int ib = 2 * i + blk;                      // the block this lane finishes
+                if (ib < n_mine) {
+                    float* dst = p.hbuf + (long long)(slot0 + 4 * blk_of(ib)) * p.D.F + (long long)io_tile * 64 + rr;
 #pragma unroll
-                for (int s = 0; s < 4; ++s) {
-                    const float g = blk == 0 ? acc[i][s] : other[s];
-                    const float up = blk == 0 ? other[s] : acc[i + 2][s];
-                    dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
+                    for (int s = 0; s < 4; ++s) {
+                        const float g = blk == 0 ? acc[2 * i][s] : other[s];
+                        const float up = blk == 0 ? other[s] : acc[2 * i + 1][s];
+                        dst[(long long)s * p.D.F] = g / (1.0f + __expf(-g)) * up;
+                    }
                 }
             }
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < NB; ++i) {
             if (i < n_mine) {
                 float* dst = p.obuf + (long long)io_split * p.R_alloc * p.D.d
-                           + (long long)(slot0 + 4 * ((blks >> (8 * i)) & 255u)) * p.D.d + (long long)io_tile * 128 + blk * 64 + rr;
+                           + (long long)(slot0 + 4 * blk_of(i)) * p.D.d + (long long)io_tile * 128 + blk * 64 + rr;
 #pragma unroll
                 for (int s = 0; s < 4; ++s) dst[(long long)s * p.D.d] = acc[i][s];
             }
@@ -289,9 +296,11 @@ static __device__ __noinline__ void i8_write_out(const I8Params& p, int wg, int 
     }
 }
 
-template <int GS, int SWPACK>
-__global__ void __launch_bounds__(I8_THREADS, 2)
+template <int GS, int SWPACK, int NF>
+__global__ void __launch_bounds__(i8_threads(NF), 2)
 ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMaps maps) {
+    constexpr int I8_WARP_PROD = 4 + 4 * NF, I8_WARP_MMA = 5 + 4 * NF;
+    constexpr int NB = 8 / NF;                 // token blocks a fold warpgroup takes at most
     constexpr int GPS = 128 / GS;              // groups per ring stage (a stage spans 128 input columns)
     constexpr int KSTEPS = GS / 32;            // MMAs (K = 32) per segment and group
     extern __shared__ uint8_t smem_raw[];
@@ -331,15 +340,15 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 12); }
+        for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 4 + 4 * NF); }
         // an activation stage is released by the MMA issuer (its products have read the tile) and by
         // the eight folding warps (they have read the sums)
-        for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 9); }
+        for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 1 + 4 * NF); }
         for (int wg = 0; wg < 2; ++wg)
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 4); mbar_init(A_EMPTY(wg, sl), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 4 * NF); }
         // a queue entry is released by the issuer warp, the four unpack warps and the eight fold warps
-        for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 13); }
+        for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 5 + 4 * NF); }
         *abort_flag = 0;
         *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -627,10 +636,10 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
             }
         }
-    } else if (warp < 12) {
-        // -------- two fold warpgroups: every group's accumulator into fp32 sums, each for half of the token blocks;
-        // output phase --------
-        const int wg = (warp >> 2) - 1;            // 0, 1
+    } else if (warp < 4 + 4 * NF) {
+        // -------- the fold warpgroups: every group's accumulator into fp32 sums; with two warpgroups each takes half of the
+        // unit's token blocks (at most 4), one takes all (at most 8); output phase --------
+        const int wg = (warp >> 2) - 1;            // 0 .. NF - 1
         const int r = threadIdx.x & 127;           // row of the tile = TMEM lane
         const int blk = r & 1, rr = r >> 1;         // lanes 2i, 2i + 1: row i of the tile's two packed blocks
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
@@ -662,16 +671,21 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 }
             }
             const int h0 = (nblk + 1) >> 1;
-            const int n_mine = wg == 0 ? h0 : nblk - h0;        // my token blocks (at most 4)
-            uint32_t myblks = 0;                                 // byte i: first slot / 4 of my block i
+            const int f0 = (NF == 2 && wg == 1) ? h0 : 0;        // my first block
+            const int n_mine = NF == 2 ? (wg == 0 ? h0 : nblk - h0) : nblk;     // my token blocks (at most NB)
+            uint32_t myblks[2] = {0, 0};                         // byte i of word i / 4: first slot / 4 of my block i
 #pragma unroll
-            for (int i = 0; i < 4; ++i) myblks |= (uint32_t)u->blk[min((wg == 0 ? 0 : h0) + i, 7)] << (8 * i);
-            uint32_t blk_r[4];
+            for (int i = 0; i < NB; ++i) myblks[i >> 2] |= (uint32_t)u->blk[min(f0 + i, 7)] << (8 * (i & 3));
+            uint32_t blk_r[NB];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) blk_r[i] = (myblks >> (8 * i)) & 255u;
-            float acc[4][4];
+            for (int i = 0; i < NB; ++i) blk_r[i] = (myblks[i >> 2] >> (8 * (i & 3))) & 255u;
+            // the round (of two blocks) after whose loads the accumulator is released: with one fold warpgroup the last
+            // one that loads anything (up to four rounds), with two always the second (a warpgroup without blocks of
+            // its own still releases)
+            const int last_rd = NF == 1 ? (n_mine > 0 ? (n_mine - 1) >> 1 : 0) : NB / 2 - 1;
+            float acc[NB][4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < NB; ++i)
 #pragma unroll
                 for (int s = 0; s < 4; ++s) acc[i][s] = 0.0f;
 
@@ -713,18 +727,21 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                                 acc[b][s] = fmaf(cx, xk[2 * s], acc[b][s]);
                             }
                         };
-                        // two rounds of two blocks, one set of loaded values at a time (registers)
+                        // rounds of two blocks, one set of loaded values at a time (registers); the accumulator is released
+                        // as soon as the last round's values are in registers
 #pragma unroll
-                        for (int rd = 0; rd < 2; ++rd) {
-                            uint32_t v[2][8];
+                        for (int rd = 0; rd < NB / 2; ++rd) {
+                            if (rd <= last_rd) {
+                                uint32_t v[2][8];
 #pragma unroll
-                            for (int i = 0; i < 2; ++i)
-                                if (2 * rd + i < n_mine) tc_ld8(d_addr + 8 * blk_r[2 * rd + i], v[i]);
-                            tc_wait_ld();
-                            if (rd == 1) { tc_fence_before(); __syncwarp(); if (lane == 0) mbar_arrive(D_EMPTY(buf)); }
+                                for (int i = 0; i < 2; ++i)
+                                    if (2 * rd + i < n_mine) tc_ld8(d_addr + 8 * blk_r[2 * rd + i], v[i]);
+                                tc_wait_ld();
+                                if (rd == last_rd) { tc_fence_before(); __syncwarp(); if (lane == 0) mbar_arrive(D_EMPTY(buf)); }
 #pragma unroll
-                            for (int i = 0; i < 2; ++i)
-                                if (2 * rd + i < n_mine) fold_block(2 * rd + i, v[i]);
+                                for (int i = 0; i < 2; ++i)
+                                    if (2 * rd + i < n_mine) fold_block(2 * rd + i, v[i]);
+                            }
                         }
                         ++gc;
                     }
@@ -735,12 +752,12 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
             }
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
-            float out[4][4];                   // a copy: acc itself must stay in registers
+            float out[NB][4];                  // a copy: acc itself must stay in registers
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < NB; ++i)
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) out[i][q4] = acc[i][q4];
-            i8_write_out(p, wg, r, n_mine, myblks, out, smem);
+            i8_write_out<NB>(p, r, n_mine, myblks[0], myblks[1], out, smem);
         }
     }
 
@@ -1153,20 +1170,27 @@ cudaError_t launch_ffn_i8(const d2moe_config* c, const MoeDims& D, const PackLay
         mark(mode == 0 ? 1 : 2);
         // width lists of at most four segments that have a specialised kernel (nibble j = width of segment j)
         const int wpack = i8_wpack(D);
+        // fold warpgroups: one when a unit is expected to hold few tokens (measured crossover on the Mixtral shape:
+        // about 14 tokens per expert), two when the units are full (shared experts take every token)
+        const long long per_expert = ((long long)D.A + D.E - 1) / D.E;
+        const long long per_unit = D.n_shared > 0 ? (D.T < 32 ? D.T : 32) : 0;
+        const int nf = (per_expert <= 12 && per_unit <= 12) ? 1 : 2;
         auto launch = [&](auto kc) -> cudaError_t {
             constexpr auto kern = decltype(kc)::value;
             cudaError_t err = ensure_dynamic_smem<kern>(smem_bytes);
             if (err != cudaSuccess) return err;
-            launch_chained(kern, dim3(ffn_grid), dim3(I8_THREADS), smem_bytes, st, p, mode == 0 ? maps_x : maps_h);
+            launch_chained(kern, dim3(ffn_grid), dim3(i8_threads(nf)), smem_bytes, st, p, mode == 0 ? maps_x : maps_h);
             return cudaSuccess;
         };
-#define I8_KERNEL(GS_, WP_) std::integral_constant<decltype(&ffn_i8_kernel<GS_, WP_>), &ffn_i8_kernel<GS_, WP_>>{}
+#define I8_KERNEL(GS_, WP_, NF_) std::integral_constant<decltype(&ffn_i8_kernel<GS_, WP_, NF_>), &ffn_i8_kernel<GS_, WP_, NF_>>{}
+#define I8_LAUNCH(GS_, WP_) (nf == 1 ? launch(I8_KERNEL(GS_, WP_, 1)) : launch(I8_KERNEL(GS_, WP_, 2)))
         cudaError_t e;
-        if (D.g == 128 && wpack == 0x4112) e = launch(I8_KERNEL(128, 0x4112));        // {2,3,4,8}
-        else if (D.g == 128 && wpack == 0x422) e = launch(I8_KERNEL(128, 0x422));     // {2,4,8}
-        else if (D.g == 128 && wpack == 0x1115) e = launch(I8_KERNEL(128, 0x1115));   // {5,6,7,8}: the 5-bit step stored as 4 + 1
-        else if (D.g == 128) e = launch(I8_KERNEL(128, 0));
-        else e = launch(I8_KERNEL(64, 0));
+        if (D.g == 128 && wpack == 0x4112) e = I8_LAUNCH(128, 0x4112);        // {2,3,4,8}
+        else if (D.g == 128 && wpack == 0x422) e = I8_LAUNCH(128, 0x422);     // {2,4,8}
+        else if (D.g == 128 && wpack == 0x1115) e = I8_LAUNCH(128, 0x1115);   // {5,6,7,8}: the 5-bit step stored as 4 + 1
+        else if (D.g == 128) e = I8_LAUNCH(128, 0);
+        else e = I8_LAUNCH(64, 0);
+#undef I8_LAUNCH
 #undef I8_KERNEL
         if (e != cudaSuccess) return e;
         e = cudaGetLastError();
