@@ -362,6 +362,15 @@ def test_other_width_lists_on_the_tensor_core_paths(B, bits, g):
     assert cross < TOL and err < TOL, (cross, err)
 
 
+@pytest.mark.parametrize("bits,g,T", [((2, 3, 4, 8), 128, 24), ((2, 4, 8), 128, 20), ((5, 6, 7, 8), 128, 24),
+                                      ((2, 3, 4), 64, 22)])
+def test_few_tokens_per_expert_on_average_but_one_crowded_expert(B, bits, g, T):
+    # at most 12 tokens per expert on average: the decode kernel runs with ONE fold warpgroup, which must then fold
+    # every token block of a full unit (expert 0 gets all T tokens: more than four blocks of four slots)
+    cross, err = small_layer_case(B, d=256, F=256, E=4, k=2, g=g, bits=bits, T=T, one_expert=True)
+    assert cross < TOL and err < TOL, (cross, err)
+
+
 def test_all_tokens_on_one_expert_and_shared_experts(B):
     # 80 tokens all choose expert 0 (units beyond the per-unit token cap), one shared expert on top
     cross, err = small_layer_case(B, d=256, F=256, E=4, k=2, g=128, bits=(2, 3, 4, 8), T=80, n_shared=1,
