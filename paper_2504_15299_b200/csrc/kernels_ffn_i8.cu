@@ -645,7 +645,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32)) << 16;
         const uint32_t d_base = d_tmem + lane_addr;
         uint32_t gc = 0;                           // groups folded so far
-        uint32_t ws = 0, wph = 0, bs = 0, bph = 0; // ring positions and phases
+        uint32_t ws = 0, bs = 0;                   // ring positions
         uint32_t w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes;
         const float s1_factor = __int_as_float((127 - (p.L.top - p.L.b1)) << 23);
         for (uint32_t qi = 0;; ++qi) {
@@ -691,29 +691,33 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
 
             for (int G = ii.g0; G < ii.g1; G += GPS) {
                 const int ng = min(GPS, ii.g1 - G);
-                // the scales of this stage's groups, then the stage is released as far as this warpgroup goes
-                mbar_wait_blk(W_FULL(ws), wph);
+                // The fold waits for one thing only, the finished accumulator of a group: its products were issued after
+                // the issuer had seen the stage's activation tile arrive and after the unpack warps had seen the stage's
+                // packed blocks arrive, so both are in shared memory by then (the fold still releases both stages: they are
+                // not refilled before it has read its part of them).
                 uint32_t meta[GPS];
-#pragma unroll
-                for (int sub = 0; sub < GPS; ++sub)
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta[sub])
-                                 : "r"(w_addr + (uint32_t)(2 * sub) * (uint32_t)p.L.block_bytes + 4u * rr));
-                __syncwarp();
-                if (lane == 0) mbar_arrive(W_EMPTY(ws));
-                w_addr += w_slot_bytes;
-                if (++ws == (uint32_t)nsw) { ws = 0; wph ^= 1; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
-                mbar_wait_blk(B_FULL(bs), bph);
 #pragma unroll
                 for (int sub = 0; sub < GPS; ++sub) {
                     if (sub < ng) {
                         const int buf = gc & 1;
+                        mbar_wait_blk(D_FULL(buf), (gc >> 1) & 1);
+                        tc_fence_after();
+                        if (sub == 0) {
+                            // the scales of this stage's groups, then the stage is released as far as this warp goes
+#pragma unroll
+                            for (int s2 = 0; s2 < GPS; ++s2)
+                                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(meta[s2])
+                                             : "r"(w_addr + (uint32_t)(2 * s2) * (uint32_t)p.L.block_bytes + 4u * rr));
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(W_EMPTY(ws));
+                            w_addr += w_slot_bytes;
+                            if (++ws == (uint32_t)nsw) { ws = 0; w_addr = wbuf + (uint32_t)blk * (uint32_t)p.L.block_bytes; }
+                        }
                         const __half2 mh = as_h2(meta[sub]);
                         const float s1p = __low2float(mh) * s1_factor;
                         const float lo = __high2float(mh);
                         const uint32_t xk_addr = xkbuf + (bs * 2 + sub) * I8_XK_BYTES;
                         const uint32_t d_addr = d_base + buf * I8_D_COLS;
-                        mbar_wait_blk(D_FULL(buf), (gc >> 1) & 1);
-                        tc_fence_after();
                         auto fold_block = [&](int b, const uint32_t (&v)[8]) {
                             float xk[8];
                             const uint32_t a = xk_addr + 32u * blk_r[b];
@@ -748,7 +752,7 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(B_EMPTY(bs));
-                if (++bs == I8_NSB) { bs = 0; bph ^= 1; }
+                if (++bs == I8_NSB) bs = 0;
             }
 
             // ---- write out: y = sigma * acc (out of line: its registers are not the loop's) ----
