@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, each from one ncu capture of
 # the same workload through this script (the summaries of those captures are committed beside the numbers
 # they come from); key = workload:tokens:stage:path
-NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1042693176, "mixtral_decode:T64:down:auto": 536510960,
-               "mixtral_prefill:T2048:gate_up:auto": 1651062560, "mixtral_prefill:T2048:down:auto": 1008406424,
-               "finegrained:T256:gate_up:auto": 463764480, "finegrained:T256:down:auto": 234219776}
+NCU_TRAFFIC = {"mixtral_decode:T64:gate_up:auto": 1042948288, "mixtral_decode:T64:down:auto": 536264624,
+               "mixtral_prefill:T2048:gate_up:auto": 1649747408, "mixtral_prefill:T2048:down:auto": 1008871152,
+               "finegrained:T256:gate_up:auto": 462040064, "finegrained:T256:down:auto": 234176768}
 
 
 def measured_peaks():
