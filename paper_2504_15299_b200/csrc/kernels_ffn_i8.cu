@@ -342,12 +342,12 @@ ffn_i8_kernel(const __grid_constant__ I8Params p, const __grid_constant__ TmaMap
     if (threadIdx.x == 0) {
         for (int i = 0; i < I8_MAX_NSW; ++i) { mbar_init(W_FULL(i), 1); mbar_init(W_EMPTY(i), 4 + 4 * NF); }
         // an activation stage is released by the MMA issuer (its products have read the tile) and by
-        // the eight folding warps (they have read the sums)
+        // the fold warps (they have read the sums)
         for (int i = 0; i < I8_NSB; ++i) { mbar_init(B_FULL(i), 1); mbar_init(B_EMPTY(i), 1 + 4 * NF); }
         for (int wg = 0; wg < 2; ++wg)
             for (int sl = 0; sl < 2; ++sl) { mbar_init(A_FULL(wg, sl), 4); mbar_init(A_EMPTY(wg, sl), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(D_FULL(b), 1); mbar_init(D_EMPTY(b), 4 * NF); }
-        // a queue entry is released by the issuer warp, the four unpack warps and the eight fold warps
+        // a queue entry is released by the issuer warp, the four unpack warps and the fold warps
         for (int i = 0; i < I8_NSQ; ++i) { mbar_init(SQ_FULL(i), 1); mbar_init(SQ_EMPTY(i), 5 + 4 * NF); }
         *abort_flag = 0;
         *reinterpret_cast<int32_t**>(reinterpret_cast<uint8_t*>(bars) + 496) = p.status;
@@ -908,7 +908,7 @@ i8_prep_kernel(MoeDims D, RouteBufs R, I8Unit* units, int* n_units, int32_t* pad
                 for (int k = 0; k < 4; ++k)
                     if (mk == k) mine[k] = u;
             }
-            // work per group: one warpgroup unpacks every operand, each of the other two folds half of the blocks
+            // work per group: one warpgroup unpacks every operand, the fold warps take the blocks (half each when there are two warpgroups)
             cost[nu] = 80 * (u.kmax + 1) + 25 * ((u.nblk + 1) / 2);
         }
     }
